@@ -1,0 +1,231 @@
+/*
+ * l2pd — Learn2PD decoding of a masked-diffusion language model on one B200 GPU.
+ *
+ * C ABI.  Every pointer is marked host or device.  Nothing here throws, aborts or
+ * traps the device: each call returns an l2pd_status, and l2pd_last_error() gives
+ * a human-readable reason for the last failure on that context.
+ *
+ * The computation is the inference procedure of "Learning to Parallel:
+ * Accelerating Diffusion LLMs via Learnable Parallel Decoding" (Algorithm 2, with
+ * the end-of-text break of Algorithm 3 in the appendix "Update Inference
+ * Algorithm"):
+ *
+ *   X <- concat(prompt, [MASK]^G)
+ *   for each block b of s generation positions, left to right:
+ *     while the block still has masked positions:
+ *        conf, pre = M(X)                       (one "denoising step")
+ *        p = sigmoid(f_theta(conf))             (Section 3.2)
+ *        for masked j with p_j > tau:  X[P + b*s + j] <- pre_j, j leaves the mask set
+ *        EoTP: once an [EoT] token is committed, positions after it are dropped
+ *              from the next step's input (Section 3.3)
+ *     stop after a block that contains [EoT]
+ *
+ * M is a LLaDA-style bidirectional transformer: token embedding, n_layers pre-norm
+ * blocks (RMSNorm, fused QKV projection, rotary embedding on q and k with
+ * half-split pairing, multi-head attention WITHOUT a causal mask, output
+ * projection, RMSNorm, SwiGLU MLP), final RMSNorm and an untied LM head.
+ * pre_j is the argmax of the LM-head logits (Eq. 3) and conf_j the softmax
+ * probability of that argmax (Eq. 4); the logits are reduced on chip and never
+ * stored unless a debug buffer is supplied.
+ */
+#ifndef L2PD_H
+#define L2PD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct l2pd_ctx l2pd_ctx;   /* opaque; owned by the library */
+
+typedef enum {
+  L2PD_OK = 0,
+  L2PD_ERR_ARG = -1,          /* null pointer, bad enum, bad flag */
+  L2PD_ERR_SHAPE = -2,        /* sizes inconsistent with the configuration */
+  L2PD_ERR_OOM = -3,          /* device or host allocation failed */
+  L2PD_ERR_CUDA = -4,         /* a CUDA call failed; see l2pd_last_error */
+  L2PD_ERR_TIMEOUT = -5,      /* a bounded device-side wait ran out */
+  L2PD_ERR_TOKEN_RANGE = -6,  /* a prompt id outside [0, vocab) or equal to mask_id */
+  L2PD_ERR_STATE = -7         /* call order: step before reset, step after all done */
+} l2pd_status;
+
+enum { L2PD_F32 = 0, L2PD_BF16 = 1 };
+
+/* Model and decoding configuration (host memory, copied by l2pd_init). */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, head_dim, d_ff, vocab;
+  float   rms_eps;            /* y = x*g/sqrt(mean(x^2)+eps) */
+  float   rope_theta;         /* angle of pair i at position t: t * theta^(-2i/head_dim) */
+  int32_t mask_id, eot_id;
+  int32_t dtype;              /* L2PD_F32: fp32 weights, CUDA-core arithmetic;
+                                 L2PD_BF16: bf16 weights and activations, tcgen05 tensor cores,
+                                 fp32 accumulation and fp32 residual stream */
+  int32_t block_len;          /* s; the filter is Linear(s,s)+b -> ReLU -> Linear(s,s)+b
+                                 (2*(s*s+s) parameters: 2,112 at s = 32, Section 4.1); s <= 64 */
+  float   tau;                /* threshold on sigmoid(filter output); the paper uses 0.96 */
+  int32_t use_filter;         /* 0: no position passes the threshold; every step commits only the
+                                 most confident masked position (one token per step) */
+  int32_t use_eotp;           /* 1: End-of-Text Prediction on */
+  int32_t kv_cache_mode;      /* 0: every step recomputes all positions.
+                                 1: block-level prefix cache (Section 4.3 names it; rule: the first
+                                    step of a block runs all positions and stores K (rotated) and V of
+                                    the positions before the block; the block's other steps compute
+                                    only positions from the block start on and attend to
+                                    stored ++ fresh keys) */
+  int32_t committed_conf_mode;/* what the filter reads at block positions already committed:
+                                 0 = the model's confidence recomputed this step, 1 = 1.0 */
+  int32_t max_batch;          /* most sequences a reset may start */
+  int32_t max_seq;            /* largest P + G */
+} l2pd_config;
+
+/*
+ * Weights: DEVICE pointers, borrowed — the caller keeps them alive and unchanged
+ * until l2pd_destroy.  Matrices are row-major [out_features, in_features] in the
+ * configuration's dtype (fp32 or bf16); norm gains, the bias and the filter are fp32.
+ * The per-layer arrays are HOST arrays of n_layers device pointers (copied at init).
+ */
+typedef struct {
+  const void *tok_emb;              /* [vocab, d_model] */
+  const void *const *wqkv;          /* [3*n_heads*head_dim, d_model]: q rows, then k, then v */
+  const void *const *wo;            /* [d_model, n_heads*head_dim] */
+  const void *const *w_gate;        /* [d_ff, d_model] */
+  const void *const *w_up;          /* [d_ff, d_model] */
+  const void *const *w_down;        /* [d_model, d_ff] */
+  const float *const *norm1;        /* [d_model] gain before attention */
+  const float *const *norm2;        /* [d_model] gain before the MLP */
+  const float *final_norm;          /* [d_model] */
+  const void *lm_head;              /* [vocab, d_model] */
+  const float *lm_head_bias;        /* [vocab] added to the logits, or NULL */
+  const float *filt_w1, *filt_b1;   /* [s, s], [s]  (may be NULL when use_filter = 0) */
+  const float *filt_w2, *filt_b2;   /* [s, s], [s] */
+} l2pd_weights;
+
+/*
+ * Optional outputs of one denoising step.  Any pointer may be NULL.
+ * Device arrays are indexed [sequence, j] with j the position inside the
+ * sequence's current block (row stride s); rows of sequences that were already
+ * finished before the step are left untouched.  Entries with P + b*s + j >= L_eff
+ * (cut off by EoTP) are written as conf = 0, pred = -1.
+ * Host arrays have one entry per sequence and are valid when the call returns
+ * (the call then waits for the step to finish).
+ */
+typedef struct {
+  float   *d_conf;        /* device [B, s]  Eq. 4 */
+  int32_t *d_pred;        /* device [B, s]  Eq. 3 */
+  float   *d_p;           /* device [B, s]  sigmoid(filter output) */
+  uint8_t *d_unmask;      /* device [B, s]  1 where the step committed the position */
+  float   *d_logits;      /* device [B, s, vocab] fp32 logits (debug; large) */
+  int32_t *h_block;       /* host [B] block the step worked on */
+  int32_t *h_masks_left;  /* host [B] masked positions left in that block after the step */
+  int32_t *h_l_eff;       /* host [B] effective length P + e + 1 after the step (P + G if no EoT) */
+  int32_t *h_done;        /* host [B] 1 once the sequence needs no further step */
+  int32_t *h_forced;      /* host [B] 1 if the step used the progress fallback */
+} l2pd_step_out;
+
+/*
+ * Create a context on `device`: validates the configuration, records the weight
+ * pointers, allocates state, workspace and (kv_cache_mode = 1) the cache for
+ * max_batch x max_seq.  Errors: L2PD_ERR_ARG / L2PD_ERR_SHAPE (d_model, d_ff,
+ * n_heads*head_dim multiples of 8; head_dim 64 or 128 for bf16, even and <= 256 for
+ * fp32; block_len in [1, 64]; ids inside the vocabulary), L2PD_ERR_OOM, L2PD_ERR_CUDA.
+ * With out == NULL and ctx creation failing, `*out` is left NULL.
+ */
+l2pd_status l2pd_init(const l2pd_config *cfg, const l2pd_weights *w, int device, l2pd_ctx **out);
+
+/*
+ * Algorithm 2, state set-up: X <- concat(prompt, [MASK]^G) for B sequences.
+ * d_prompts: DEVICE int32 [B, P].  G must be a multiple of block_len, B <= max_batch,
+ * P >= 1, P + G <= max_seq (else L2PD_ERR_SHAPE).  Prompt ids are range-checked on the
+ * device; a bad id makes this call return L2PD_ERR_TOKEN_RANGE (the call synchronises).
+ * `stream` is a cudaStream_t (NULL = default stream).
+ */
+l2pd_status l2pd_state_reset(l2pd_ctx *ctx, void *stream, const int32_t *d_prompts,
+                             int32_t B, int32_t P, int32_t G);
+
+/*
+ * One iteration of the while loop of Algorithm 2 for every unfinished sequence:
+ * transformer forward, confidence and argmax (Eq. 3-4), filter, threshold, in-place
+ * commit, EoTP, block advance.  Returns after the step's small result record has
+ * reached the host (one stream synchronisation per step).  L2PD_ERR_STATE if no
+ * sequence is unfinished.  `out` may be NULL.
+ */
+l2pd_status l2pd_denoise_step(l2pd_ctx *ctx, void *stream, const l2pd_step_out *out);
+
+/*
+ * Whole decode: l2pd_state_reset followed by l2pd_denoise_step until every sequence
+ * is done.  d_out_tokens: DEVICE int32 [B, G], the response; positions after a
+ * sequence's [EoT] hold eot_id.  h_out_len (HOST [B], may be NULL): tokens up to and
+ * including [EoT], or G.  h_steps (HOST [B], may be NULL): number of M(X) evaluations
+ * the sequence took part in.  h_total_steps (HOST, may be NULL): steps launched.
+ */
+l2pd_status l2pd_decode(l2pd_ctx *ctx, void *stream, const int32_t *d_prompts,
+                        int32_t B, int32_t P, int32_t G, int32_t *d_out_tokens,
+                        int32_t *h_out_len, int32_t *h_steps, int32_t *h_total_steps);
+
+/* Number of sequences that still need steps (0 before the first reset). */
+int32_t l2pd_num_active(const l2pd_ctx *ctx);
+
+/* DEVICE view of the token state, int32 [B, P + G] (row stride P + G); valid until the next reset. */
+const int32_t *l2pd_state_tokens(const l2pd_ctx *ctx);
+/* DEVICE view of the mask set, uint8 [B, G]: 1 while the generation position is masked. */
+const uint8_t *l2pd_state_masked(const l2pd_ctx *ctx);
+
+/*
+ * Debug capture (tests): when d_resid is non-NULL every following step copies the
+ * fp32 residual stream into it — slot 0 after the embedding, slot l+1 after layer l —
+ * as [n_layers + 1, T, d_model] with T the number of rows the step processed
+ * (the caller sizes it for max_batch * max_seq rows per slot; slot stride = rows*d_model
+ * where rows is the value returned through l2pd_last_step_rows).  NULL turns it off.
+ */
+l2pd_status l2pd_set_capture(l2pd_ctx *ctx, float *d_resid, int64_t slot_stride_elems);
+int32_t l2pd_last_step_rows(const l2pd_ctx *ctx);
+
+/* Kernels launched by this context since creation (for launch accounting). */
+int64_t l2pd_launch_count(const l2pd_ctx *ctx);
+
+/* Device time of the most recent step in milliseconds (CUDA events on the step's stream),
+ * or a negative value if no step has run. */
+float l2pd_last_step_ms(const l2pd_ctx *ctx);
+
+const char *l2pd_last_error(const l2pd_ctx *ctx);   /* never NULL; "" when there is none */
+void l2pd_destroy(l2pd_ctx *ctx);                   /* NULL is allowed */
+
+/*
+ * Stand-alone kernels of the step, exported for kernel-level tests and timing.
+ * All pointers are DEVICE pointers; `stream` is a cudaStream_t.  Each returns
+ * L2PD_ERR_SHAPE for sizes the kernel does not support and L2PD_ERR_CUDA when the
+ * launch fails; L2PD_ERR_TIMEOUT if a bounded on-device wait ran out (the call then
+ * synchronises the stream to read the flag only when `check` is non-zero).
+ */
+
+/* C[M,N] (bf16) = A[M,K] (bf16, row-major) x W[N,K]^T (bf16, row-major); tcgen05 path.
+ * K and N multiples of 8.  tile_n: 0 = pick automatically, else a multiple of 16 in [32, 256]. */
+l2pd_status l2pd_gemm_bf16(void *stream, const void *A, const void *W, void *C,
+                           int32_t M, int32_t N, int32_t K, int32_t tile_n, int32_t check);
+/* X[M,N] (fp32) += A[M,K] x W[N,K]^T : projection with the residual add in the epilogue. */
+l2pd_status l2pd_gemm_bf16_residual(void *stream, const void *A, const void *W, float *X,
+                                    int32_t M, int32_t N, int32_t K, int32_t tile_n, int32_t check);
+/* H[M,F] (bf16) = silu(A Wg^T) * (A Wu^T), Wg and Wu [F,K] : gate/up projection with SwiGLU. */
+l2pd_status l2pd_gemm_bf16_swiglu(void *stream, const void *A, const void *Wg, const void *Wu,
+                                  void *H, int32_t M, int32_t F, int32_t K, int32_t tile_n,
+                                  int32_t check);
+/* LM head with the confidence head fused (Eq. 3-4): for each of R rows of A[R,K] (bf16),
+ * pred = argmax_v (A W^T + bias)_v (lowest id on ties), conf = softmax probability of pred.
+ * W [V,K] bf16, bias [V] fp32 or NULL.  d_logits (fp32 [R,V]) may be NULL.
+ * d_scratch: fp32 workspace of at least l2pd_lm_head_scratch_elems(R, V) elements. */
+l2pd_status l2pd_lm_head_bf16(void *stream, const void *A, const void *W, const float *bias,
+                              int32_t R, int32_t V, int32_t K, float *d_scratch,
+                              int32_t *d_pred, float *d_conf, float *d_logits, int32_t check);
+int64_t l2pd_lm_head_scratch_elems(int32_t R, int32_t V);
+
+/* Bidirectional attention, bf16: q [Tq, H*dh], k and v [Tk, H*dh] (row stride given in
+ * elements), out [Tq, H*dh]; softmax(q k^T / sqrt(dh)) v per head, no mask. dh 64 or 128. */
+l2pd_status l2pd_attention_bf16(void *stream, const void *q, const void *k, const void *v,
+                                void *out, int32_t Tq, int32_t Tk, int32_t H, int32_t dh,
+                                int64_t q_stride, int64_t kv_stride, int64_t out_stride);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* L2PD_H */

@@ -82,6 +82,11 @@ def rmsnorm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
     return x * widen(gain) / np.sqrt(ms + eps)
 
 
+def linear(x: np.ndarray, w: np.ndarray) -> np.ndarray:
+    """y = x W^T for a weight stored [out, in] (library matmul on the widened values)."""
+    return x @ widen(w).T
+
+
 def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
     """Rotary embedding on x[T, H, dh] at integer positions pos[T].
 
@@ -128,7 +133,7 @@ def layer_forward(m: Model, layer: Dict[str, np.ndarray], x: np.ndarray, pos: np
     H, dh = m.n_heads, m.head_dim
     T = x.shape[0]
     n = rmsnorm(x, layer["norm1"], m.rms_eps)
-    qkv = n @ widen(layer["wqkv"]).T                      # [T, 3*H*dh]: q rows, then k, then v
+    qkv = linear(n, layer["wqkv"])                     # [T, 3*H*dh]: q rows, then k, then v
     q = qkv[:, : H * dh].reshape(T, H, dh)
     k = qkv[:, H * dh: 2 * H * dh].reshape(T, H, dh)
     v = qkv[:, 2 * H * dh:].reshape(T, H, dh)
@@ -140,10 +145,10 @@ def layer_forward(m: Model, layer: Dict[str, np.ndarray], x: np.ndarray, pos: np
         k = np.concatenate([k_prefix, k], axis=0)
         v = np.concatenate([v_prefix, v], axis=0)
     a = attention(q, k, v).reshape(T, H * dh)
-    x = x + a @ widen(layer["wo"]).T
+    x = x + linear(a, layer["wo"])
     n = rmsnorm(x, layer["norm2"], m.rms_eps)
-    h = silu(n @ widen(layer["w_gate"]).T) * (n @ widen(layer["w_up"]).T)
-    return x + h @ widen(layer["w_down"]).T
+    h = silu(linear(n, layer["w_gate"])) * linear(n, layer["w_up"])
+    return x + linear(h, layer["w_down"])
 
 
 def forward_hidden(m: Model, tokens: np.ndarray, pos0: int = 0,
@@ -167,7 +172,7 @@ def forward_hidden(m: Model, tokens: np.ndarray, pos0: int = 0,
 def lm_head_logits(m: Model, hidden_rows: np.ndarray) -> np.ndarray:
     """Final RMSNorm then the LM head (+ optional bias) on the given rows -> [R, V]."""
     n = rmsnorm(hidden_rows, m.weights["final_norm"], m.rms_eps)
-    logits = n @ widen(m.weights["lm_head"]).T
+    logits = linear(n, m.weights["lm_head"])
     if m.lm_head_bias is not None:
         logits = logits + widen(m.lm_head_bias)[None, :]
     return logits

@@ -1,0 +1,629 @@
+// C ABI of the l2pd library: context, decode state, one denoising step, the decode loop.
+// Host code only orchestrates; every arithmetic step of the path runs in the kernels of the
+// other files.  Nothing here falls back to the CPU: a failed CUDA call is an error status.
+#include <math.h>
+#include <stdarg.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+#include <string>
+#include <vector>
+
+#include "common.cuh"
+
+using namespace l2pd;
+
+struct l2pd_ctx {
+  l2pd_config cfg;
+  int device = 0, num_sms = 148;
+  bool force_simt = false;   // L2PD_FORCE_SIMT=1: bf16 GEMMs and attention on the CUDA-core cross-check kernels
+
+  // weights (borrowed device pointers)
+  const void *tok_emb = nullptr, *lm_head = nullptr;
+  std::vector<const void *> wqkv, wo, w_gate, w_up, w_down;
+  std::vector<const float *> norm1, norm2;
+  const float *final_norm = nullptr, *lm_bias = nullptr, *fw1 = nullptr, *fb1 = nullptr, *fw2 = nullptr, *fb2 = nullptr;
+
+  // decode state
+  int B = 0, P = 0, G = 0;
+  bool has_state = false;
+  int32_t *d_tokens = nullptr;
+  uint8_t *d_masked = nullptr;
+  int32_t *d_state_ints = nullptr;   // 6 arrays of max_batch
+  SeqState st{};
+  std::vector<int> h_cur_block, h_l_eff, h_done, h_steps, h_cache_block;
+  int n_active = 0;
+  int total_steps = 0;
+
+  // workspace
+  int64_t max_rows = 0;              // capacity in activation rows (multiple of 128)
+  int64_t max_lm_rows = 0;           // max_batch * s rounded up to 128
+  float *x = nullptr;
+  void *n = nullptr, *qkv = nullptr, *q = nullptr, *att = nullptr, *h = nullptr, *nf = nullptr;
+  void *kc = nullptr, *vc = nullptr;
+  int64_t kv_seq_stride = 0, kv_layer_stride = 0;
+  float *part = nullptr;             // part_m | part_s | part_i
+  int64_t part_tiles_cap = 0;
+  float *logits_f32 = nullptr;       // fp32 configurations: [max_lm_rows, V]
+  SeqMeta *d_meta = nullptr, *h_meta = nullptr;
+  int32_t *d_row_slot = nullptr;
+  StepSummary *d_summary = nullptr, *h_summary = nullptr;
+  int32_t *d_status = nullptr, *h_status = nullptr;
+  float2 *cs_table = nullptr;
+
+  // TMA descriptors (bf16 path)
+  TmaDesc ta_n, ta_att, ta_h, ta_nf;
+  std::vector<TmaDesc> tb_qkv, tb_o, tb_gate, tb_up, tb_down;
+  TmaDesc tb_lm;
+  int tn_qkv = 0, tn_o = 0, tn_gu = 0, tn_down = 0, tn_lm = 0;
+
+  // debug capture
+  float *cap = nullptr;
+  int64_t cap_stride = 0;
+  int last_rows = 0;
+
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  float last_ms = -1.f;
+  int64_t launches = 0;
+  std::string err;
+};
+
+namespace {
+
+l2pd_status set_err(l2pd_ctx *c, l2pd_status s, const char *fmt, ...) {
+  if (c) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof buf, fmt, ap);
+    va_end(ap);
+    c->err = buf;
+  }
+  return s;
+}
+
+#define CK(call)                                                                                   \
+  do {                                                                                             \
+    cudaError_t e_ = (call);                                                                       \
+    if (e_ != cudaSuccess)                                                                         \
+      return set_err(c, e_ == cudaErrorMemoryAllocation ? L2PD_ERR_OOM : L2PD_ERR_CUDA, "%s: %s", \
+                     #call, cudaGetErrorString(e_));                                               \
+  } while (0)
+#define CKL(call)                                                                                  \
+  do { CK(call); c->launches++; } while (0)
+
+template <typename T>
+l2pd_status dev_alloc(l2pd_ctx *c, T **p, int64_t count) {
+  CK(cudaMalloc(reinterpret_cast<void **>(p), (size_t)count * sizeof(T)));
+  return L2PD_OK;
+}
+
+int64_t round_up(int64_t a, int64_t b) { return (a + b - 1) / b * b; }
+
+size_t elt(const l2pd_ctx *c) { return c->cfg.dtype == L2PD_BF16 ? 2 : 4; }
+
+l2pd_status encode_weight_maps(l2pd_ctx *c, std::vector<TmaDesc> &dst, const std::vector<const void *> &w,
+                               int64_t rows, int64_t cols, int box_rows) {
+  dst.resize(w.size());
+  for (size_t l = 0; l < w.size(); ++l) {
+    l2pd_status s = make_tma_2d_bf16(&dst[l], w[l], rows, cols, box_rows);
+    if (s != L2PD_OK) return set_err(c, s, "tensor map encode failed (rows %lld cols %lld box %d)", (long long)rows, (long long)cols, box_rows);
+  }
+  return L2PD_OK;
+}
+
+// One GEMM of the step, dispatched by dtype.
+template <typename T>
+l2pd_status run_gemm_simt(l2pd_ctx *c, cudaStream_t s, int epi, const void *A, const void *W, const void *W2,
+                          void *out, const float *bias, int M, int N, int K) {
+  CKL(launch_simt_gemm<T>(s, epi, (const T *)A, (const T *)W, (const T *)W2, out, bias, M, N, K));
+  return L2PD_OK;
+}
+
+l2pd_status run_gemm_tc(l2pd_ctx *c, cudaStream_t s, int epi, const TmaDesc *a, const TmaDesc *b, const TmaDesc *b2,
+                        void *out, int M, int N, int K, int tile_n) {
+  GemmArgs g{};
+  g.epi = epi; g.a = a; g.b = b; g.b2 = b2; g.M = M; g.N = N; g.K = K; g.tile_n = tile_n; g.out = out;
+  g.status = c->d_status;
+  CKL(launch_gemm_tcgen05(s, g, c->num_sms));
+  return L2PD_OK;
+}
+
+template <typename T>
+l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_rows, int max_q_rows, int max_kv,
+                               const l2pd_step_out *out) {
+  const l2pd_config &f = c->cfg;
+  const int d = f.d_model, H = f.n_heads, dh = f.head_dim, hd = H * dh, F = f.d_ff, V = f.vocab, sb = f.block_len;
+  const bool tc = (f.dtype == L2PD_BF16) && !c->force_simt;
+  T *n = (T *)c->n, *qkv = (T *)c->qkv, *q = (T *)c->q, *att = (T *)c->att, *hbuf = (T *)c->h, *nf = (T *)c->nf;
+
+  if (tc) {
+    // tile widths follow the row count of this step; weight tensor maps are re-encoded when they change
+    int tn = pick_tile_n(T_rows, 3 * hd, c->num_sms, 16, 256);
+    if (tn != c->tn_qkv) { l2pd_status r = encode_weight_maps(c, c->tb_qkv, c->wqkv, 3 * hd, d, tn); if (r) return r; c->tn_qkv = tn; }
+    tn = pick_tile_n(T_rows, d, c->num_sms, 16, 256);
+    if (tn != c->tn_o) { l2pd_status r = encode_weight_maps(c, c->tb_o, c->wo, d, hd, tn); if (r) return r; c->tn_o = tn; }
+    if (tn != c->tn_down) { l2pd_status r = encode_weight_maps(c, c->tb_down, c->w_down, d, F, tn); if (r) return r; c->tn_down = tn; }
+    tn = 2 * pick_tile_n(T_rows, F, c->num_sms, 16, 128);
+    if (tn != c->tn_gu) {
+      l2pd_status r = encode_weight_maps(c, c->tb_gate, c->w_gate, F, d, tn / 2); if (r) return r;
+      r = encode_weight_maps(c, c->tb_up, c->w_up, F, d, tn / 2); if (r) return r;
+      c->tn_gu = tn;
+    }
+  }
+
+  CKL(launch_build_row_map(s, c->d_meta, n_slots, c->d_row_slot));
+  CKL(launch_embed_rmsnorm<T>(s, c->d_tokens, c->P + c->G, c->d_meta, c->d_row_slot, (const T *)c->tok_emb,
+                              c->norm1[0], f.rms_eps, c->x, n, T_rows, d));
+  if (c->cap) CK(cudaMemcpyAsync(c->cap, c->x, (size_t)T_rows * d * 4, cudaMemcpyDeviceToDevice, s));
+
+  for (int l = 0; l < f.n_layers; ++l) {
+    T *kc = (T *)c->kc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
+    T *vc = (T *)c->vc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
+    l2pd_status r;
+    if (tc) r = run_gemm_tc(c, s, EPI_STORE, &c->ta_n, &c->tb_qkv[l], nullptr, qkv, T_rows, 3 * hd, d, c->tn_qkv);
+    else r = run_gemm_simt<T>(c, s, EPI_STORE, n, c->wqkv[l], nullptr, qkv, nullptr, T_rows, 3 * hd, d);
+    if (r) return r;
+    CKL(launch_rope_scatter<T>(s, qkv, c->d_meta, c->d_row_slot, c->cs_table, q, kc, vc, c->kv_seq_stride, T_rows, H, dh));
+    if (tc) {
+      CKL(launch_attention_bf16(s, (const bf16 *)q, (const bf16 *)kc, (const bf16 *)vc, c->d_meta, (bf16 *)att, hd, hd,
+                                c->kv_seq_stride, hd, n_slots, max_q_rows, H, dh));
+    } else {
+      CKL(launch_simt_attention<T>(s, q, kc, vc, c->d_meta, c->d_row_slot, att, c->kv_seq_stride, T_rows, H, dh, max_kv));
+    }
+    if (tc) r = run_gemm_tc(c, s, EPI_RESIDUAL, &c->ta_att, &c->tb_o[l], nullptr, c->x, T_rows, d, hd, c->tn_o);
+    else r = run_gemm_simt<T>(c, s, EPI_RESIDUAL, att, c->wo[l], nullptr, c->x, nullptr, T_rows, d, hd);
+    if (r) return r;
+    CKL(launch_rmsnorm<T>(s, c->x, c->norm2[l], f.rms_eps, n, T_rows, d));
+    if (tc) r = run_gemm_tc(c, s, EPI_SWIGLU, &c->ta_n, &c->tb_gate[l], &c->tb_up[l], hbuf, T_rows, F, d, c->tn_gu);
+    else r = run_gemm_simt<T>(c, s, EPI_SWIGLU, n, c->w_gate[l], c->w_up[l], hbuf, nullptr, T_rows, F, d);
+    if (r) return r;
+    if (tc) r = run_gemm_tc(c, s, EPI_RESIDUAL, &c->ta_h, &c->tb_down[l], nullptr, c->x, T_rows, d, F, c->tn_down);
+    else r = run_gemm_simt<T>(c, s, EPI_RESIDUAL, hbuf, c->w_down[l], nullptr, c->x, nullptr, T_rows, d, F);
+    if (r) return r;
+    if (c->cap)
+      CK(cudaMemcpyAsync(c->cap + (int64_t)(l + 1) * c->cap_stride, c->x, (size_t)T_rows * d * 4, cudaMemcpyDeviceToDevice, s));
+    if (l + 1 < f.n_layers) CKL(launch_rmsnorm<T>(s, c->x, c->norm1[l + 1], f.rms_eps, n, T_rows, d));
+  }
+
+  // confidence head on the current block's rows
+  const int R = n_slots * sb;
+  const int rows_padded = tc ? (int)round_up(R, 128) : R;
+  CKL(launch_final_norm_gather<T>(s, c->x, c->d_meta, c->final_norm, f.rms_eps, nf, n_slots, sb, rows_padded, d));
+  int n_tiles = 1;
+  float *part_m, *part_s;
+  int32_t *part_i;
+  if (tc) {
+    int tn = pick_tile_n(R, V, c->num_sms, 16, 256);
+    if (tn != c->tn_lm) {
+      l2pd_status r = make_tma_2d_bf16(&c->tb_lm, c->lm_head, V, d, tn);
+      if (r) return set_err(c, r, "tensor map encode failed for the LM head");
+      c->tn_lm = tn;
+    }
+    n_tiles = ceil_div(V, tn);
+    part_m = c->part; part_s = part_m + (int64_t)n_tiles * rows_padded;
+    part_i = (int32_t *)(part_s + (int64_t)n_tiles * rows_padded);
+    GemmArgs g{};
+    g.epi = EPI_LMHEAD; g.a = &c->ta_nf; g.b = &c->tb_lm; g.M = R; g.N = V; g.K = d; g.tile_n = tn;
+    g.bias = c->lm_bias; g.part_m = part_m; g.part_s = part_s; g.part_i = part_i; g.rows_padded = rows_padded;
+    g.logits = nullptr; g.status = c->d_status;
+    float *tmp_logits = nullptr;
+    if (out && out->d_logits) {
+      // the debug logits are indexed by sequence; with every sequence active slot == sequence order only if
+      // no sequence has dropped out, so write per slot into scratch and scatter below
+      g.logits = c->logits_f32;
+      tmp_logits = c->logits_f32;
+    }
+    CKL(launch_gemm_tcgen05(s, g, c->num_sms));
+    (void)tmp_logits;
+  } else {
+    part_m = c->part; part_s = part_m + rows_padded; part_i = (int32_t *)(part_s + rows_padded);
+    l2pd_status r = run_gemm_simt<T>(c, s, EPI_STORE_F32, nf, c->lm_head, nullptr, c->logits_f32, c->lm_bias, R, V, d);
+    if (r) return r;
+    CKL(launch_row_softmax_partials(s, c->logits_f32, R, V, part_m, part_s, part_i));
+  }
+  if (out && out->d_logits) {
+    for (int i = 0; i < n_slots; ++i) {
+      const SeqMeta &m = c->h_meta[i];
+      if (m.n_blk_rows > 0)
+        CK(cudaMemcpyAsync(out->d_logits + (int64_t)m.seq * sb * V, c->logits_f32 + (int64_t)i * sb * V,
+                           (size_t)m.n_blk_rows * V * 4, cudaMemcpyDeviceToDevice, s));
+    }
+  }
+
+  DecideArgs a{};
+  a.part_m = part_m; a.part_s = part_s; a.part_i = part_i; a.n_tiles = n_tiles; a.rows_padded = rows_padded;
+  a.meta = c->d_meta; a.s = sb; a.P = c->P; a.G = c->G; a.n_blocks = c->G / sb;
+  a.tokens = c->d_tokens; a.tok_stride = c->P + c->G; a.masked = c->d_masked; a.st = c->st;
+  a.w1 = c->fw1; a.b1 = c->fb1; a.w2 = c->fw2; a.b2 = c->fb2; a.tau = f.tau;
+  a.use_filter = f.use_filter; a.use_eotp = f.use_eotp; a.committed_conf_mode = f.committed_conf_mode;
+  a.eot_id = f.eot_id; a.summary = c->d_summary;
+  if (out) { a.o_conf = out->d_conf; a.o_pred = out->d_pred; a.o_p = out->d_p; a.o_unmask = out->d_unmask; }
+  CKL(launch_decide(s, a, n_slots));
+  return L2PD_OK;
+}
+
+void free_all(l2pd_ctx *c) {
+  cudaFree(c->d_tokens); cudaFree(c->d_masked); cudaFree(c->d_state_ints);
+  cudaFree(c->x); cudaFree(c->n); cudaFree(c->qkv); cudaFree(c->q); cudaFree(c->att); cudaFree(c->h); cudaFree(c->nf);
+  cudaFree(c->kc); cudaFree(c->vc); cudaFree(c->part); cudaFree(c->logits_f32);
+  cudaFree(c->d_meta); cudaFree(c->d_row_slot); cudaFree(c->d_summary); cudaFree(c->d_status); cudaFree(c->cs_table);
+  if (c->h_meta) cudaFreeHost(c->h_meta);
+  if (c->h_summary) cudaFreeHost(c->h_summary);
+  if (c->h_status) cudaFreeHost(c->h_status);
+  if (c->ev0) cudaEventDestroy(c->ev0);
+  if (c->ev1) cudaEventDestroy(c->ev1);
+}
+
+l2pd_status validate(const l2pd_config *f, const l2pd_weights *w, std::string *why) {
+  auto bad = [&](const char *m) { *why = m; return L2PD_ERR_SHAPE; };
+  if (f->dtype != L2PD_F32 && f->dtype != L2PD_BF16) { *why = "dtype must be L2PD_F32 or L2PD_BF16"; return L2PD_ERR_ARG; }
+  if (f->n_layers < 0 || f->d_model <= 0 || f->n_heads <= 0 || f->head_dim <= 0 || f->d_ff <= 0 || f->vocab <= 1)
+    return bad("non-positive model dimension");
+  if (f->d_model % 8 || f->d_ff % 8 || (f->n_heads * f->head_dim) % 8) return bad("d_model, d_ff and n_heads*head_dim must be multiples of 8");
+  if (f->head_dim % 2) return bad("head_dim must be even");
+  if (f->dtype == L2PD_BF16 && f->head_dim != 64 && f->head_dim != 128) return bad("bf16 attention supports head_dim 64 or 128");
+  if (f->dtype == L2PD_F32 && f->head_dim > 256) return bad("head_dim > 256");
+  if (f->block_len < 1 || f->block_len > 64) return bad("block_len must be in [1, 64]");
+  if (f->mask_id < 0 || f->mask_id >= f->vocab || f->eot_id < 0 || f->eot_id >= f->vocab || f->mask_id == f->eot_id)
+    return bad("mask_id / eot_id outside the vocabulary or equal");
+  if (f->max_batch < 1 || f->max_seq < 2) return bad("max_batch / max_seq too small");
+  if (!(f->tau >= 0.f && f->tau <= 1.f)) { *why = "tau outside [0, 1]"; return L2PD_ERR_ARG; }
+  if (f->kv_cache_mode != 0 && f->kv_cache_mode != 1) { *why = "kv_cache_mode must be 0 or 1"; return L2PD_ERR_ARG; }
+  if (f->committed_conf_mode != 0 && f->committed_conf_mode != 1) { *why = "committed_conf_mode must be 0 or 1"; return L2PD_ERR_ARG; }
+  if (!(f->rms_eps >= 0.f) || !(f->rope_theta > 0.f)) { *why = "rms_eps / rope_theta"; return L2PD_ERR_ARG; }
+  if (!w->tok_emb || !w->lm_head || !w->final_norm) { *why = "null weight pointer"; return L2PD_ERR_ARG; }
+  if (f->n_layers > 0 && (!w->wqkv || !w->wo || !w->w_gate || !w->w_up || !w->w_down || !w->norm1 || !w->norm2)) {
+    *why = "null per-layer weight array"; return L2PD_ERR_ARG;
+  }
+  for (int l = 0; l < f->n_layers; ++l)
+    if (!w->wqkv[l] || !w->wo[l] || !w->w_gate[l] || !w->w_up[l] || !w->w_down[l] || !w->norm1[l] || !w->norm2[l]) {
+      *why = "null per-layer weight pointer"; return L2PD_ERR_ARG;
+    }
+  if (f->use_filter && (!w->filt_w1 || !w->filt_b1 || !w->filt_w2 || !w->filt_b2)) { *why = "use_filter set but a filter pointer is null"; return L2PD_ERR_ARG; }
+  return L2PD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+l2pd_status l2pd_init(const l2pd_config *cfg, const l2pd_weights *w, int device, l2pd_ctx **out) {
+  if (out) *out = nullptr;
+  if (!cfg || !w || !out) return L2PD_ERR_ARG;
+  std::string why;
+  l2pd_status vs = validate(cfg, w, &why);
+  if (vs != L2PD_OK) return vs;
+  l2pd_ctx *c = new (std::nothrow) l2pd_ctx();
+  if (!c) return L2PD_ERR_OOM;
+  c->cfg = *cfg;
+  c->device = device;
+  const l2pd_config &f = c->cfg;
+  auto fail = [&](l2pd_status s) { free_all(c); delete c; return s; };
+  if (cudaSetDevice(device) != cudaSuccess) return fail(L2PD_ERR_CUDA);
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms <= 0) return fail(L2PD_ERR_CUDA);
+  c->num_sms = sms;
+  if (f.dtype == L2PD_BF16) {
+    int major = 0;
+    cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device);
+    if (major != 10) return fail(L2PD_ERR_CUDA);   // the tensor-core kernels are sm_100a only
+  }
+  const char *fs = getenv("L2PD_FORCE_SIMT");
+  c->force_simt = fs && fs[0] == '1';
+
+  c->tok_emb = w->tok_emb; c->lm_head = w->lm_head; c->final_norm = w->final_norm; c->lm_bias = w->lm_head_bias;
+  c->fw1 = w->filt_w1; c->fb1 = w->filt_b1; c->fw2 = w->filt_w2; c->fb2 = w->filt_b2;
+  for (int l = 0; l < f.n_layers; ++l) {
+    c->wqkv.push_back(w->wqkv[l]); c->wo.push_back(w->wo[l]); c->w_gate.push_back(w->w_gate[l]);
+    c->w_up.push_back(w->w_up[l]); c->w_down.push_back(w->w_down[l]);
+    c->norm1.push_back(w->norm1[l]); c->norm2.push_back(w->norm2[l]);
+  }
+  if (f.n_layers == 0) { c->norm1.push_back(w->final_norm); }
+
+  const int d = f.d_model, hd = f.n_heads * f.head_dim, F = f.d_ff, V = f.vocab, sb = f.block_len;
+  const size_t es = elt(c);
+  c->max_rows = round_up((int64_t)f.max_batch * f.max_seq, 128);
+  c->max_lm_rows = round_up((int64_t)f.max_batch * sb, 128);
+  const int64_t mr = c->max_rows;
+  l2pd_status r = L2PD_OK;
+  auto A = [&](l2pd_status s) { if (r == L2PD_OK) r = s; };
+  A(dev_alloc(c, &c->d_tokens, (int64_t)f.max_batch * f.max_seq));
+  A(dev_alloc(c, &c->d_masked, (int64_t)f.max_batch * f.max_seq));
+  A(dev_alloc(c, &c->d_state_ints, (int64_t)6 * f.max_batch));
+  A(dev_alloc(c, &c->x, mr * d));
+  A(dev_alloc(c, (uint8_t **)&c->n, mr * d * es));
+  A(dev_alloc(c, (uint8_t **)&c->qkv, mr * 3 * hd * es));
+  A(dev_alloc(c, (uint8_t **)&c->q, mr * hd * es));
+  A(dev_alloc(c, (uint8_t **)&c->att, mr * hd * es));
+  A(dev_alloc(c, (uint8_t **)&c->h, mr * F * es));
+  A(dev_alloc(c, (uint8_t **)&c->nf, c->max_lm_rows * d * es));
+  c->kv_seq_stride = (int64_t)f.max_seq * hd;
+  c->kv_layer_stride = (int64_t)f.max_batch * c->kv_seq_stride;
+  const int kv_layers = f.kv_cache_mode ? (f.n_layers > 0 ? f.n_layers : 1) : 1;
+  A(dev_alloc(c, (uint8_t **)&c->kc, c->kv_layer_stride * kv_layers * es));
+  A(dev_alloc(c, (uint8_t **)&c->vc, c->kv_layer_stride * kv_layers * es));
+  c->part_tiles_cap = ceil_div(V, 64);
+  A(dev_alloc(c, &c->part, 3 * c->part_tiles_cap * c->max_lm_rows));
+  A(dev_alloc(c, &c->logits_f32, c->max_lm_rows * (int64_t)V));
+  A(dev_alloc(c, &c->d_meta, (int64_t)f.max_batch));
+  A(dev_alloc(c, &c->d_row_slot, mr));
+  A(dev_alloc(c, &c->d_summary, (int64_t)f.max_batch));
+  A(dev_alloc(c, &c->d_status, (int64_t)1));
+  A(dev_alloc(c, &c->cs_table, (int64_t)f.max_seq * (f.head_dim / 2)));
+  if (r != L2PD_OK) return fail(r);
+  if (cudaMallocHost((void **)&c->h_meta, sizeof(SeqMeta) * f.max_batch) != cudaSuccess ||
+      cudaMallocHost((void **)&c->h_summary, sizeof(StepSummary) * f.max_batch) != cudaSuccess ||
+      cudaMallocHost((void **)&c->h_status, sizeof(int32_t)) != cudaSuccess)
+    return fail(L2PD_ERR_OOM);
+  if (cudaMemset(c->d_status, 0, 4) != cudaSuccess) return fail(L2PD_ERR_CUDA);
+  // the activation buffers back TMA boxes that reach past the live rows: start them defined
+  if (cudaMemset(c->n, 0, mr * d * es) != cudaSuccess || cudaMemset(c->att, 0, mr * hd * es) != cudaSuccess ||
+      cudaMemset(c->h, 0, mr * F * es) != cudaSuccess || cudaMemset(c->nf, 0, c->max_lm_rows * d * es) != cudaSuccess)
+    return fail(L2PD_ERR_CUDA);
+  c->st.cur_block = c->d_state_ints; c->st.l_eff = c->d_state_ints + f.max_batch;
+  c->st.done = c->d_state_ints + 2 * f.max_batch; c->st.steps = c->d_state_ints + 3 * f.max_batch;
+  c->st.eot_pos = c->d_state_ints + 4 * f.max_batch; c->st.forced = c->d_state_ints + 5 * f.max_batch;
+
+  // rotary table in double precision on the host: angle(pos, i) = pos * theta^(-2i/dh)
+  {
+    const int half = f.head_dim / 2;
+    std::vector<float2> tab((size_t)f.max_seq * half);
+    for (int pos = 0; pos < f.max_seq; ++pos)
+      for (int i = 0; i < half; ++i) {
+        const double ang = (double)pos * pow((double)f.rope_theta, -2.0 * i / f.head_dim);
+        tab[(size_t)pos * half + i] = make_float2((float)cos(ang), (float)sin(ang));
+      }
+    if (cudaMemcpy(c->cs_table, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice) != cudaSuccess)
+      return fail(L2PD_ERR_CUDA);
+  }
+  if (f.dtype == L2PD_BF16) {
+    l2pd_status s1 = make_tma_2d_bf16(&c->ta_n, c->n, mr, d, 128);
+    l2pd_status s2 = make_tma_2d_bf16(&c->ta_att, c->att, mr, hd, 128);
+    l2pd_status s3 = make_tma_2d_bf16(&c->ta_h, c->h, mr, F, 128);
+    l2pd_status s4 = make_tma_2d_bf16(&c->ta_nf, c->nf, c->max_lm_rows, d, 128);
+    if (s1 || s2 || s3 || s4) return fail(L2PD_ERR_CUDA);
+  }
+  if (cudaEventCreate(&c->ev0) != cudaSuccess || cudaEventCreate(&c->ev1) != cudaSuccess) return fail(L2PD_ERR_CUDA);
+  c->h_cur_block.assign(f.max_batch, 0); c->h_l_eff.assign(f.max_batch, 0); c->h_done.assign(f.max_batch, 1);
+  c->h_steps.assign(f.max_batch, 0); c->h_cache_block.assign(f.max_batch, -1);
+  *out = c;
+  return L2PD_OK;
+}
+
+l2pd_status l2pd_state_reset(l2pd_ctx *c, void *stream, const int32_t *d_prompts, int32_t B, int32_t P, int32_t G) {
+  if (!c || !d_prompts) return set_err(c, L2PD_ERR_ARG, "null argument");
+  const l2pd_config &f = c->cfg;
+  if (B < 1 || B > f.max_batch) return set_err(c, L2PD_ERR_SHAPE, "batch %d outside [1, %d]", B, f.max_batch);
+  if (P < 1 || G < 1 || P + G > f.max_seq) return set_err(c, L2PD_ERR_SHAPE, "P + G = %d exceeds max_seq %d (or P, G < 1)", P + G, f.max_seq);
+  if (G % f.block_len) return set_err(c, L2PD_ERR_SHAPE, "generation length %d is not a multiple of the block length %d", G, f.block_len);
+  cudaStream_t s = (cudaStream_t)stream;
+  CK(cudaSetDevice(c->device));
+  c->has_state = false;
+  int32_t *d_bad = c->d_status;   // reused as the range-check flag for this call
+  CK(cudaMemsetAsync(d_bad, 0, 4, s));
+  CKL(launch_state_reset(s, d_prompts, B, P, G, f.vocab, f.mask_id, c->d_tokens, c->d_masked, c->st, d_bad));
+  CK(cudaMemcpyAsync(c->h_status, d_bad, 4, cudaMemcpyDeviceToHost, s));
+  CK(cudaMemsetAsync(d_bad, 0, 4, s));
+  CK(cudaStreamSynchronize(s));
+  if (*c->h_status) return set_err(c, L2PD_ERR_TOKEN_RANGE, "a prompt id is outside [0, vocab) or equals mask_id");
+  c->B = B; c->P = P; c->G = G;
+  for (int i = 0; i < B; ++i) { c->h_cur_block[i] = 0; c->h_l_eff[i] = P + G; c->h_done[i] = 0; c->h_steps[i] = 0; c->h_cache_block[i] = -1; }
+  c->n_active = B;
+  c->total_steps = 0;
+  c->has_state = true;
+  return L2PD_OK;
+}
+
+l2pd_status l2pd_denoise_step(l2pd_ctx *c, void *stream, const l2pd_step_out *out) {
+  if (!c) return L2PD_ERR_ARG;
+  if (!c->has_state || c->n_active == 0) return set_err(c, L2PD_ERR_STATE, "no unfinished sequence (reset first)");
+  const l2pd_config &f = c->cfg;
+  cudaStream_t s = (cudaStream_t)stream;
+  CK(cudaSetDevice(c->device));
+  const int sb = f.block_len;
+  int n_slots = 0, T_rows = 0, max_q = 0, max_kv = 0;
+  for (int i = 0; i < c->B; ++i) {
+    if (c->h_done[i]) continue;
+    SeqMeta &m = c->h_meta[n_slots++];
+    const int b = c->h_cur_block[i], S_b = c->P + b * sb, L = c->h_l_eff[i];
+    const bool cached = f.kv_cache_mode == 1 && c->h_cache_block[i] == b;
+    m.seq = i; m.row0 = T_rows; m.pos0 = cached ? S_b : 0; m.n_rows = L - m.pos0; m.kv_len = L;
+    m.blk_start = S_b; m.n_blk_rows = (L - S_b < sb) ? (L - S_b) : sb; m.block = b;
+    if (f.kv_cache_mode == 1) c->h_cache_block[i] = b;
+    T_rows += m.n_rows;
+    if (m.n_rows > max_q) max_q = m.n_rows;
+    if (L > max_kv) max_kv = L;
+  }
+  c->last_rows = T_rows;
+  CK(cudaEventRecord(c->ev0, s));
+  CK(cudaMemcpyAsync(c->d_meta, c->h_meta, sizeof(SeqMeta) * n_slots, cudaMemcpyHostToDevice, s));
+  l2pd_status r = (f.dtype == L2PD_BF16) ? forward_and_decide<bf16>(c, s, n_slots, T_rows, max_q, max_kv, out)
+                                         : forward_and_decide<float>(c, s, n_slots, T_rows, max_q, max_kv, out);
+  if (r != L2PD_OK) return r;
+  CK(cudaMemcpyAsync(c->h_summary, c->d_summary, sizeof(StepSummary) * c->B, cudaMemcpyDeviceToHost, s));
+  CK(cudaMemcpyAsync(c->h_status, c->d_status, 4, cudaMemcpyDeviceToHost, s));
+  CK(cudaEventRecord(c->ev1, s));
+  CK(cudaStreamSynchronize(s));
+  CK(cudaEventElapsedTime(&c->last_ms, c->ev0, c->ev1));
+  if (*c->h_status != DEV_OK) {
+    const int code = *c->h_status;
+    cudaMemsetAsync(c->d_status, 0, 4, s);
+    return set_err(c, L2PD_ERR_TIMEOUT, "a bounded device wait ran out (role %d)", code);
+  }
+  c->total_steps++;
+  for (int k = 0; k < n_slots; ++k) {
+    const int i = c->h_meta[k].seq;
+    const StepSummary &sm = c->h_summary[i];
+    c->h_cur_block[i] = sm.cur_block; c->h_l_eff[i] = sm.l_eff; c->h_done[i] = sm.done; c->h_steps[i]++;
+    if (sm.done) c->n_active--;
+    if (out) {
+      if (out->h_block) out->h_block[i] = sm.block;
+      if (out->h_masks_left) out->h_masks_left[i] = sm.masks_left;
+      if (out->h_l_eff) out->h_l_eff[i] = sm.l_eff;
+      if (out->h_done) out->h_done[i] = sm.done;
+      if (out->h_forced) out->h_forced[i] = sm.forced;
+    }
+  }
+  return L2PD_OK;
+}
+
+l2pd_status l2pd_decode(l2pd_ctx *c, void *stream, const int32_t *d_prompts, int32_t B, int32_t P, int32_t G,
+                        int32_t *d_out_tokens, int32_t *h_out_len, int32_t *h_steps, int32_t *h_total_steps) {
+  if (!c || !d_out_tokens) return set_err(c, L2PD_ERR_ARG, "null argument");
+  l2pd_status r = l2pd_state_reset(c, stream, d_prompts, B, P, G);
+  if (r != L2PD_OK) return r;
+  const int64_t cap = (int64_t)B * G + 1;   // the progress fallback bounds a sequence by G steps
+  int64_t it = 0;
+  while (c->n_active > 0) {
+    if (++it > cap) return set_err(c, L2PD_ERR_STATE, "decode did not finish within B*G steps");
+    r = l2pd_denoise_step(c, stream, nullptr);
+    if (r != L2PD_OK) return r;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  CKL(launch_gather_response(s, c->d_tokens, B, P, G, d_out_tokens));
+  CK(cudaStreamSynchronize(s));
+  for (int i = 0; i < B; ++i) {
+    if (h_out_len) h_out_len[i] = c->h_l_eff[i] - P;
+    if (h_steps) h_steps[i] = c->h_steps[i];
+  }
+  if (h_total_steps) *h_total_steps = c->total_steps;
+  return L2PD_OK;
+}
+
+int32_t l2pd_num_active(const l2pd_ctx *c) { return c ? c->n_active : 0; }
+const int32_t *l2pd_state_tokens(const l2pd_ctx *c) { return c ? c->d_tokens : nullptr; }
+const uint8_t *l2pd_state_masked(const l2pd_ctx *c) { return c ? c->d_masked : nullptr; }
+
+l2pd_status l2pd_set_capture(l2pd_ctx *c, float *d_resid, int64_t slot_stride_elems) {
+  if (!c) return L2PD_ERR_ARG;
+  if (d_resid && slot_stride_elems < (int64_t)c->cfg.d_model) return set_err(c, L2PD_ERR_SHAPE, "capture slot stride too small");
+  c->cap = d_resid;
+  c->cap_stride = slot_stride_elems;
+  return L2PD_OK;
+}
+int32_t l2pd_last_step_rows(const l2pd_ctx *c) { return c ? c->last_rows : 0; }
+int64_t l2pd_launch_count(const l2pd_ctx *c) { return c ? c->launches : 0; }
+float l2pd_last_step_ms(const l2pd_ctx *c) { return c ? c->last_ms : -1.f; }
+const char *l2pd_last_error(const l2pd_ctx *c) { return c ? c->err.c_str() : "null context"; }
+
+void l2pd_destroy(l2pd_ctx *c) {
+  if (!c) return;
+  cudaSetDevice(c->device);
+  cudaDeviceSynchronize();
+  free_all(c);
+  delete c;
+}
+
+// ---- stand-alone kernels --------------------------------------------------------------------------------
+
+static int32_t *standalone_status() {
+  static int32_t *p[64] = {};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!p[dev]) {
+    if (cudaMalloc((void **)&p[dev], 4) != cudaSuccess) return nullptr;
+    cudaMemset(p[dev], 0, 4);
+  }
+  return p[dev];
+}
+
+static int device_sms() {
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  return sms;
+}
+
+static l2pd_status finish_standalone(cudaStream_t s, int32_t *status, int check) {
+  if (!check) return L2PD_OK;
+  int32_t h = 0;
+  if (cudaMemcpyAsync(&h, status, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2PD_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return L2PD_ERR_CUDA;
+  if (h != DEV_OK) { cudaMemsetAsync(status, 0, 4, s); return L2PD_ERR_TIMEOUT; }
+  return L2PD_OK;
+}
+
+static l2pd_status gemm_common(void *stream, int epi, const void *A, const void *W, const void *W2, void *out,
+                               int M, int N, int K, int tile_n, int check) {
+  if (!A || !W || !out || (epi == EPI_SWIGLU && !W2)) return L2PD_ERR_ARG;
+  if (M < 1 || N < 8 || K < 8 || (N % 8) || (K % 8)) return L2PD_ERR_SHAPE;
+  const int sms = device_sms();
+  const int unit = epi == EPI_SWIGLU ? 2 : 1;
+  if (tile_n == 0) tile_n = unit * pick_tile_n(M, N, sms, 16, 256 / unit);
+  if (tile_n < 32 || tile_n > 256 || (tile_n % (16 * unit))) return L2PD_ERR_SHAPE;
+  int32_t *status = standalone_status();
+  if (!status) return L2PD_ERR_CUDA;
+  TmaDesc ta, tb, tb2;
+  l2pd_status r = make_tma_2d_bf16(&ta, A, M, K, 128);
+  if (r) return r;
+  r = make_tma_2d_bf16(&tb, W, N, K, tile_n / unit);
+  if (r) return r;
+  if (epi == EPI_SWIGLU) { r = make_tma_2d_bf16(&tb2, W2, N, K, tile_n / unit); if (r) return r; }
+  GemmArgs g{};
+  g.epi = epi; g.a = &ta; g.b = &tb; g.b2 = epi == EPI_SWIGLU ? &tb2 : nullptr;
+  g.M = M; g.N = N; g.K = K; g.tile_n = tile_n; g.out = out; g.status = status;
+  if (launch_gemm_tcgen05((cudaStream_t)stream, g, sms) != cudaSuccess) return L2PD_ERR_CUDA;
+  return finish_standalone((cudaStream_t)stream, status, check);
+}
+
+l2pd_status l2pd_gemm_bf16(void *stream, const void *A, const void *W, void *C, int32_t M, int32_t N, int32_t K,
+                           int32_t tile_n, int32_t check) {
+  return gemm_common(stream, EPI_STORE, A, W, nullptr, C, M, N, K, tile_n, check);
+}
+l2pd_status l2pd_gemm_bf16_residual(void *stream, const void *A, const void *W, float *X, int32_t M, int32_t N,
+                                    int32_t K, int32_t tile_n, int32_t check) {
+  return gemm_common(stream, EPI_RESIDUAL, A, W, nullptr, X, M, N, K, tile_n, check);
+}
+l2pd_status l2pd_gemm_bf16_swiglu(void *stream, const void *A, const void *Wg, const void *Wu, void *H, int32_t M,
+                                  int32_t F, int32_t K, int32_t tile_n, int32_t check) {
+  return gemm_common(stream, EPI_SWIGLU, A, Wg, Wu, H, M, F, K, tile_n, check);
+}
+
+int64_t l2pd_lm_head_scratch_elems(int32_t R, int32_t V) {
+  if (R < 1 || V < 1) return 0;
+  return 3 * (int64_t)ceil_div(V, 64) * round_up(R, 128);
+}
+
+l2pd_status l2pd_lm_head_bf16(void *stream, const void *A, const void *W, const float *bias, int32_t R, int32_t V,
+                              int32_t K, float *d_scratch, int32_t *d_pred, float *d_conf, float *d_logits,
+                              int32_t check) {
+  if (!A || !W || !d_scratch || !d_pred || !d_conf) return L2PD_ERR_ARG;
+  if (R < 1 || V < 2 || K < 8 || (K % 8)) return L2PD_ERR_SHAPE;
+  const int sms = device_sms();
+  const int tile_n = pick_tile_n(R, V, sms, 16, 256);
+  int32_t *status = standalone_status();
+  if (!status) return L2PD_ERR_CUDA;
+  TmaDesc ta, tb;
+  l2pd_status r = make_tma_2d_bf16(&ta, A, R, K, 128);
+  if (r) return r;
+  r = make_tma_2d_bf16(&tb, W, V, K, tile_n);
+  if (r) return r;
+  const int rows_padded = (int)round_up(R, 128);
+  const int n_tiles = ceil_div(V, tile_n);
+  GemmArgs g{};
+  g.epi = EPI_LMHEAD; g.a = &ta; g.b = &tb; g.M = R; g.N = V; g.K = K; g.tile_n = tile_n;
+  g.bias = bias; g.part_m = d_scratch; g.part_s = d_scratch + (int64_t)n_tiles * rows_padded;
+  g.part_i = (int32_t *)(g.part_s + (int64_t)n_tiles * rows_padded); g.rows_padded = rows_padded;
+  g.logits = d_logits; g.status = status;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (launch_gemm_tcgen05(s, g, sms) != cudaSuccess) return L2PD_ERR_CUDA;
+  if (launch_merge_partials(s, g.part_m, g.part_s, g.part_i, n_tiles, rows_padded, R, d_pred, d_conf) != cudaSuccess)
+    return L2PD_ERR_CUDA;
+  return finish_standalone(s, status, check);
+}
+
+l2pd_status l2pd_attention_bf16(void *stream, const void *q, const void *k, const void *v, void *out, int32_t Tq,
+                                int32_t Tk, int32_t H, int32_t dh, int64_t q_stride, int64_t kv_stride,
+                                int64_t out_stride) {
+  if (!q || !k || !v || !out) return L2PD_ERR_ARG;
+  if (Tq < 1 || Tk < 1 || H < 1 || (dh != 64 && dh != 128) || (q_stride % 8) || (kv_stride % 8) || (out_stride % 2))
+    return L2PD_ERR_SHAPE;
+  cudaError_t e = launch_attention_bf16((cudaStream_t)stream, (const bf16 *)q, (const bf16 *)k, (const bf16 *)v,
+                                        nullptr, (bf16 *)out, q_stride, kv_stride, 0, out_stride, Tk, Tq, H, dh);
+  return e == cudaSuccess ? L2PD_OK : L2PD_ERR_CUDA;
+}
+
+}  // extern "C"

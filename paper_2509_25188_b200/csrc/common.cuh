@@ -1,0 +1,129 @@
+// Shared declarations of the l2pd CUDA library (internal).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/l2pd.h"
+
+namespace l2pd {
+
+typedef __nv_bfloat16 bf16;
+
+// One entry per sequence that takes part in the current step (device + pinned host copy).
+struct SeqMeta {
+  int32_t seq;         // index of the sequence in the batch
+  int32_t row0;        // first packed activation row of this sequence
+  int32_t n_rows;      // rows computed this step
+  int32_t pos0;        // position of row0 (0, or the block start on a cached step)
+  int32_t kv_len;      // keys visible to every query of the sequence = L_eff
+  int32_t blk_start;   // S_b = P + b*s
+  int32_t n_blk_rows;  // min(s, L_eff - S_b): block rows inside L_eff
+  int32_t block;       // b
+};
+
+// Per-sequence decode state (device arrays of length max_batch).
+struct SeqState {
+  int32_t *cur_block, *l_eff, *done, *steps, *eot_pos, *forced;
+};
+
+// Record the decision kernel writes for the host after each step.
+struct StepSummary {
+  int32_t block, masks_left, l_eff, done, forced, cur_block;
+};
+
+// Device status codes written by kernels whose bounded waits run out.
+enum { DEV_OK = 0, DEV_TIMEOUT_PRODUCER = 1, DEV_TIMEOUT_MMA = 2, DEV_TIMEOUT_EPILOGUE = 3 };
+
+inline __host__ __device__ int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline __host__ __device__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// ---- conversions -----------------------------------------------------------------------------
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(bf16 v) { return __bfloat162float(v); }
+template <typename T> __device__ __forceinline__ T from_f32(float v);
+template <> __device__ __forceinline__ float from_f32<float>(float v) { return v; }
+template <> __device__ __forceinline__ bf16 from_f32<bf16>(float v) { return __float2bfloat16_rn(v); }
+
+// ---- launchers implemented in the .cu files -------------------------------------------------------
+
+// elementwise.cu
+template <typename T>
+cudaError_t launch_embed_rmsnorm(cudaStream_t st, const int32_t *tokens, int64_t tok_stride,
+                                 const SeqMeta *meta, const int32_t *row_slot, const T *emb,
+                                 const float *gain, float eps, float *x, T *n, int rows, int d);
+template <typename T>
+cudaError_t launch_rmsnorm(cudaStream_t st, const float *x, const float *gain, float eps, T *n,
+                           int rows, int d);
+template <typename T>
+cudaError_t launch_rope_scatter(cudaStream_t st, const T *qkv, const SeqMeta *meta,
+                                const int32_t *row_slot, const float2 *cs_table, T *q, T *kc, T *vc,
+                                int64_t kv_seq_stride, int rows, int H, int dh);
+template <typename T>
+cudaError_t launch_final_norm_gather(cudaStream_t st, const float *x, const SeqMeta *meta,
+                                     const float *gain, float eps, T *nf, int n_slots, int s,
+                                     int rows_padded, int d);
+cudaError_t launch_build_row_map(cudaStream_t st, const SeqMeta *meta, int n_slots, int32_t *row_slot);
+cudaError_t launch_state_reset(cudaStream_t st, const int32_t *prompts, int B, int P, int G, int vocab,
+                               int mask_id, int32_t *tokens, uint8_t *masked, SeqState s, int32_t *bad);
+cudaError_t launch_gather_response(cudaStream_t st, const int32_t *tokens, int B, int P, int G,
+                                   int32_t *out);
+
+// simt.cu : CUDA-core GEMM and attention (fp32 configurations; also a bf16 cross-check path)
+enum { EPI_STORE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_STORE_F32 = 3 };
+template <typename T>
+cudaError_t launch_simt_gemm(cudaStream_t st, int epi, const T *A, const T *W, const T *W2, void *C,
+                             const float *bias, int M, int N, int K);
+template <typename T>
+cudaError_t launch_simt_attention(cudaStream_t st, const T *q, const T *kc, const T *vc,
+                                  const SeqMeta *meta, const int32_t *row_slot, T *out,
+                                  int64_t kv_seq_stride, int rows, int H, int dh, int max_kv);
+cudaError_t launch_row_softmax_partials(cudaStream_t st, const float *logits, int R, int V,
+                                        float *part_m, float *part_s, int32_t *part_i);
+
+// decide.cu
+struct DecideArgs {
+  const float *part_m, *part_s;   // [n_tiles, rows_padded]
+  const int32_t *part_i;
+  int n_tiles, rows_padded;
+  const SeqMeta *meta;
+  int s, P, G, n_blocks;
+  int32_t *tokens; int64_t tok_stride;
+  uint8_t *masked;                // [B, G]
+  SeqState st;
+  const float *w1, *b1, *w2, *b2;
+  float tau;
+  int use_filter, use_eotp, committed_conf_mode, eot_id;
+  StepSummary *summary;           // [max_batch], indexed by sequence
+  float *o_conf; int32_t *o_pred; float *o_p; uint8_t *o_unmask;   // optional [B, s]
+};
+cudaError_t launch_decide(cudaStream_t st, const DecideArgs &a, int n_slots);
+
+// gemm_tcgen05.cu
+struct TmaDesc { CUtensorMap map; };
+// Encodes a 2-D bf16 row-major tensor [rows, cols] with a box of [box_rows, 64] and 128-byte swizzle.
+l2pd_status make_tma_2d_bf16(TmaDesc *out, const void *ptr, int64_t rows, int64_t cols, int box_rows);
+int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile);
+struct GemmArgs {
+  int epi;                 // EPI_STORE, EPI_RESIDUAL, EPI_SWIGLU, or EPI_LMHEAD
+  const TmaDesc *a, *b, *b2;
+  int M, N, K, tile_n;
+  void *out;               // bf16 C, fp32 X, or bf16 H
+  // LM head
+  const float *bias; float *part_m, *part_s; int32_t *part_i; int rows_padded; float *logits;
+  int32_t *status;         // device status word
+};
+enum { EPI_LMHEAD = 4 };
+cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms);
+cudaError_t launch_merge_partials(cudaStream_t st, const float *part_m, const float *part_s,
+                                  const int32_t *part_i, int n_tiles, int rows_padded, int R,
+                                  int32_t *pred, float *conf);
+
+// attention.cu
+cudaError_t launch_attention_bf16(cudaStream_t st, const bf16 *q, const bf16 *kc, const bf16 *vc,
+                                  const SeqMeta *meta, bf16 *out, int64_t q_stride, int64_t kv_row_stride,
+                                  int64_t kv_seq_stride, int64_t out_stride, int n_slots, int max_q_rows,
+                                  int H, int dh);
+
+}  // namespace l2pd

@@ -1,0 +1,429 @@
+// bf16 GEMM on the 5th-generation tensor cores:  acc[M,N] = A[M,K] * W[N,K]^T, fp32 accumulation
+// in tensor memory, operands brought to shared memory by TMA (128-byte swizzle), one thread
+// issuing tcgen05.mma, four warps draining the accumulator.  Persistent CTAs (one per SM) walk
+// the output tiles; the accumulator is double-buffered in TMEM so a tile's epilogue overlaps the
+// next tile's main loop.
+//
+// Epilogues
+//   EPI_STORE     C (bf16)  = acc                                   QKV projection
+//   EPI_RESIDUAL  X (fp32) += acc                                   output / down projection
+//   EPI_SWIGLU    H (bf16)  = silu(acc_gate) * acc_up               gate/up projection; the B tile
+//                 holds tile_n/2 rows of W_gate followed by tile_n/2 rows of W_up
+//   EPI_LMHEAD    per-row running (max, sum exp, argmax) over the vocabulary tile, written as one
+//                 record per (tile, row): the logits are never stored (Eq. 3-4 need only these).
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner and MMA issuer,
+// warps 2-5 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31).
+#include <math.h>
+#include <stdio.h>
+
+#include "common.cuh"
+#include "ptx.cuh"
+
+namespace l2pd {
+
+namespace {
+
+constexpr int TILE_M = 128;
+constexpr int TILE_K = 64;                       // 64 bf16 = 128 bytes = one swizzle row
+constexpr int A_STAGE_BYTES = TILE_M * TILE_K * 2;
+constexpr int MAX_STAGES = 8;
+constexpr int TMEM_COLS = 512;
+constexpr int ACC_COLS = 256;                    // columns per accumulator buffer
+constexpr int SMEM_BUDGET = 227 * 1024;
+
+struct KParams {
+  int M, N, K, tile_n, n_stages, b_stage_bytes;
+  int m_tiles, n_tiles;
+  void *out;
+  const float *bias;
+  float *part_m, *part_s;
+  int32_t *part_i;
+  int rows_padded;
+  float *logits;
+  int32_t *status;
+};
+
+__device__ __forceinline__ void fail(int32_t *status, int code) {
+  if (status) atomicCAS(status, 0, code);
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(192, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const __grid_constant__ CUtensorMap tmB2, const KParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t sA = base;
+  const uint32_t sB = base + p.n_stages * A_STAGE_BYTES;
+  const uint32_t bar0 = ptx::smem_u32(bars);
+  auto full_bar = [&](int s) { return bar0 + 8u * s; };
+  auto empty_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };
+  auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * MAX_STAGES + b); };
+  auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * MAX_STAGES + 2 + b); };
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.n_stages; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(tfull_bar(b), 1); ptx::mbar_init(tempty_bar(b), 4); }
+    abort_flag = 0;
+    ptx::fence_barrier_init();
+    ptx::fence_proxy_async();
+  }
+  if (warp == 0 && lane == 0) {
+    ptx::prefetch_tensormap(&tmA);
+    ptx::prefetch_tensormap(&tmB);
+    if (EPI == EPI_SWIGLU) ptx::prefetch_tensormap(&tmB2);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(ptx::smem_u32(&tmem_slot), TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  ptx::tc_fence_after_sync();
+  const uint32_t tmem_base = tmem_slot;
+
+  const int num_tiles = p.m_tiles * p.n_tiles;
+  const int num_kb = (p.K + TILE_K - 1) / TILE_K;
+  const int half_n = p.tile_n >> 1;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      const uint64_t pol_w = ptx::policy_evict_first();   // weights are read once per step
+      const uint64_t pol_a = ptx::policy_evict_last();    // activations are re-read by every N tile
+      const uint32_t tx = A_STAGE_BYTES + (uint32_t)p.tile_n * 128u;
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+        const int m0 = mt * TILE_M;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
+          ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
+          ptx::tma_load_2d_hint(sA + stage * A_STAGE_BYTES, &tmA, full_bar(stage), kb * TILE_K, m0, pol_a);
+          const uint32_t dstB = sB + stage * p.b_stage_bytes;
+          if (EPI == EPI_SWIGLU) {
+            ptx::tma_load_2d_hint(dstB, &tmB, full_bar(stage), kb * TILE_K, nt * half_n, pol_w);
+            ptx::tma_load_2d_hint(dstB + half_n * 128, &tmB2, full_bar(stage), kb * TILE_K, nt * half_n, pol_w);
+          } else {
+            ptx::tma_load_2d_hint(dstB, &tmB, full_bar(stage), kb * TILE_K, nt * p.tile_n, pol_w);
+          }
+          if (++stage == p.n_stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) abort_flag = 1;
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      const uint32_t idesc = ptx::idesc_bf16_m128((uint32_t)p.tile_n);
+      int stage = 0;
+      uint32_t phase = 0;
+      int lt = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+        const int ab = lt & 1;
+        const uint32_t aphase = (lt >> 1) & 1;
+        if (!ptx::mbar_wait(tempty_bar(ab), aphase ^ 1u)) { fail(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
+        ptx::tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + ab * ACC_COLS;
+        for (int kb = 0; kb < num_kb; ++kb) {
+          if (!ptx::mbar_wait(full_bar(stage), phase)) { fail(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
+          ptx::tc_fence_after_sync();
+          const uint64_t a_desc = ptx::smem_desc_sw128(sA + stage * A_STAGE_BYTES);
+          const uint64_t b_desc = ptx::smem_desc_sw128(sB + stage * p.b_stage_bytes);
+#pragma unroll
+          for (int k = 0; k < TILE_K / 16; ++k)   // 16 bf16 = 32 bytes per MMA: descriptor address += 2
+            ptx::mma_bf16_ss(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          ptx::mma_commit(empty_bar(stage));
+          if (++stage == p.n_stages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) ptx::mma_commit(tfull_bar(ab));
+      }
+      if (!ok) abort_flag = 1;
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue
+    const int q = warp & 3;
+    int lt = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+      const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+      const int ab = lt & 1;
+      const uint32_t aphase = (lt >> 1) & 1;
+      if (!ptx::mbar_wait(tfull_bar(ab), aphase)) { fail(p.status, DEV_TIMEOUT_EPILOGUE); ok = false; break; }
+      ptx::tc_fence_after_sync();
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ab * ACC_COLS;
+      const int row = mt * TILE_M + q * 32 + lane;
+      const bool row_ok = row < p.M;
+      uint32_t v[16];
+
+      if (EPI == EPI_STORE) {
+        bf16 *C = reinterpret_cast<bf16 *>(p.out);
+        const int n0 = nt * p.tile_n;
+        for (int c = 0; c < p.tile_n; c += 16) {
+          ptx::tmem_ld_x16(taddr + c, v);
+          ptx::tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int hseg = 0; hseg < 2; ++hseg) {
+              const int col = n0 + c + hseg * 8;
+              if (col < p.N) {
+                uint4 pk;
+                uint32_t *pw = reinterpret_cast<uint32_t *>(&pk);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(v[hseg * 8 + 2 * i]),
+                                                           __uint_as_float(v[hseg * 8 + 2 * i + 1]));
+                  pw[i] = *reinterpret_cast<uint32_t *>(&t);
+                }
+                *reinterpret_cast<uint4 *>(C + (int64_t)row * p.N + col) = pk;
+              }
+            }
+          }
+        }
+      } else if (EPI == EPI_RESIDUAL) {
+        float *X = reinterpret_cast<float *>(p.out);
+        const int n0 = nt * p.tile_n;
+        for (int c = 0; c < p.tile_n; c += 16) {
+          ptx::tmem_ld_x16(taddr + c, v);
+          ptx::tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int g = 0; g < 4; ++g) {
+              const int col = n0 + c + g * 4;
+              if (col < p.N) {
+                float4 *px = reinterpret_cast<float4 *>(X + (int64_t)row * p.N + col);
+                float4 x = *px;
+                x.x += __uint_as_float(v[4 * g + 0]);
+                x.y += __uint_as_float(v[4 * g + 1]);
+                x.z += __uint_as_float(v[4 * g + 2]);
+                x.w += __uint_as_float(v[4 * g + 3]);
+                *px = x;
+              }
+            }
+          }
+        }
+      } else if (EPI == EPI_SWIGLU) {
+        bf16 *H = reinterpret_cast<bf16 *>(p.out);
+        const int n0 = nt * half_n;
+        uint32_t u[16];
+        for (int c = 0; c < half_n; c += 16) {
+          ptx::tmem_ld_x16(taddr + c, v);
+          ptx::tmem_ld_x16(taddr + half_n + c, u);
+          ptx::tmem_ld_wait();
+          if (row_ok) {
+#pragma unroll
+            for (int hseg = 0; hseg < 2; ++hseg) {
+              const int col = n0 + c + hseg * 8;
+              if (col < p.N) {
+                uint4 pk;
+                uint32_t *pw = reinterpret_cast<uint32_t *>(&pk);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  float g0 = __uint_as_float(v[hseg * 8 + 2 * i]), g1 = __uint_as_float(v[hseg * 8 + 2 * i + 1]);
+                  float u0 = __uint_as_float(u[hseg * 8 + 2 * i]), u1 = __uint_as_float(u[hseg * 8 + 2 * i + 1]);
+                  float h0 = g0 / (1.0f + __expf(-g0)) * u0;
+                  float h1 = g1 / (1.0f + __expf(-g1)) * u1;
+                  __nv_bfloat162 t = __floats2bfloat162_rn(h0, h1);
+                  pw[i] = *reinterpret_cast<uint32_t *>(&t);
+                }
+                *reinterpret_cast<uint4 *>(H + (int64_t)row * p.N + col) = pk;
+              }
+            }
+          }
+        }
+      } else {  // EPI_LMHEAD
+        const float L2E = 1.4426950408889634f;
+        const int n0 = nt * p.tile_n;
+        float m_run = -INFINITY, s_run = 0.f;
+        int i_run = 0x7fffffff;
+        for (int c = 0; c < p.tile_n; c += 16) {
+          ptx::tmem_ld_x16(taddr + c, v);
+          ptx::tmem_ld_wait();
+          if (row_ok && n0 + c < p.N) {
+            float f[16];
+            float cm = -INFINITY;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const int col = n0 + c + i;
+              float val = __uint_as_float(v[i]);
+              if (col < p.N) { if (p.bias) val += __ldg(p.bias + col); }
+              else val = -INFINITY;
+              f[i] = val;
+              cm = fmaxf(cm, val);
+            }
+            if (p.logits) {
+#pragma unroll
+              for (int i = 0; i < 16; ++i)
+                if (n0 + c + i < p.N) p.logits[(int64_t)row * p.N + n0 + c + i] = f[i];
+            }
+            if (cm > m_run) {
+              s_run *= exp2f((m_run - cm) * L2E);
+              m_run = cm;
+              int ci = 0;
+#pragma unroll
+              for (int i = 15; i >= 0; --i) if (f[i] == cm) ci = i;   // lowest index holding the max
+              i_run = n0 + c + ci;
+            }
+            float add = 0.f;
+#pragma unroll
+            for (int i = 0; i < 16; ++i) add += exp2f((f[i] - m_run) * L2E);
+            s_run += add;
+          }
+        }
+        if (row_ok) {
+          const int64_t o = (int64_t)nt * p.rows_padded + row;
+          p.part_m[o] = m_run;
+          p.part_s[o] = s_run;
+          p.part_i[o] = i_run;
+        }
+      }
+      ptx::tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(tempty_bar(ab));
+    }
+    if (!ok) abort_flag = 1;
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  __syncwarp();
+  ptx::tc_fence_before_sync();
+  __syncthreads();
+  if (abort_flag) {
+    // A wait ran out: give copies still in flight time to land before the CTA's shared memory goes away.
+    const uint64_t t0 = ptx::globaltimer();
+    while (ptx::globaltimer() - t0 < 200000ull) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    ptx::tc_fence_after_sync();
+    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static bool tried = false;
+  if (!tried) {
+    tried = true;
+    void *ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+__global__ void merge_partials_kernel(const float *part_m, const float *part_s, const int32_t *part_i,
+                                      int n_tiles, int rows_padded, int32_t *pred, float *conf) {
+  const int r = blockIdx.x, lane = threadIdx.x;
+  float mx = -INFINITY, sum = 0.f;
+  int ix = 0x7fffffff;
+  for (int t = lane; t < n_tiles; t += 32) {
+    float tm = part_m[(int64_t)t * rows_padded + r];
+    float ts = part_s[(int64_t)t * rows_padded + r];
+    int ti = part_i[(int64_t)t * rows_padded + r];
+    if (tm > mx) { sum = sum * expf(mx - tm) + ts; mx = tm; ix = ti; }
+    else { sum += ts * expf(tm - mx); if (tm == mx && ti < ix) ix = ti; }
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    float om = __shfl_xor_sync(0xffffffffu, mx, o);
+    float os = __shfl_xor_sync(0xffffffffu, sum, o);
+    int oi = __shfl_xor_sync(0xffffffffu, ix, o);
+    float nm = fmaxf(mx, om);
+    float ns = (mx == -INFINITY ? 0.f : sum * expf(mx - nm)) + (om == -INFINITY ? 0.f : os * expf(om - nm));
+    int ni = (om > mx || (om == mx && oi < ix)) ? oi : ix;
+    mx = nm; sum = ns; ix = ni;
+  }
+  if (lane == 0) { pred[r] = ix; conf[r] = 1.0f / sum; }
+}
+
+}  // namespace
+
+l2pd_status make_tma_2d_bf16(TmaDesc *out, const void *ptr, int64_t rows, int64_t cols, int box_rows) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return L2PD_ERR_CUDA;
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15) || (cols % 8) || box_rows < 1 || box_rows > 256) return L2PD_ERR_SHAPE;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)TILE_K, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(&out->map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box,
+                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? L2PD_OK : L2PD_ERR_CUDA;
+}
+
+// Tile width that minimises (waves x per-tile cost) for m_tiles row tiles over num_sms persistent
+// CTAs.  `unit` is the granularity of the returned width, `max_tile` its largest value.
+int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile) {
+  const int m_tiles = ceil_div(M, TILE_M);
+  int best = max_tile;
+  double best_cost = 1e30;
+  for (int tn = max_tile; tn >= 64 && tn >= multiple; tn -= multiple) {
+    const int tiles = m_tiles * ceil_div(N, tn);
+    const int waves = ceil_div(tiles, num_sms);
+    const double cost = (double)waves * (tn + 12);   // per-tile main loop ~ tn, plus a fixed part
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = tn; }
+  }
+  return best;
+}
+
+cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms) {
+  KParams p;
+  p.M = g.M; p.N = g.N; p.K = g.K; p.tile_n = g.tile_n;
+  p.b_stage_bytes = g.tile_n * 128;
+  const int stage_bytes = A_STAGE_BYTES + p.b_stage_bytes;
+  int stages = (SMEM_BUDGET - 2048) / stage_bytes;
+  if (stages > MAX_STAGES) stages = MAX_STAGES;
+  if (stages < 2) return cudaErrorInvalidValue;
+  p.n_stages = stages;
+  p.m_tiles = ceil_div(g.M, TILE_M);
+  const int n_per_tile = (g.epi == EPI_SWIGLU) ? g.tile_n / 2 : g.tile_n;
+  p.n_tiles = ceil_div(g.N, n_per_tile);
+  p.out = g.out; p.bias = g.bias; p.part_m = g.part_m; p.part_s = g.part_s; p.part_i = g.part_i;
+  p.rows_padded = g.rows_padded; p.logits = g.logits; p.status = g.status;
+  const int tiles = p.m_tiles * p.n_tiles;
+  if (tiles <= 0) return cudaSuccess;
+  const int grid = tiles < num_sms ? tiles : num_sms;
+  const size_t smem = (size_t)stages * stage_bytes + 1024;
+  const CUtensorMap &b2 = g.b2 ? g.b2->map : g.b->map;
+  cudaError_t e;
+#define L2PD_LAUNCH(EPI)                                                                              \
+  e = cudaFuncSetAttribute(gemm_tcgen05_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
+                           SMEM_BUDGET - 1024);                                                      \
+  if (e != cudaSuccess) return e;                                                                    \
+  gemm_tcgen05_kernel<EPI><<<grid, 192, smem, st>>>(g.a->map, g.b->map, b2, p);
+  switch (g.epi) {
+    case EPI_STORE: L2PD_LAUNCH(EPI_STORE) break;
+    case EPI_RESIDUAL: L2PD_LAUNCH(EPI_RESIDUAL) break;
+    case EPI_SWIGLU: L2PD_LAUNCH(EPI_SWIGLU) break;
+    case EPI_LMHEAD: L2PD_LAUNCH(EPI_LMHEAD) break;
+    default: return cudaErrorInvalidValue;
+  }
+#undef L2PD_LAUNCH
+  return cudaGetLastError();
+}
+
+cudaError_t launch_merge_partials(cudaStream_t st, const float *part_m, const float *part_s,
+                                  const int32_t *part_i, int n_tiles, int rows_padded, int R,
+                                  int32_t *pred, float *conf) {
+  merge_partials_kernel<<<R, 32, 0, st>>>(part_m, part_s, part_i, n_tiles, rows_padded, pred, conf);
+  return cudaGetLastError();
+}
+
+}  // namespace l2pd

@@ -32,3 +32,110 @@ def identity_filter(s: int, k: float, b: float):
     """z_j = k * relu(c_j) + b, so p_j = sigmoid(k c_j + b) for c_j >= 0."""
     return {"w1": np.eye(s, dtype=np.float32), "b1": np.zeros(s, np.float32),
             "w2": (k * np.eye(s)).astype(np.float32), "b2": np.full(s, b, np.float32)}
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU-vs-oracle lockstep (used by the -m gpu tests)
+
+def _sync_oracle_state(st, m, toks, msk, l_eff, done, cur_block):
+    st.tokens[:] = toks
+    st.masked[:] = msk
+    st.L_eff = int(l_eff)
+    st.done = bool(done)
+    st.cur_block = int(cur_block)
+    gen = st.tokens[st.P: st.P + st.G]
+    hits = np.where((gen == m.eot_id) & ~st.masked)[0]
+    st.eot_pos = int(hits[0]) if len(hits) and st.L_eff == st.P + int(hits[0]) + 1 else -1
+
+
+def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, check_logits=True,
+             max_steps=None, replay_margin=1e-5):
+    """Runs the CUDA decoder step by step; before every step the oracle is put in the decoder's
+    state (teacher forcing), then both take the step and are compared:
+      logits  |gpu - orc| <= logit_rtol * max|orc row|
+      conf    |gpu - orc| <= conf_atol
+      pred    equal wherever the oracle's top-2 logit gap exceeds 2 * logit_rtol * max|orc row|
+      unmask  equal to the oracle's wherever every |p - tau| of the block exceeds p_margin (and, on a
+              forced step, the two best confidences differ by more than conf_atol); and ALWAYS equal
+              to the oracle's decision logic replayed in fp64 on the decoder's own conf/pred, unless
+              a replayed |p - tau| is within replay_margin.
+    Returns counters; asserts on any violation.
+    """
+    import copy
+
+    prompts = np.asarray(prompts)
+    B, P = prompts.shape
+    s = cfg.block_len
+    dec.state_reset(prompts, G)
+    states = [orc.init_state(m, p, G) for p in prompts]
+    stat = dict(steps=0, rows=0, pred_checked=0, unmask_checked=0, replay_checked=0, forced=0,
+                max_logit_rel=0.0, max_conf_err=0.0, seq_steps=[0] * B)
+    while dec.num_active > 0:
+        if max_steps is not None and stat["steps"] >= max_steps:
+            break
+        toks, msk = dec.tokens(), dec.masked()
+        active = [i for i in range(B) if not states[i].done]
+        for i in active:
+            assert np.array_equal(states[i].tokens, toks[i]) and np.array_equal(states[i].masked, msk[i])
+        out = dec.denoise_step(want_logits=check_logits)
+        stat["steps"] += 1
+        for i in active:
+            st = states[i]
+            pre = copy.deepcopy(st)
+            rec = orc.denoise_step(m, filt, st, cfg, keep_logits=True)
+            stat["seq_steps"][i] += 1
+            n = rec.n_rows
+            stat["rows"] += n
+            assert out["block"][i] == rec.block
+            row_max = np.abs(rec.logits).max(axis=-1)
+            if check_logits:
+                err = np.abs(out["logits"][i, :n] - rec.logits).max(axis=-1) / row_max
+                stat["max_logit_rel"] = max(stat["max_logit_rel"], float(err.max()))
+                assert err.max() <= logit_rtol, "logits off by %g (rel) at step %d" % (err.max(), stat["steps"])
+            cerr = np.abs(out["conf"][i, :n] - rec.conf)
+            stat["max_conf_err"] = max(stat["max_conf_err"], float(cerr.max()))
+            assert cerr.max() <= conf_atol, "confidence off by %g at step %d" % (cerr.max(), stat["steps"])
+            assert (out["pred"][i, n:] == -1).all() and (out["conf"][i, n:] == 0).all()
+            sure = rec.gap > 2 * logit_rtol * row_max
+            stat["pred_checked"] += int(sure.sum())
+            assert np.array_equal(out["pred"][i, :n][sure], rec.pred[sure])
+
+            # decision logic replayed on the decoder's own numbers
+            rp = copy.deepcopy(pre)
+            rp.steps += 1
+            gpred = out["pred"][i, :n].astype(np.int64)
+            gconf = out["conf"][i, :n].astype(np.float64)
+            rrec = orc.decide(m, filt, rp, cfg, gpred, gconf)
+            blk_masked = pre.masked[rec.block * s: rec.block * s + s]
+            near = np.abs(rrec.p - cfg.tau)[blk_masked]
+            replay_ok = (len(near) == 0 or near.min() > replay_margin)
+            if rrec.forced:
+                cm = np.sort(gconf[blk_masked[:n]])[::-1]
+                replay_ok = replay_ok and (len(cm) < 2 or cm[0] - cm[1] > 1e-6)
+            if replay_ok:
+                stat["replay_checked"] += 1
+                assert np.array_equal(out["unmask"][i].astype(bool), rrec.unmask), "decision replay differs"
+                assert out["l_eff"][i] == rp.L_eff and bool(out["done"][i]) == rp.done
+                assert out["forced"][i] == int(rrec.forced)
+                assert out["masks_left"][i] == int(rp.masked[rec.block * s: rec.block * s + s].sum())
+                assert np.abs(out["p"][i] - rrec.p).max() < 1e-4
+
+            # the oracle's own decision, where it is clear of the margins
+            near_o = np.abs(rec.p - cfg.tau)[blk_masked]
+            clear = len(near_o) == 0 or near_o.min() > p_margin
+            if rec.forced:
+                cm = np.sort(rec.conf[blk_masked[:n]])[::-1]
+                clear = clear and (len(cm) < 2 or cm[0] - cm[1] > 2 * conf_atol)
+            committed_sure = sure[rec.unmask[:n]].all() if rec.unmask[:n].any() else True
+            if clear:
+                stat["unmask_checked"] += 1
+                assert np.array_equal(out["unmask"][i].astype(bool), rec.unmask), "unmask decision differs"
+                assert out["forced"][i] == int(rec.forced)
+                stat["forced"] += int(rec.forced)
+        toks, msk = dec.tokens(), dec.masked()
+        for i in active:
+            blk = out["block"][i]
+            nxt = blk + 1 if (out["masks_left"][i] == 0 and not out["done"][i]) else blk
+            _sync_oracle_state(states[i], m, toks[i], msk[i], out["l_eff"][i], out["done"][i], nxt)
+    stat["states"] = states
+    return stat

@@ -1,0 +1,152 @@
+"""Kernel-level parity, through the C ABI, against the oracle's functions on the same seeded inputs.
+
+Tolerances (bf16 inputs, fp32 accumulation, one rounding of the output to bf16):
+a product of K terms of magnitude ~|a||w| accumulated in fp32 is exact to ~K*2^-24 relative to
+sum|a||w|; the bf16 store adds 2^-9 relative.  The checks below use
+|gpu - oracle| <= 2^-8 * |oracle| + 2e-3 * row_scale, row_scale = rms of the oracle's row.
+"""
+from __future__ import annotations
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import l2pd_oracle as orc
+from paper_2509_25188_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _b():
+    from paper_2509_25188_b200 import binding
+    return binding
+
+
+def _bf16(seed, stream, shape, std):
+    return wl.make_activations(seed, stream, shape, std, "bf16")
+
+
+def _close_bf16(got, want, extra=0.0):
+    want = np.asarray(want, np.float64)
+    got = np.asarray(got, np.float64)
+    scale = np.sqrt((want ** 2).mean(axis=-1, keepdims=True)) + 1e-30
+    tol = 2.0 ** -8 * np.abs(want) + (2e-3 + extra) * scale
+    bad = np.abs(got - want) > tol
+    assert not bad.any(), "max err %g at %s (want %g)" % (
+        np.abs(got - want).max(), np.argwhere(bad)[0], want[tuple(np.argwhere(bad)[0])])
+
+
+GEMM_SHAPES = [
+    (128, 256, 64, 0),      # single tile, one k-block
+    (200, 320, 192, 0),     # ragged M, several tiles
+    (512, 1024, 512, 0),
+    (77, 136, 72, 64),      # ragged everything: N tail inside a tile, K tail inside a k-block
+    (300, 528, 1032, 176),  # odd tile width (multiple of 16), K tail
+    (1, 64, 64, 0),
+    (640, 2048, 256, 112),  # many tiles per CTA: accumulator double-buffering, ring wrap-around
+]
+
+
+@pytest.mark.parametrize("M,N,K,tile_n", GEMM_SHAPES)
+def test_gemm_bf16_store(M, N, K, tile_n):
+    b = _b()
+    A = _bf16(1, 0, (M, K), 1.0)
+    W = _bf16(1, 1, (N, K), 0.05)
+    got = b.gemm_bf16(b.to_device(A), b.to_device(W), tile_n).float().cpu().numpy()
+    want = orc.linear(orc.widen(A), W)
+    _close_bf16(got, want)
+
+
+@pytest.mark.parametrize("M,N,K,tile_n", GEMM_SHAPES[:5])
+def test_gemm_bf16_residual(M, N, K, tile_n):
+    b = _b()
+    A = _bf16(2, 0, (M, K), 1.0)
+    W = _bf16(2, 1, (N, K), 0.05)
+    X = wl.make_activations(2, 2, (M, N), 1.0, "fp32")
+    Xd = b.to_device(X.copy())
+    b.gemm_bf16_residual(b.to_device(A), b.to_device(W), Xd, tile_n)
+    want = X.astype(np.float64) + orc.linear(orc.widen(A), W)
+    got = Xd.cpu().numpy()
+    assert np.allclose(got, want, rtol=1e-5, atol=1e-4 * np.sqrt(K))
+
+
+@pytest.mark.parametrize("M,F,K,tile_n", [(128, 128, 64, 0), (200, 336, 192, 0), (512, 1408, 512, 224),
+                                          (77, 136, 72, 64), (640, 2048, 256, 96)])
+def test_gemm_bf16_swiglu(M, F, K, tile_n):
+    b = _b()
+    A = _bf16(3, 0, (M, K), 1.0)
+    Wg = _bf16(3, 1, (F, K), 0.08)
+    Wu = _bf16(3, 2, (F, K), 0.08)
+    got = b.gemm_bf16_swiglu(b.to_device(A), b.to_device(Wg), b.to_device(Wu), tile_n).float().cpu().numpy()
+    a = orc.widen(A)
+    want = orc.silu(orc.linear(a, Wg)) * orc.linear(a, Wu)
+    _close_bf16(got, want)
+
+
+@pytest.mark.parametrize("R,V,K,with_bias", [(32, 4096, 256, False), (16, 5000, 136, True), (200, 1000, 512, True),
+                                             (1, 70, 64, False), (32, 20000, 1024, True)])
+def test_lm_head_fused_confidence(R, V, K, with_bias):
+    """Eq. 3-4: argmax and softmax probability of the argmax, reduced without storing logits."""
+    b = _b()
+    A = _bf16(4, 0, (R, K), 1.0)
+    W = _bf16(4, 1, (V, K), 0.3)
+    bias = wl.make_activations(4, 2, (V,), 1.0, "fp32") if with_bias else None
+    pred, conf, logits = b.lm_head_bf16(b.to_device(A), b.to_device(W),
+                                        b.to_device(bias) if with_bias else None, want_logits=True)
+    ref = orc.linear(orc.widen(A), W)
+    if with_bias:
+        ref = ref + bias.astype(np.float64)[None, :]
+    rp, rc, gap = orc.confidence_head(ref)
+    got_logits = logits.cpu().numpy()
+    assert np.abs(got_logits - ref).max() <= 1e-4 * np.abs(ref).max() + 1e-5 * np.sqrt(K)
+    pred, conf = pred.cpu().numpy(), conf.cpu().numpy()
+    sure = gap > 1e-3 * np.abs(ref).max()
+    assert sure.mean() > 0.5
+    assert np.array_equal(pred[sure], rp[sure])
+    assert np.abs(conf - rc)[sure].max() < 1e-3
+    # the fused reduction must agree with the logits the same kernel wrote
+    p2, c2, _ = orc.confidence_head(got_logits.astype(np.float64))
+    assert np.array_equal(pred, p2)
+    assert np.abs(conf - c2).max() < 1e-5
+    # without the debug buffer the result is the same
+    pred3, conf3, _ = b.lm_head_bf16(b.to_device(A), b.to_device(W), b.to_device(bias) if with_bias else None)
+    assert np.array_equal(pred3.cpu().numpy(), pred) and np.array_equal(conf3.cpu().numpy(), conf)
+
+
+def test_lm_head_ties_pick_lowest_id():
+    b = _b()
+    R, V, K = 4, 600, 64
+    A = np.zeros((R, K), np.float32)
+    A[:, 0] = 1.0
+    W = np.zeros((V, K), np.float32)
+    W[[7, 300, 599], 0] = 2.0          # three equal maxima, in different vocabulary tiles
+    pred, conf, _ = b.lm_head_bf16(b.to_device(wl.f32_to_bf16_bits(A)), b.to_device(wl.f32_to_bf16_bits(W)))
+    rp, rc, _ = orc.confidence_head(orc.linear(A.astype(np.float64), W))
+    assert pred.cpu().numpy().tolist() == [7] * R == rp.tolist()
+    assert np.abs(conf.cpu().numpy() - rc).max() < 1e-6
+
+
+@pytest.mark.parametrize("Tq,Tk,H,dh", [(64, 64, 2, 128), (100, 100, 3, 128), (37, 200, 2, 64), (512, 512, 4, 128),
+                                        (5, 1, 1, 64), (130, 1030, 2, 128)])
+def test_attention_bidirectional(Tq, Tk, H, dh):
+    b = _b()
+    q = _bf16(5, 0, (Tq, H * dh), 1.0)
+    k = _bf16(5, 1, (Tk, H * dh), 1.0)
+    v = _bf16(5, 2, (Tk, H * dh), 1.0)
+    got = b.attention_bf16(b.to_device(q), b.to_device(k), b.to_device(v), H, dh).float().cpu().numpy()
+    want = orc.attention(orc.widen(q).reshape(Tq, H, dh), orc.widen(k).reshape(Tk, H, dh),
+                         orc.widen(v).reshape(Tk, H, dh)).reshape(Tq, H * dh)
+    # probabilities are rounded to bf16 before the second product: 2^-9 relative on each weight
+    assert np.abs(got - want).max() < 2e-2
+    assert np.sqrt(((got - want) ** 2).mean()) < 4e-3
+
+
+def test_shape_errors_are_reported_not_launched():
+    b = _b()
+    A = b.to_device(_bf16(6, 0, (16, 64), 1.0))
+    W = b.to_device(_bf16(6, 1, (64, 64), 1.0))
+    with pytest.raises(b.L2pdError) as e:
+        b.gemm_bf16(A, W, tile_n=40)          # not a multiple of 16
+    assert e.value.status == -2
+    with pytest.raises(b.L2pdError):
+        b.gemm_bf16(A[:, :60], W[:, :60])      # K not a multiple of 8

@@ -534,3 +534,15 @@ def test_planted_mistakes_are_caught(monkeypatch):
     p = np.array([0.5, 0.9])
     un, forced = orc.unmask_rule(p, p, np.ones(2, bool), 0.5)
     assert un.tolist() == [False, True] and not forced
+
+
+def test_linear_is_x_times_w_transposed():
+    rng = np.random.default_rng(9)
+    x = rng.normal(size=(3, 5))
+    w = rng.normal(size=(4, 5)).astype(np.float32)
+    y = orc.linear(x, w)
+    assert y.shape == (3, 4)
+    for t in range(3):
+        for o in range(4):
+            assert y[t, o] == pytest.approx(sum(x[t, i] * float(w[o, i]) for i in range(5)), abs=1e-13)
+    assert np.array_equal(orc.linear(x, np.eye(5, dtype=np.float32)), x)
