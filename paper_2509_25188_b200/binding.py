@@ -267,11 +267,11 @@ class Decoder:
 
 
 class _DeviceView:
-    """Read-only view of library-owned device memory (CUDA array interface)."""
+    """View of library-owned device memory (CUDA array interface); callers only read it."""
 
     def __init__(self, ptr: int, shape, typestr: str):
         self.__cuda_array_interface__ = {"shape": tuple(shape), "typestr": typestr,
-                                         "data": (int(ptr), True), "version": 2}
+                                         "data": (int(ptr), False), "version": 2}
 
 
 # ---- stand-alone kernels -------------------------------------------------------------------------

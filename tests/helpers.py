@@ -48,21 +48,24 @@ def _sync_oracle_state(st, m, toks, msk, l_eff, done, cur_block):
     st.eot_pos = int(hits[0]) if len(hits) and st.L_eff == st.P + int(hits[0]) + 1 else -1
 
 
-def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, check_logits=True,
-             max_steps=None, replay_margin=1e-5):
+def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, conf_margin=None,
+             check_logits=True, max_steps=None, replay_margin=1e-5):
     """Runs the CUDA decoder step by step; before every step the oracle is put in the decoder's
     state (teacher forcing), then both take the step and are compared:
       logits  |gpu - orc| <= logit_rtol * max|orc row|
       conf    |gpu - orc| <= conf_atol
       pred    equal wherever the oracle's top-2 logit gap exceeds 2 * logit_rtol * max|orc row|
       unmask  equal to the oracle's wherever every |p - tau| of the block exceeds p_margin (and, on a
-              forced step, the two best confidences differ by more than conf_atol); and ALWAYS equal
-              to the oracle's decision logic replayed in fp64 on the decoder's own conf/pred, unless
-              a replayed |p - tau| is within replay_margin.
+              forced step, the two best confidences differ by more than conf_margin, default
+              2 * conf_atol); and ALWAYS equal to the oracle's decision logic replayed in fp64 on the
+              decoder's own conf/pred, unless a replayed |p - tau| is within replay_margin (the
+              decoder evaluates the filter in fp32).
     Returns counters; asserts on any violation.
     """
     import copy
 
+    if conf_margin is None:
+        conf_margin = 2 * conf_atol
     prompts = np.asarray(prompts)
     B, P = prompts.shape
     s = cfg.block_len
@@ -109,9 +112,6 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
             blk_masked = pre.masked[rec.block * s: rec.block * s + s]
             near = np.abs(rrec.p - cfg.tau)[blk_masked]
             replay_ok = (len(near) == 0 or near.min() > replay_margin)
-            if rrec.forced:
-                cm = np.sort(gconf[blk_masked[:n]])[::-1]
-                replay_ok = replay_ok and (len(cm) < 2 or cm[0] - cm[1] > 1e-6)
             if replay_ok:
                 stat["replay_checked"] += 1
                 assert np.array_equal(out["unmask"][i].astype(bool), rrec.unmask), "decision replay differs"
@@ -125,8 +125,7 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
             clear = len(near_o) == 0 or near_o.min() > p_margin
             if rec.forced:
                 cm = np.sort(rec.conf[blk_masked[:n]])[::-1]
-                clear = clear and (len(cm) < 2 or cm[0] - cm[1] > 2 * conf_atol)
-            committed_sure = sure[rec.unmask[:n]].all() if rec.unmask[:n].any() else True
+                clear = clear and (len(cm) < 2 or cm[0] - cm[1] > conf_margin)
             if clear:
                 stat["unmask_checked"] += 1
                 assert np.array_equal(out["unmask"][i].astype(bool), rec.unmask), "unmask decision differs"
@@ -139,3 +138,17 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
             _sync_oracle_state(states[i], m, toks[i], msk[i], out["l_eff"][i], out["done"][i], nxt)
     stat["states"] = states
     return stat
+
+
+def find_eot_bias(m, shape, filt, G, cfg, prompt_len, seeds=range(3, 40), grid=None):
+    """Seeded search, on the oracle only, for (prompt seed, EoT bias) whose decode stops with
+    G/4 <= out_len <= 3G/4, so that EoTP fires in mid-sequence.  Returns (seed, bias, result)."""
+    grid = np.arange(10.0, 24.0, 0.5) if grid is None else grid
+    for seed in seeds:
+        prompt = wl.make_prompts(1, prompt_len, shape, seed=seed)[0]
+        for v in grid:
+            m.lm_head_bias = wl.make_eot_bias(shape, float(v))
+            r = orc.decode(m, filt, prompt, G, cfg, keep_trace=False)
+            if G // 4 <= r.out_len <= 3 * G // 4:
+                return seed, float(v), r
+    raise AssertionError("no (seed, bias) on the grid stops mid-sequence")
