@@ -1,0 +1,365 @@
+#!/usr/bin/env python
+"""Benchmark of the Learn2PD denoising step on B200.
+
+  python bench.py --gpus N --steps K --warmup W            (this implementation)
+  python bench.py --impl reference --steps K --warmup W    (the CPU oracle, timed as it stands)
+
+Workload (N = 1 and every replica at N > 1): one denoising step of the LLaDA-8B-shaped
+model — batch 1, 256 prompt tokens + 256 masked positions, block 32 — i.e. the state set-up of
+Algorithm 2 followed by M(X), the confidence head, the filter, the threshold and EoTP.
+A "step" of the timed loop is exactly that, repeated K times on the same seeded prompt.
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2509_25188_b200 import workloads as wl  # noqa: E402
+
+WORKLOAD = "C1"
+SHAPE = wl.LLADA_8B
+DEC = wl.DECODES[WORKLOAD]
+METRIC, UNIT = "generated_tokens_per_s", "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def step_work(shape, T, Lk, R):
+    """Algorithmic FLOPs and bytes of one denoising step over T rows, keys Lk per query, R LM-head rows."""
+    d, F, V, NL = shape.d_model, shape.d_ff, shape.vocab, shape.n_layers
+    hd = shape.n_heads * shape.head_dim
+    gemm = 2.0 * T * NL * (d * 3 * hd + hd * d + 3 * d * F)
+    attn = 4.0 * NL * hd * T * Lk
+    head = 2.0 * R * d * V
+    w_bytes = 2.0 * (NL * (d * 3 * hd + hd * d + 3 * d * F) + V * d)
+    act_bytes = 44.0 * T * d * NL
+    return {"flops": gemm + attn + head, "gemm_flops": gemm, "attn_flops": attn, "head_flops": head,
+            "weight_bytes": w_bytes, "act_bytes": act_bytes}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle leg (shared by cpu_baseline and --impl reference)
+
+class OracleSample:
+    """Times the oracle on a bounded sample of the step: the embedding, `n_sample` of the model's
+    layers and the LM head + decision on the block's rows; the layer time is scaled to full depth."""
+
+    def __init__(self, n_sample=4, budget_s=None, calls=1):
+        if budget_s is not None:   # about 2 s per layer and 1 s for the head on 8 cores
+            n_sample = int(min(4, max(1, (budget_s / max(calls, 1) - 1.0) // 2)))
+        from oracle import l2pd_oracle as orc
+        self.orc = orc
+        self.n_sample = n_sample
+        shape = wl.thin(SHAPE, n_sample)
+        w = wl.make_weights(shape, seed=0, final_norm_gain=wl.spread_gain(SHAPE), threads=os.cpu_count() or 8)
+        self.model = orc.Model(n_layers=n_sample, d_model=shape.d_model, n_heads=shape.n_heads, head_dim=shape.head_dim,
+                               d_ff=shape.d_ff, vocab=shape.vocab, rms_eps=shape.rms_eps, rope_theta=shape.rope_theta,
+                               mask_id=shape.mask_id, eot_id=shape.eot_id, weights=w)
+        self.filt = wl.make_filter(DEC.block_len, DEC.tau, seed=0)
+        self.prompt = wl.make_prompts(1, DEC.prompt_len, SHAPE, seed=1)[0]
+        self.cfg = orc.DecodeConfig(block_len=DEC.block_len, tau=DEC.tau)
+
+    def one(self):
+        """Returns (extrapolated seconds for a full-depth step, tokens the sample's step committed)."""
+        orc = self.orc
+        st = orc.init_state(self.model, self.prompt, DEC.gen_len)
+        t0 = time.perf_counter()
+        w = self.model.weights
+        x = orc.widen(w["tok_emb"][st.tokens[: st.L_eff]])
+        pos = np.arange(st.L_eff)
+        t1 = time.perf_counter()
+        for layer in w["layers"]:
+            x = orc.layer_forward(self.model, layer, x, pos)
+        t2 = time.perf_counter()
+        S_b = st.P
+        logits = orc.lm_head_logits(self.model, x[S_b: S_b + DEC.block_len])
+        pred, conf, gap = orc.confidence_head(logits)
+        rec = orc.decide(self.model, self.filt, st, self.cfg, pred, conf)
+        t3 = time.perf_counter()
+        full = (t1 - t0) + (t2 - t1) * SHAPE.n_layers / self.n_sample + (t3 - t2)
+        return full, int(rec.unmask.sum()), (t3 - t0)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import threadpoolctl
+    cores = max(i["num_threads"] for i in threadpoolctl.threadpool_info() or [{"num_threads": os.cpu_count()}])
+    smp = OracleSample(budget_s=150.0, calls=args.steps + args.warmup)
+    for _ in range(args.warmup):
+        smp.one()
+    times, toks, raw = [], 0, 0.0
+    for _ in range(args.steps):
+        t, n, r = smp.one()
+        times.append(t)
+        toks += n
+        raw += r
+    total = sum(times)
+    value = toks / total
+    sample = ("embedding + %d of %d layers + LM head/decision on %d rows at T=%d, layer time scaled x%d; "
+              "tokens = commits of the sample's own step" % (smp.n_sample, SHAPE.n_layers, DEC.block_len,
+                                                            DEC.prompt_len + DEC.gen_len, SHAPE.n_layers // smp.n_sample))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict(), "gpu_launches": 0,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                             "measured_s_per_sample": raw / args.steps},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def config_dict():
+    return {"workload": "%s: one denoising step, LLaDA-8B-shaped model (32 layers, d 4096, 32 heads x 128, "
+                        "SwiGLU 12288, vocab 126464), batch 1, prompt %d + %d masked, block %d, filter + EoTP"
+                        % (WORKLOAD, DEC.prompt_len, DEC.gen_len, DEC.block_len),
+            "tokens_per_step_rows": DEC.prompt_len + DEC.gen_len, "block_len": DEC.block_len, "tau": DEC.tau,
+            "l2": "inputs larger than L2: every step streams 15 GB of weights",
+            "weights": "N(0, 0.02^2) bf16, drawn on the device with torch's generator, seed 0",
+            "parallelism": "replicas"}
+
+
+# ------------------------------------------------------------------------------------------------
+# GPU leg
+
+def device_weights(shape, device, seed=0):
+    """Random-init weights drawn on the device (same distribution as workloads.make_weights)."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    d, F, V = shape.d_model, shape.d_ff, shape.vocab
+    hd = shape.n_heads * shape.head_dim
+
+    def mat(r, c):
+        return (torch.randn(r, c, generator=g, device=device, dtype=torch.float32) * 0.02).to(torch.bfloat16)
+
+    ones = torch.ones(d, device=device, dtype=torch.float32)
+    layers = []
+    for _ in range(shape.n_layers):
+        layers.append({"wqkv": mat(3 * hd, d), "wo": mat(d, hd), "w_gate": mat(F, d), "w_up": mat(F, d),
+                       "w_down": mat(d, F), "norm1": ones, "norm2": ones})
+    return {"tok_emb": mat(V, d), "lm_head": mat(V, d),
+            "final_norm": torch.full((d,), wl.spread_gain(shape), device=device, dtype=torch.float32), "layers": layers}
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            pass
+        self.f.flush()
+        rows = [r.split(",") for r in open(self.f.name).read().strip().splitlines() if r.count(",") >= 8]
+        os.unlink(self.f.name)
+        if not rows:
+            return out
+        sm = [float(r[1]) for r in rows]
+        out["sm_mhz"] = statistics.median(sm)
+        out["sm_max_mhz"] = float(rows[0][2])
+        out["power_w_max"] = max(float(r[3]) for r in rows)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        out["reasons"] = [n for i, n in enumerate(names) if any("Active" == r[5 + i].strip() for r in rows)]
+        out["samples"] = len(rows)
+        return out
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2509_25188_b200 import binding
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = "cuda:%d" % local
+    pk, pk_src = peaks()
+
+    w = device_weights(SHAPE, dev)
+    filt = wl.make_filter(DEC.block_len, DEC.tau, seed=0)
+    B, P, G, s = DEC.batch, DEC.prompt_len, DEC.gen_len, DEC.block_len
+    dec = binding.Decoder(SHAPE, w, filt, block_len=s, tau=DEC.tau, max_batch=B, max_seq=P + G, device=local)
+    prompts = wl.make_prompts(B, P, SHAPE, seed=1 + rank)
+    h_prompts = torch.from_numpy(prompts).pin_memory()
+    d_prompts = h_prompts.to(dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def one_resident():
+        dec.state_reset_device(d_prompts, G)
+        return dec.denoise_step_host()
+
+    for _ in range(max(args.warmup, 3)):
+        one_resident()
+
+    # ---- timed region 1: inputs resident in HBM
+    sampler = ClockSampler(local) if rank == 0 else None
+    dec.profile_enable(["gemm_gate_up"])
+    launches0 = dec.launch_count
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    tokens = 0
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        h = one_resident()
+        tokens += int((s - h["masks_left"]).sum())
+    ev1.record()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = dec.launch_count - launches0
+    prof = dec.profile_read()
+    dec.profile_enable([])
+
+    # ---- timed region 2: host buffers in, host results out, through the same calls
+    dev_in = torch.empty_like(d_prompts)
+    o_conf = torch.empty(B, s, device=dev)
+    o_pred = torch.empty(B, s, dtype=torch.int32, device=dev)
+    o_un = torch.empty(B, s, dtype=torch.uint8, device=dev)
+    h_conf, h_pred, h_un = (torch.empty_like(t, device="cpu").pin_memory() for t in (o_conf, o_pred, o_un))
+    tokens_e2e = 0
+    barrier()
+    ev0.record()
+    for _ in range(args.steps):
+        dev_in.copy_(h_prompts, non_blocking=True)
+        dec.state_reset_device(dev_in, G)
+        dec.denoise_step_into(o_conf, o_pred, o_un)
+        h_conf.copy_(o_conf, non_blocking=True)
+        h_pred.copy_(o_pred, non_blocking=True)
+        h_un.copy_(o_un, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        tokens_e2e += int(h_un.sum())
+    ev1.record()
+    barrier()
+    ms_e2e = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if sampler else None
+
+    if world > 1:
+        t = torch.tensor([ms, ms_e2e], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, ms_e2e = float(t[0]), float(t[1])
+        c = torch.tensor([tokens, tokens_e2e, launches], device=dev, dtype=torch.float64)
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+        tokens, tokens_e2e, launches = int(c[0]), int(c[1]), int(c[2])
+
+    # ---- untimed: per-kernel breakdown of one step
+    breakdown = {}
+    if rank == 0:
+        dec.profile_enable(binding.KINDS)
+        for _ in range(3):
+            one_resident()
+        for k, (t_ms, n) in dec.profile_read().items():
+            breakdown[k] = {"ms_per_step": round(t_ms / 3, 4), "launches_per_step": n // 3}
+        dec.profile_enable([])
+
+    if rank == 0:
+        T, R = B * (P + G), B * s
+        work = step_work(SHAPE, T, P + G, R)
+        t_flops = work["flops"] / (pk["bf16_tflops_sustained"] * 1e12)
+        t_bytes = (work["weight_bytes"] + work["act_bytes"]) / (pk["hbm_gbs"] * 1e9)
+        t_roof_ms = 1e3 * max(t_flops, t_bytes)
+        ms_step = ms / args.steps
+        gu_ms, gu_n = prof.get("gemm_gate_up", (0.0, 0))
+        gu_flops = 2.0 * T * SHAPE.d_model * 2 * SHAPE.d_ff
+        achieved = gu_flops / (gu_ms / gu_n * 1e-3) / 1e12 if gu_n else None
+        line = {
+            "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config_dict(),
+            "clocks": clocks,
+            "e2e": {"value": tokens_e2e / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e / args.steps,
+                    "h2d_bytes_per_step": int(h_prompts.numel() * 4),
+                    "d2h_bytes_per_step": int(h_conf.numel() * 4 + h_pred.numel() * 4 + h_un.numel() + 6 * 4 * B + 4)},
+            "gpu_launches": int(launches),
+            "tokens_per_step": tokens / (args.steps * world),
+            "roofline": {"kernel": "gemm_tcgen05_kernel<EPI_SWIGLU> (gate/up projection + SwiGLU)", "bound": "tensor",
+                         "achieved": achieved, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                         "frac": (achieved / pk["bf16_tflops_sustained"]) if achieved else None,
+                         "peak_source": pk_src + " (sustained bf16, kernel timed inside a long step)",
+                         "flops_per_launch": gu_flops, "avg_launch_ms": gu_ms / gu_n if gu_n else None,
+                         "traffic": None},
+            "step_roofline": {"flops": work["flops"], "weight_bytes": work["weight_bytes"], "act_bytes": work["act_bytes"],
+                              "t_flops_ms": 1e3 * t_flops, "t_bytes_ms": 1e3 * t_bytes, "t_roof_ms": t_roof_ms,
+                              "frac": t_roof_ms / ms_step, "peaks": pk, "peak_source": pk_src},
+            "breakdown": breakdown,
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            import threadpoolctl
+            smp = OracleSample()
+            cores = max(i["num_threads"] for i in threadpoolctl.threadpool_info() or [{"num_threads": os.cpu_count()}])
+            smp.one()
+            full_s, n_tok, raw = smp.one()
+            line["cpu_baseline"] = {
+                "value": (tokens / (args.steps * world)) / full_s, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "ms_per_step": 1e3 * full_s,
+                "sample": "embedding + %d of %d layers + LM head/decision on %d rows at T=%d (%.1f s measured), layer "
+                          "time scaled x%d; tokens per step taken from the GPU run of the same workload"
+                          % (smp.n_sample, SHAPE.n_layers, s, T, raw, SHAPE.n_layers // smp.n_sample)}
+        print(json.dumps(line))
+    dec.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps == 30:
+            args.steps = 3
+        if args.warmup == 5:
+            args.warmup = 1
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -184,6 +184,29 @@ int32_t l2pd_last_step_rows(const l2pd_ctx *ctx);
 /* Kernels launched by this context since creation (for launch accounting). */
 int64_t l2pd_launch_count(const l2pd_ctx *ctx);
 
+/*
+ * Per-kernel timing.  Kinds of kernels a step launches: */
+enum {
+  L2PD_K_EMBED = 0,       /* embedding gather + first RMSNorm */
+  L2PD_K_GEMM_QKV = 1,    /* fused QKV projection */
+  L2PD_K_ROPE = 2,        /* rotary embedding + K/V scatter */
+  L2PD_K_ATTENTION = 3,   /* bidirectional attention */
+  L2PD_K_GEMM_O = 4,      /* output projection + residual */
+  L2PD_K_RMSNORM = 5,     /* RMSNorm */
+  L2PD_K_GEMM_GATE_UP = 6,/* gate/up projection + SwiGLU */
+  L2PD_K_GEMM_DOWN = 7,   /* down projection + residual */
+  L2PD_K_FINAL_NORM = 8,  /* block-row gather + final RMSNorm */
+  L2PD_K_LM_HEAD = 9,     /* LM head + confidence/argmax reduction */
+  L2PD_K_DECIDE = 10,     /* filter, threshold, commit, EoTP */
+  L2PD_K_OTHER = 11,
+  L2PD_K_COUNT = 12
+};
+/* Selects kinds (bit k = kind k) whose launches are bracketed by CUDA events on the step's
+ * stream from now on, and clears the accumulated totals; mask 0 turns timing off. */
+l2pd_status l2pd_profile_enable(l2pd_ctx *ctx, uint32_t kind_mask);
+/* Accumulated device time (ms) and launch count of one kind since the last enable. */
+l2pd_status l2pd_profile_read(const l2pd_ctx *ctx, int32_t kind, double *ms_total, int64_t *launches);
+
 /* Device time of the most recent step in milliseconds (CUDA events on the step's stream),
  * or a negative value if no step has run. */
 float l2pd_last_step_ms(const l2pd_ctx *ctx);

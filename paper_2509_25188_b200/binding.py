@@ -56,9 +56,13 @@ class StepOut(C.Structure):
 
 EXPORTS = ["l2pd_init", "l2pd_state_reset", "l2pd_denoise_step", "l2pd_decode", "l2pd_num_active",
            "l2pd_state_tokens", "l2pd_state_masked", "l2pd_set_capture", "l2pd_last_step_rows",
-           "l2pd_launch_count", "l2pd_last_step_ms", "l2pd_last_error", "l2pd_destroy",
+           "l2pd_launch_count", "l2pd_last_step_ms", "l2pd_profile_enable", "l2pd_profile_read", "l2pd_last_error", "l2pd_destroy",
            "l2pd_gemm_bf16", "l2pd_gemm_bf16_residual", "l2pd_gemm_bf16_swiglu", "l2pd_lm_head_bf16",
            "l2pd_lm_head_scratch_elems", "l2pd_attention_bf16"]
+
+
+KINDS = ["embed", "gemm_qkv", "rope", "attention", "gemm_o", "rmsnorm", "gemm_gate_up", "gemm_down",
+         "final_norm", "lm_head", "decide", "other"]
 
 
 def _load() -> C.CDLL:
@@ -82,6 +86,8 @@ def _load() -> C.CDLL:
     lib.l2pd_launch_count.restype = i64
     lib.l2pd_last_step_ms.argtypes = [vp]
     lib.l2pd_last_step_ms.restype = f32
+    lib.l2pd_profile_enable.argtypes = [vp, C.c_uint32]
+    lib.l2pd_profile_read.argtypes = [vp, i32, C.POINTER(C.c_double), C.POINTER(i64)]
     lib.l2pd_last_error.argtypes = [vp]
     lib.l2pd_last_error.restype = C.c_char_p
     lib.l2pd_destroy.argtypes = [vp]
@@ -208,6 +214,26 @@ class Decoder:
         out.update(h)
         return out
 
+    def state_reset_device(self, d_prompts: torch.Tensor, G: int):
+        """state_reset on a caller-owned device tensor int32 [B, P] (no copy, no allocation)."""
+        self.B, self.P, self.G = int(d_prompts.shape[0]), int(d_prompts.shape[1]), int(G)
+        _check(lib.l2pd_state_reset(self.ctx, _stream(), d_prompts.data_ptr(), self.B, self.P, self.G), self.ctx)
+
+    def denoise_step_host(self) -> dict:
+        """One step; returns only the per-sequence host record (no device outputs)."""
+        if getattr(self, "_hrec", None) is None or len(self._hrec["done"]) != self.B:
+            self._hrec = {k: np.full(self.B, -1, np.int32) for k in ("block", "masks_left", "l_eff", "done", "forced")}
+        h = self._hrec
+        o = StepOut(h_block=h["block"].ctypes.data, h_masks_left=h["masks_left"].ctypes.data,
+                    h_l_eff=h["l_eff"].ctypes.data, h_done=h["done"].ctypes.data, h_forced=h["forced"].ctypes.data)
+        _check(lib.l2pd_denoise_step(self.ctx, _stream(), C.byref(o)), self.ctx)
+        return h
+
+    def denoise_step_into(self, d_conf: torch.Tensor, d_pred: torch.Tensor, d_unmask: torch.Tensor):
+        """One step writing conf / pred / unmask [B, s] into caller-owned device tensors."""
+        o = StepOut(d_conf=d_conf.data_ptr(), d_pred=d_pred.data_ptr(), d_unmask=d_unmask.data_ptr())
+        _check(lib.l2pd_denoise_step(self.ctx, _stream(), C.byref(o)), self.ctx)
+
     def decode(self, prompts, G: int):
         """Returns (tokens [B,G] int32 numpy, out_len [B], steps [B], total_steps)."""
         p = prompts if isinstance(prompts, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(prompts))
@@ -252,6 +278,21 @@ class Decoder:
             _check(lib.l2pd_set_capture(self.ctx, None, 0), self.ctx)
         else:
             _check(lib.l2pd_set_capture(self.ctx, tensor.data_ptr(), tensor.stride(0)), self.ctx)
+
+    def profile_enable(self, kinds):
+        mask = 0
+        for k in kinds:
+            mask |= 1 << KINDS.index(k)
+        _check(lib.l2pd_profile_enable(self.ctx, mask), self.ctx)
+
+    def profile_read(self) -> dict:
+        out = {}
+        for i, k in enumerate(KINDS):
+            ms, n = C.c_double(0), C.c_int64(0)
+            _check(lib.l2pd_profile_read(self.ctx, i, C.byref(ms), C.byref(n)), self.ctx)
+            if n.value:
+                out[k] = (ms.value, n.value)
+        return out
 
     @property
     def last_step_rows(self) -> int:

@@ -66,6 +66,13 @@ struct l2pd_ctx {
 
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   float last_ms = -1.f;
+
+  // per-kernel timing (CUDA events around the launches of the selected kinds)
+  uint32_t prof_mask = 0;
+  std::vector<cudaEvent_t> prof_events;          // pairs: begin, end
+  std::vector<int> prof_pending_kind;            // kind of each recorded pair of the current step
+  double prof_ms[L2PD_K_COUNT] = {};
+  int64_t prof_launches[L2PD_K_COUNT] = {};
   int64_t launches = 0;
   std::string err;
 };
@@ -93,6 +100,43 @@ l2pd_status set_err(l2pd_ctx *c, l2pd_status s, const char *fmt, ...) {
   } while (0)
 #define CKL(call)                                                                                  \
   do { CK(call); c->launches++; } while (0)
+// launch of a profiled kind: bracketed by events when that kind is selected
+#define CKLK(kind, call)                                                                           \
+  do {                                                                                             \
+    const bool prof_ = (c->prof_mask >> (kind)) & 1u;                                              \
+    if (prof_) CK(prof_mark(c, s, (kind), true));                                                  \
+    CK(call);                                                                                      \
+    c->launches++;                                                                                 \
+    if (prof_) CK(prof_mark(c, s, (kind), false));                                                 \
+  } while (0)
+
+cudaError_t prof_mark(l2pd_ctx *c, cudaStream_t s, int kind, bool begin) {
+  size_t idx = c->prof_pending_kind.size() * 2 + (begin ? 0 : 1);
+  if (!begin) idx -= 2;
+  while (c->prof_events.size() <= idx) {
+    cudaEvent_t e;
+    cudaError_t r = cudaEventCreate(&e);
+    if (r != cudaSuccess) return r;
+    c->prof_events.push_back(e);
+  }
+  if (begin) {
+    cudaError_t r = cudaEventRecord(c->prof_events[idx], s);
+    if (r == cudaSuccess) c->prof_pending_kind.push_back(kind);
+    return r;
+  }
+  return cudaEventRecord(c->prof_events[idx], s);
+}
+
+void prof_collect(l2pd_ctx *c) {
+  for (size_t i = 0; i < c->prof_pending_kind.size(); ++i) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, c->prof_events[2 * i], c->prof_events[2 * i + 1]) == cudaSuccess) {
+      c->prof_ms[c->prof_pending_kind[i]] += ms;
+      c->prof_launches[c->prof_pending_kind[i]] += 1;
+    }
+  }
+  c->prof_pending_kind.clear();
+}
 
 template <typename T>
 l2pd_status dev_alloc(l2pd_ctx *c, T **p, int64_t count) {
@@ -116,18 +160,18 @@ l2pd_status encode_weight_maps(l2pd_ctx *c, std::vector<TmaDesc> &dst, const std
 
 // One GEMM of the step, dispatched by dtype.
 template <typename T>
-l2pd_status run_gemm_simt(l2pd_ctx *c, cudaStream_t s, int epi, const void *A, const void *W, const void *W2,
-                          void *out, const float *bias, int M, int N, int K) {
-  CKL(launch_simt_gemm<T>(s, epi, (const T *)A, (const T *)W, (const T *)W2, out, bias, M, N, K));
+l2pd_status run_gemm_simt(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const void *A, const void *W,
+                          const void *W2, void *out, const float *bias, int M, int N, int K) {
+  CKLK(kind, launch_simt_gemm<T>(s, epi, (const T *)A, (const T *)W, (const T *)W2, out, bias, M, N, K));
   return L2PD_OK;
 }
 
-l2pd_status run_gemm_tc(l2pd_ctx *c, cudaStream_t s, int epi, const TmaDesc *a, const TmaDesc *b, const TmaDesc *b2,
-                        void *out, int M, int N, int K, int tile_n) {
+l2pd_status run_gemm_tc(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const TmaDesc *a, const TmaDesc *b,
+                        const TmaDesc *b2, void *out, int M, int N, int K, int tile_n) {
   GemmArgs g{};
   g.epi = epi; g.a = a; g.b = b; g.b2 = b2; g.M = M; g.N = N; g.K = K; g.tile_n = tile_n; g.out = out;
   g.status = c->d_status;
-  CKL(launch_gemm_tcgen05(s, g, c->num_sms));
+  CKLK(kind, launch_gemm_tcgen05(s, g, c->num_sms));
   return L2PD_OK;
 }
 
@@ -154,8 +198,8 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     }
   }
 
-  CKL(launch_build_row_map(s, c->d_meta, n_slots, c->d_row_slot));
-  CKL(launch_embed_rmsnorm<T>(s, c->d_tokens, c->P + c->G, c->d_meta, c->d_row_slot, (const T *)c->tok_emb,
+  CKLK(L2PD_K_OTHER, launch_build_row_map(s, c->d_meta, n_slots, c->d_row_slot));
+  CKLK(L2PD_K_EMBED, launch_embed_rmsnorm<T>(s, c->d_tokens, c->P + c->G, c->d_meta, c->d_row_slot, (const T *)c->tok_emb,
                               c->norm1[0], f.rms_eps, c->x, n, T_rows, d));
   if (c->cap) CK(cudaMemcpyAsync(c->cap, c->x, (size_t)T_rows * d * 4, cudaMemcpyDeviceToDevice, s));
 
@@ -163,35 +207,35 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     T *kc = (T *)c->kc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
     T *vc = (T *)c->vc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
     l2pd_status r;
-    if (tc) r = run_gemm_tc(c, s, EPI_STORE, &c->ta_n, &c->tb_qkv[l], nullptr, qkv, T_rows, 3 * hd, d, c->tn_qkv);
-    else r = run_gemm_simt<T>(c, s, EPI_STORE, n, c->wqkv[l], nullptr, qkv, nullptr, T_rows, 3 * hd, d);
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_QKV, EPI_STORE, &c->ta_n, &c->tb_qkv[l], nullptr, qkv, T_rows, 3 * hd, d, c->tn_qkv);
+    else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_QKV, EPI_STORE, n, c->wqkv[l], nullptr, qkv, nullptr, T_rows, 3 * hd, d);
     if (r) return r;
-    CKL(launch_rope_scatter<T>(s, qkv, c->d_meta, c->d_row_slot, c->cs_table, q, kc, vc, c->kv_seq_stride, T_rows, H, dh));
+    CKLK(L2PD_K_ROPE, launch_rope_scatter<T>(s, qkv, c->d_meta, c->d_row_slot, c->cs_table, q, kc, vc, c->kv_seq_stride, T_rows, H, dh));
     if (tc) {
-      CKL(launch_attention_bf16(s, (const bf16 *)q, (const bf16 *)kc, (const bf16 *)vc, c->d_meta, (bf16 *)att, hd, hd,
+      CKLK(L2PD_K_ATTENTION, launch_attention_bf16(s, (const bf16 *)q, (const bf16 *)kc, (const bf16 *)vc, c->d_meta, (bf16 *)att, hd, hd,
                                 c->kv_seq_stride, hd, n_slots, max_q_rows, H, dh));
     } else {
-      CKL(launch_simt_attention<T>(s, q, kc, vc, c->d_meta, c->d_row_slot, att, c->kv_seq_stride, T_rows, H, dh, max_kv));
+      CKLK(L2PD_K_ATTENTION, launch_simt_attention<T>(s, q, kc, vc, c->d_meta, c->d_row_slot, att, c->kv_seq_stride, T_rows, H, dh, max_kv));
     }
-    if (tc) r = run_gemm_tc(c, s, EPI_RESIDUAL, &c->ta_att, &c->tb_o[l], nullptr, c->x, T_rows, d, hd, c->tn_o);
-    else r = run_gemm_simt<T>(c, s, EPI_RESIDUAL, att, c->wo[l], nullptr, c->x, nullptr, T_rows, d, hd);
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_O, EPI_RESIDUAL, &c->ta_att, &c->tb_o[l], nullptr, c->x, T_rows, d, hd, c->tn_o);
+    else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_O, EPI_RESIDUAL, att, c->wo[l], nullptr, c->x, nullptr, T_rows, d, hd);
     if (r) return r;
-    CKL(launch_rmsnorm<T>(s, c->x, c->norm2[l], f.rms_eps, n, T_rows, d));
-    if (tc) r = run_gemm_tc(c, s, EPI_SWIGLU, &c->ta_n, &c->tb_gate[l], &c->tb_up[l], hbuf, T_rows, F, d, c->tn_gu);
-    else r = run_gemm_simt<T>(c, s, EPI_SWIGLU, n, c->w_gate[l], c->w_up[l], hbuf, nullptr, T_rows, F, d);
+    CKLK(L2PD_K_RMSNORM, launch_rmsnorm<T>(s, c->x, c->norm2[l], f.rms_eps, n, T_rows, d));
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_GATE_UP, EPI_SWIGLU, &c->ta_n, &c->tb_gate[l], &c->tb_up[l], hbuf, T_rows, F, d, c->tn_gu);
+    else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_GATE_UP, EPI_SWIGLU, n, c->w_gate[l], c->w_up[l], hbuf, nullptr, T_rows, F, d);
     if (r) return r;
-    if (tc) r = run_gemm_tc(c, s, EPI_RESIDUAL, &c->ta_h, &c->tb_down[l], nullptr, c->x, T_rows, d, F, c->tn_down);
-    else r = run_gemm_simt<T>(c, s, EPI_RESIDUAL, hbuf, c->w_down[l], nullptr, c->x, nullptr, T_rows, d, F);
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_DOWN, EPI_RESIDUAL, &c->ta_h, &c->tb_down[l], nullptr, c->x, T_rows, d, F, c->tn_down);
+    else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_DOWN, EPI_RESIDUAL, hbuf, c->w_down[l], nullptr, c->x, nullptr, T_rows, d, F);
     if (r) return r;
     if (c->cap)
       CK(cudaMemcpyAsync(c->cap + (int64_t)(l + 1) * c->cap_stride, c->x, (size_t)T_rows * d * 4, cudaMemcpyDeviceToDevice, s));
-    if (l + 1 < f.n_layers) CKL(launch_rmsnorm<T>(s, c->x, c->norm1[l + 1], f.rms_eps, n, T_rows, d));
+    if (l + 1 < f.n_layers) CKLK(L2PD_K_RMSNORM, launch_rmsnorm<T>(s, c->x, c->norm1[l + 1], f.rms_eps, n, T_rows, d));
   }
 
   // confidence head on the current block's rows
   const int R = n_slots * sb;
   const int rows_padded = tc ? (int)round_up(R, 128) : R;
-  CKL(launch_final_norm_gather<T>(s, c->x, c->d_meta, c->final_norm, f.rms_eps, nf, n_slots, sb, rows_padded, d));
+  CKLK(L2PD_K_FINAL_NORM, launch_final_norm_gather<T>(s, c->x, c->d_meta, c->final_norm, f.rms_eps, nf, n_slots, sb, rows_padded, d));
   int n_tiles = 1;
   float *part_m, *part_s;
   int32_t *part_i;
@@ -216,13 +260,13 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
       g.logits = c->logits_f32;
       tmp_logits = c->logits_f32;
     }
-    CKL(launch_gemm_tcgen05(s, g, c->num_sms));
+    CKLK(L2PD_K_LM_HEAD, launch_gemm_tcgen05(s, g, c->num_sms));
     (void)tmp_logits;
   } else {
     part_m = c->part; part_s = part_m + rows_padded; part_i = (int32_t *)(part_s + rows_padded);
-    l2pd_status r = run_gemm_simt<T>(c, s, EPI_STORE_F32, nf, c->lm_head, nullptr, c->logits_f32, c->lm_bias, R, V, d);
+    l2pd_status r = run_gemm_simt<T>(c, s, L2PD_K_LM_HEAD, EPI_STORE_F32, nf, c->lm_head, nullptr, c->logits_f32, c->lm_bias, R, V, d);
     if (r) return r;
-    CKL(launch_row_softmax_partials(s, c->logits_f32, R, V, part_m, part_s, part_i));
+    CKLK(L2PD_K_LM_HEAD, launch_row_softmax_partials(s, c->logits_f32, R, V, part_m, part_s, part_i));
   }
   if (out && out->d_logits) {
     for (int i = 0; i < n_slots; ++i) {
@@ -241,7 +285,7 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
   a.use_filter = f.use_filter; a.use_eotp = f.use_eotp; a.committed_conf_mode = f.committed_conf_mode;
   a.eot_id = f.eot_id; a.summary = c->d_summary;
   if (out) { a.o_conf = out->d_conf; a.o_pred = out->d_pred; a.o_p = out->d_p; a.o_unmask = out->d_unmask; }
-  CKL(launch_decide(s, a, n_slots));
+  CKLK(L2PD_K_DECIDE, launch_decide(s, a, n_slots));
   return L2PD_OK;
 }
 
@@ -253,6 +297,7 @@ void free_all(l2pd_ctx *c) {
   if (c->h_meta) cudaFreeHost(c->h_meta);
   if (c->h_summary) cudaFreeHost(c->h_summary);
   if (c->h_status) cudaFreeHost(c->h_status);
+  for (cudaEvent_t e : c->prof_events) cudaEventDestroy(e);
   if (c->ev0) cudaEventDestroy(c->ev0);
   if (c->ev1) cudaEventDestroy(c->ev1);
 }
@@ -448,6 +493,7 @@ l2pd_status l2pd_denoise_step(l2pd_ctx *c, void *stream, const l2pd_step_out *ou
   CK(cudaEventRecord(c->ev1, s));
   CK(cudaStreamSynchronize(s));
   CK(cudaEventElapsedTime(&c->last_ms, c->ev0, c->ev1));
+  prof_collect(c);
   if (*c->h_status != DEV_OK) {
     const int code = *c->h_status;
     cudaMemsetAsync(c->d_status, 0, 4, s);
@@ -507,6 +553,19 @@ l2pd_status l2pd_set_capture(l2pd_ctx *c, float *d_resid, int64_t slot_stride_el
 int32_t l2pd_last_step_rows(const l2pd_ctx *c) { return c ? c->last_rows : 0; }
 int64_t l2pd_launch_count(const l2pd_ctx *c) { return c ? c->launches : 0; }
 float l2pd_last_step_ms(const l2pd_ctx *c) { return c ? c->last_ms : -1.f; }
+l2pd_status l2pd_profile_enable(l2pd_ctx *c, uint32_t kind_mask) {
+  if (!c) return L2PD_ERR_ARG;
+  c->prof_mask = kind_mask & ((1u << L2PD_K_COUNT) - 1u);
+  c->prof_pending_kind.clear();
+  for (int k = 0; k < L2PD_K_COUNT; ++k) { c->prof_ms[k] = 0.0; c->prof_launches[k] = 0; }
+  return L2PD_OK;
+}
+l2pd_status l2pd_profile_read(const l2pd_ctx *c, int32_t kind, double *ms_total, int64_t *launches) {
+  if (!c || kind < 0 || kind >= L2PD_K_COUNT) return L2PD_ERR_ARG;
+  if (ms_total) *ms_total = c->prof_ms[kind];
+  if (launches) *launches = c->prof_launches[kind];
+  return L2PD_OK;
+}
 const char *l2pd_last_error(const l2pd_ctx *c) { return c ? c->err.c_str() : "null context"; }
 
 void l2pd_destroy(l2pd_ctx *c) {

@@ -1,0 +1,109 @@
+"""Runs one kernel of the denoising step stand-alone, at a layer's real shapes, and times it.
+
+  python -m paper_2509_25188_b200.kernel_cases gate_up --rows 512 [--iters 20] [--tile-n 0]
+
+Cases (LLaDA-8B layer shapes unless overridden with --d/--ff/--vocab/--heads):
+  qkv      C[T,3d]  = A[T,d] Wqkv^T                 bf16 store epilogue
+  o        X[T,d]  += A[T,d] Wo^T                   residual epilogue
+  gate_up  H[T,F]   = silu(A Wg^T) * (A Wu^T)       SwiGLU epilogue
+  down     X[T,d]  += H[T,F] Wd^T                   residual epilogue
+  lm_head  pred/conf over V for R = --rows rows     fused confidence head
+  attn     bidirectional attention, --rows queries and keys, 32 heads x 128
+
+Each iteration uses a different weight buffer out of a ring larger than L2 (126 MB), so that the
+weights come from HBM as they do inside a step.  Prints one JSON line with the mean device time
+(CUDA events on the launching stream) and the achieved TFLOP/s and GB/s.  Used for tuning and as
+the small, self-ending case for profiler captures.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import binding as b
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("case", choices=["qkv", "o", "gate_up", "down", "lm_head", "attn"])
+    ap.add_argument("--rows", type=int, default=512)
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--tile-n", type=int, default=0)
+    ap.add_argument("--d", type=int, default=4096)
+    ap.add_argument("--ff", type=int, default=12288)
+    ap.add_argument("--vocab", type=int, default=126464)
+    ap.add_argument("--heads", type=int, default=32)
+    a = ap.parse_args()
+    dev = "cuda:0"
+    torch.manual_seed(0)
+    T, d, F, V, H = a.rows, a.d, a.ff, a.vocab, a.heads
+    dh = d // H
+
+    def rnd(r, c, std=0.02):
+        return (torch.randn(r, c, device=dev) * std).to(torch.bfloat16)
+
+    def ring(r, c, min_bytes=400e6):
+        n = max(2, int(min_bytes // (r * c * 2)) + 1)
+        return [rnd(r, c) for _ in range(n)]
+
+    if a.case == "qkv":
+        A, W = rnd(T, d, 1.0), ring(3 * d, d)
+        Cc = torch.empty(T, 3 * d, dtype=torch.bfloat16, device=dev)
+        run = lambda i: b._check(b.lib.l2pd_gemm_bf16(b._stream(), A.data_ptr(), W[i % len(W)].data_ptr(),
+                                                      Cc.data_ptr(), T, 3 * d, d, a.tile_n, 0))
+        flops, byts = 2.0 * T * d * 3 * d, 2.0 * (3 * d * d + T * d + T * 3 * d)
+    elif a.case == "o":
+        A, W, X = rnd(T, d, 1.0), ring(d, d), torch.zeros(T, d, device=dev)
+        run = lambda i: b._check(b.lib.l2pd_gemm_bf16_residual(b._stream(), A.data_ptr(), W[i % len(W)].data_ptr(),
+                                                               X.data_ptr(), T, d, d, a.tile_n, 0))
+        flops, byts = 2.0 * T * d * d, 2.0 * (d * d + T * d) + 8.0 * T * d
+    elif a.case == "gate_up":
+        A, Wg, Wu = rnd(T, d, 1.0), ring(F, d, 200e6), ring(F, d, 200e6)
+        Hh = torch.empty(T, F, dtype=torch.bfloat16, device=dev)
+        run = lambda i: b._check(b.lib.l2pd_gemm_bf16_swiglu(b._stream(), A.data_ptr(), Wg[i % len(Wg)].data_ptr(),
+                                                             Wu[i % len(Wu)].data_ptr(), Hh.data_ptr(), T, F, d,
+                                                             a.tile_n, 0))
+        flops, byts = 2.0 * T * d * 2 * F, 2.0 * (2 * F * d + T * d + T * F)
+    elif a.case == "down":
+        A, W, X = rnd(T, F, 1.0), ring(d, F), torch.zeros(T, d, device=dev)
+        run = lambda i: b._check(b.lib.l2pd_gemm_bf16_residual(b._stream(), A.data_ptr(), W[i % len(W)].data_ptr(),
+                                                               X.data_ptr(), T, d, F, a.tile_n, 0))
+        flops, byts = 2.0 * T * d * F, 2.0 * (d * F + T * F) + 8.0 * T * d
+    elif a.case == "lm_head":
+        A, W = rnd(T, d, 1.0), ring(V, d, 1.1e9)
+        scratch = torch.empty(b.lib.l2pd_lm_head_scratch_elems(T, V), device=dev)
+        pred = torch.empty(T, dtype=torch.int32, device=dev)
+        conf = torch.empty(T, device=dev)
+
+        def run(i):
+            b._check(b.lib.l2pd_lm_head_bf16(b._stream(), A.data_ptr(), W[i % len(W)].data_ptr(), None, T, V, d,
+                                             scratch.data_ptr(), pred.data_ptr(), conf.data_ptr(), None, 0))
+        flops, byts = 2.0 * T * d * V, 2.0 * (V * d + T * d)
+    else:
+        q, k, v = rnd(T, d, 1.0), rnd(T, d, 1.0), rnd(T, d, 1.0)
+        out = torch.empty(T, d, dtype=torch.bfloat16, device=dev)
+        run = lambda i: b._check(b.lib.l2pd_attention_bf16(b._stream(), q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                                           out.data_ptr(), T, T, H, dh, d, d, d))
+        flops, byts = 4.0 * T * T * d, 2.0 * 4 * T * d
+
+    for i in range(a.warmup):
+        run(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    tot = 0.0
+    for i in range(a.iters):
+        e0.record()
+        run(i)
+        e1.record()
+        torch.cuda.synchronize()
+        tot += e0.elapsed_time(e1)
+    ms = tot / a.iters
+    print(json.dumps({"case": a.case, "rows": T, "tile_n": a.tile_n, "ms": ms, "tflops": flops / ms / 1e9,
+                      "gbs": byts / ms / 1e6, "flops": flops, "bytes": byts}))
+
+
+if __name__ == "__main__":
+    main()
