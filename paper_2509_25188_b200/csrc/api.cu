@@ -57,7 +57,8 @@ struct l2pd_ctx {
   TmaDesc ta_n, ta_att, ta_h, ta_nf;
   std::vector<TmaDesc> tb_qkv, tb_o, tb_gate, tb_up, tb_down;
   TmaDesc tb_lm;
-  int tn_qkv = 0, tn_o = 0, tn_gu = 0, tn_down = 0, tn_lm = 0;
+  GemmPlan pl_qkv{}, pl_o{}, pl_gu{}, pl_down{};
+  int box_qkv = 0, box_o = 0, box_gu = 0, box_down = 0, tn_lm = 0;
 
   // debug capture
   float *cap = nullptr;
@@ -167,9 +168,10 @@ l2pd_status run_gemm_simt(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const 
 }
 
 l2pd_status run_gemm_tc(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const TmaDesc *a, const TmaDesc *b,
-                        const TmaDesc *b2, void *out, int M, int N, int K, int tile_n) {
+                        const TmaDesc *b2, void *out, int M, int N, int K, const GemmPlan &pl) {
   GemmArgs g{};
-  g.epi = epi; g.a = a; g.b = b; g.b2 = b2; g.M = M; g.N = N; g.K = K; g.tile_n = tile_n; g.out = out;
+  g.epi = epi; g.a = a; g.b = b; g.b2 = b2; g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.out = out;
+  g.cta_group = pl.cta_group; g.k_splits = pl.k_splits;
   g.status = c->d_status;
   CKLK(kind, launch_gemm_tcgen05(s, g, c->num_sms));
   return L2PD_OK;
@@ -184,17 +186,23 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
   T *n = (T *)c->n, *qkv = (T *)c->qkv, *q = (T *)c->q, *att = (T *)c->att, *hbuf = (T *)c->h, *nf = (T *)c->nf;
 
   if (tc) {
-    // tile widths follow the row count of this step; weight tensor maps are re-encoded when they change
-    int tn = pick_tile_n(T_rows, 3 * hd, c->num_sms, 16, 256);
-    if (tn != c->tn_qkv) { l2pd_status r = encode_weight_maps(c, c->tb_qkv, c->wqkv, 3 * hd, d, tn); if (r) return r; c->tn_qkv = tn; }
-    tn = pick_tile_n(T_rows, d, c->num_sms, 16, 256);
-    if (tn != c->tn_o) { l2pd_status r = encode_weight_maps(c, c->tb_o, c->wo, d, hd, tn); if (r) return r; c->tn_o = tn; }
-    if (tn != c->tn_down) { l2pd_status r = encode_weight_maps(c, c->tb_down, c->w_down, d, F, tn); if (r) return r; c->tn_down = tn; }
-    tn = 2 * pick_tile_n(T_rows, F, c->num_sms, 16, 128);
-    if (tn != c->tn_gu) {
-      l2pd_status r = encode_weight_maps(c, c->tb_gate, c->w_gate, F, d, tn / 2); if (r) return r;
-      r = encode_weight_maps(c, c->tb_up, c->w_up, F, d, tn / 2); if (r) return r;
-      c->tn_gu = tn;
+    // the tiling follows the row count of this step; weight tensor maps are re-encoded when the
+    // box (rows of the weight tile one CTA loads) changes
+    c->pl_qkv = plan_gemm(EPI_STORE, T_rows, 3 * hd, d, c->num_sms, 0);
+    int box = c->pl_qkv.tile_n / c->pl_qkv.cta_group;
+    if (box != c->box_qkv) { l2pd_status r = encode_weight_maps(c, c->tb_qkv, c->wqkv, 3 * hd, d, box); if (r) return r; c->box_qkv = box; }
+    c->pl_o = plan_gemm(EPI_RESIDUAL, T_rows, d, hd, c->num_sms, 0);
+    box = c->pl_o.tile_n / c->pl_o.cta_group;
+    if (box != c->box_o) { l2pd_status r = encode_weight_maps(c, c->tb_o, c->wo, d, hd, box); if (r) return r; c->box_o = box; }
+    c->pl_down = plan_gemm(EPI_RESIDUAL, T_rows, d, F, c->num_sms, 0);
+    box = c->pl_down.tile_n / c->pl_down.cta_group;
+    if (box != c->box_down) { l2pd_status r = encode_weight_maps(c, c->tb_down, c->w_down, d, F, box); if (r) return r; c->box_down = box; }
+    c->pl_gu = plan_gemm(EPI_SWIGLU, T_rows, F, d, c->num_sms, 0);
+    box = c->pl_gu.tile_n / 2;
+    if (box != c->box_gu) {
+      l2pd_status r = encode_weight_maps(c, c->tb_gate, c->w_gate, F, d, box); if (r) return r;
+      r = encode_weight_maps(c, c->tb_up, c->w_up, F, d, box); if (r) return r;
+      c->box_gu = box;
     }
   }
 
@@ -207,7 +215,7 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     T *kc = (T *)c->kc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
     T *vc = (T *)c->vc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
     l2pd_status r;
-    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_QKV, EPI_STORE, &c->ta_n, &c->tb_qkv[l], nullptr, qkv, T_rows, 3 * hd, d, c->tn_qkv);
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_QKV, EPI_STORE, &c->ta_n, &c->tb_qkv[l], nullptr, qkv, T_rows, 3 * hd, d, c->pl_qkv);
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_QKV, EPI_STORE, n, c->wqkv[l], nullptr, qkv, nullptr, T_rows, 3 * hd, d);
     if (r) return r;
     CKLK(L2PD_K_ROPE, launch_rope_scatter<T>(s, qkv, c->d_meta, c->d_row_slot, c->cs_table, q, kc, vc, c->kv_seq_stride, T_rows, H, dh));
@@ -217,14 +225,14 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     } else {
       CKLK(L2PD_K_ATTENTION, launch_simt_attention<T>(s, q, kc, vc, c->d_meta, c->d_row_slot, att, c->kv_seq_stride, T_rows, H, dh, max_kv));
     }
-    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_O, EPI_RESIDUAL, &c->ta_att, &c->tb_o[l], nullptr, c->x, T_rows, d, hd, c->tn_o);
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_O, EPI_RESIDUAL, &c->ta_att, &c->tb_o[l], nullptr, c->x, T_rows, d, hd, c->pl_o);
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_O, EPI_RESIDUAL, att, c->wo[l], nullptr, c->x, nullptr, T_rows, d, hd);
     if (r) return r;
     CKLK(L2PD_K_RMSNORM, launch_rmsnorm<T>(s, c->x, c->norm2[l], f.rms_eps, n, T_rows, d));
-    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_GATE_UP, EPI_SWIGLU, &c->ta_n, &c->tb_gate[l], &c->tb_up[l], hbuf, T_rows, F, d, c->tn_gu);
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_GATE_UP, EPI_SWIGLU, &c->ta_n, &c->tb_gate[l], &c->tb_up[l], hbuf, T_rows, F, d, c->pl_gu);
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_GATE_UP, EPI_SWIGLU, n, c->w_gate[l], c->w_up[l], hbuf, nullptr, T_rows, F, d);
     if (r) return r;
-    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_DOWN, EPI_RESIDUAL, &c->ta_h, &c->tb_down[l], nullptr, c->x, T_rows, d, F, c->tn_down);
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_DOWN, EPI_RESIDUAL, &c->ta_h, &c->tb_down[l], nullptr, c->x, T_rows, d, F, c->pl_down);
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_DOWN, EPI_RESIDUAL, hbuf, c->w_down[l], nullptr, c->x, nullptr, T_rows, d, F);
     if (r) return r;
     if (c->cap)
@@ -609,21 +617,31 @@ static l2pd_status gemm_common(void *stream, int epi, const void *A, const void 
                                int M, int N, int K, int tile_n, int check) {
   if (!A || !W || !out || (epi == EPI_SWIGLU && !W2)) return L2PD_ERR_ARG;
   if (M < 1 || N < 8 || K < 8 || (N % 8) || (K % 8)) return L2PD_ERR_SHAPE;
+  if (tile_n < 0) return L2PD_ERR_SHAPE;
   const int sms = device_sms();
-  const int unit = epi == EPI_SWIGLU ? 2 : 1;
-  if (tile_n == 0) tile_n = unit * pick_tile_n(M, N, sms, 16, 256 / unit);
-  if (tile_n < 32 || tile_n > 256 || (tile_n % (16 * unit))) return L2PD_ERR_SHAPE;
+  // tile_n = width + 1000 * cta_group + 10000 * k_splits; any part 0 = chosen automatically
+  const int want_ks = tile_n / 10000, want_cg = (tile_n % 10000) / 1000, want_tn = tile_n % 1000;
+  const int unit = epi == EPI_SWIGLU ? 32 : 16;
+  if (want_tn && (want_tn < 32 || want_tn > 256 || (want_tn % unit))) return L2PD_ERR_SHAPE;
+  if (want_cg > 2 || want_ks > 8 || (want_ks > 1 && epi != EPI_RESIDUAL)) return L2PD_ERR_SHAPE;
+  GemmPlan pl = plan_gemm(epi, M, N, K, sms, want_tn);
+  if (want_tn) pl.tile_n = want_tn;
+  if (want_cg) pl.cta_group = want_cg;
+  if (want_ks) pl.k_splits = want_ks;
+  if (pl.k_splits > ceil_div(K, 64)) pl.k_splits = ceil_div(K, 64);
   int32_t *status = standalone_status();
   if (!status) return L2PD_ERR_CUDA;
+  const int box = epi == EPI_SWIGLU ? pl.tile_n / 2 : pl.tile_n / pl.cta_group;
   TmaDesc ta, tb, tb2;
   l2pd_status r = make_tma_2d_bf16(&ta, A, M, K, 128);
   if (r) return r;
-  r = make_tma_2d_bf16(&tb, W, N, K, tile_n / unit);
+  r = make_tma_2d_bf16(&tb, W, N, K, box);
   if (r) return r;
-  if (epi == EPI_SWIGLU) { r = make_tma_2d_bf16(&tb2, W2, N, K, tile_n / unit); if (r) return r; }
+  if (epi == EPI_SWIGLU) { r = make_tma_2d_bf16(&tb2, W2, N, K, box); if (r) return r; }
   GemmArgs g{};
   g.epi = epi; g.a = &ta; g.b = &tb; g.b2 = epi == EPI_SWIGLU ? &tb2 : nullptr;
-  g.M = M; g.N = N; g.K = K; g.tile_n = tile_n; g.out = out; g.status = status;
+  g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.cta_group = pl.cta_group; g.k_splits = pl.k_splits;
+  g.out = out; g.status = status;
   if (launch_gemm_tcgen05((cudaStream_t)stream, g, sms) != cudaSuccess) return L2PD_ERR_CUDA;
   return finish_standalone((cudaStream_t)stream, status, check);
 }

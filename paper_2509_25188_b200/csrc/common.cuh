@@ -71,7 +71,7 @@ cudaError_t launch_gather_response(cudaStream_t st, const int32_t *tokens, int B
                                    int32_t *out);
 
 // simt.cu : CUDA-core GEMM and attention (fp32 configurations; also a bf16 cross-check path)
-enum { EPI_STORE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_STORE_F32 = 3 };
+enum { EPI_STORE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_STORE_F32 = 3, EPI_LMHEAD = 4 };
 template <typename T>
 cudaError_t launch_simt_gemm(cudaStream_t st, int epi, const T *A, const T *W, const T *W2, void *C,
                              const float *bias, int M, int N, int K);
@@ -105,16 +105,21 @@ struct TmaDesc { CUtensorMap map; };
 // Encodes a 2-D bf16 row-major tensor [rows, cols] with a box of [box_rows, 64] and 128-byte swizzle.
 l2pd_status make_tma_2d_bf16(TmaDesc *out, const void *ptr, int64_t rows, int64_t cols, int box_rows);
 int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile);
+// How one GEMM is laid over the SMs: CTAs per tile (1, or 2 = a cta_group::2 pair on a 256-row tile),
+// tile width, and K slices (residual epilogue only: slices add into X with vector reductions).
+// The B tensor map's box must be tile_n / cta_group rows (SwiGLU: tile_n / 2 for either group size).
+struct GemmPlan { int cta_group, tile_n, k_splits; };
+GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n);
 struct GemmArgs {
   int epi;                 // EPI_STORE, EPI_RESIDUAL, EPI_SWIGLU, or EPI_LMHEAD
   const TmaDesc *a, *b, *b2;
   int M, N, K, tile_n;
+  int cta_group, k_splits; // 0 / 1 = single CTA, no split
   void *out;               // bf16 C, fp32 X, or bf16 H
   // LM head
   const float *bias; float *part_m, *part_s; int32_t *part_i; int rows_padded; float *logits;
   int32_t *status;         // device status word
 };
-enum { EPI_LMHEAD = 4 };
 cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms);
 cudaError_t launch_merge_partials(cudaStream_t st, const float *part_m, const float *part_s,
                                   const int32_t *part_i, int n_tiles, int rows_padded, int R,

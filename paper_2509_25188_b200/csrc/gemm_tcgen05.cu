@@ -34,7 +34,7 @@ constexpr int SMEM_BUDGET = 227 * 1024;
 
 struct KParams {
   int M, N, K, tile_n, n_stages, b_stage_bytes;
-  int m_tiles, n_tiles;
+  int m_tiles, n_tiles, k_splits;   // m_tiles counts 128-row tiles (CG = 1) or 256-row pair tiles (CG = 2)
   void *out;
   const float *bias;
   float *part_m, *part_s;
@@ -48,16 +48,159 @@ __device__ __forceinline__ void fail(int32_t *status, int code) {
   if (status) atomicCAS(status, 0, code);
 }
 
+// Drains one 128-row x tile_n accumulator from tensor memory (this warp's 32 lanes) and applies the
+// epilogue.  `atomic` (split-K residual): the partial sum is added to X with a vector reduction.
 template <int EPI>
-__global__ void __launch_bounds__(192, 1)
-gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const __grid_constant__ CUtensorMap tmB2, const KParams p) {
-  extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
-  __shared__ uint32_t tmem_slot;
-  __shared__ int abort_flag;
+__device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int row, int nt, bool atomic) {
+  const bool row_ok = row < p.M;
+  const int half_n = p.tile_n >> 1;
+  uint32_t v[16];
+  if (EPI == EPI_STORE) {
+    bf16 *C = reinterpret_cast<bf16 *>(p.out);
+    const int n0 = nt * p.tile_n;
+    for (int c = 0; c < p.tile_n; c += 16) {
+      ptx::tmem_ld_x16(taddr + c, v);
+      ptx::tmem_ld_wait();
+      if (row_ok) {
+#pragma unroll
+        for (int hseg = 0; hseg < 2; ++hseg) {
+          const int col = n0 + c + hseg * 8;
+          if (col < p.N) {
+            uint4 pk;
+            uint32_t *pw = reinterpret_cast<uint32_t *>(&pk);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(v[hseg * 8 + 2 * i]),
+                                                       __uint_as_float(v[hseg * 8 + 2 * i + 1]));
+              pw[i] = *reinterpret_cast<uint32_t *>(&t);
+            }
+            *reinterpret_cast<uint4 *>(C + (int64_t)row * p.N + col) = pk;
+          }
+        }
+      }
+    }
+  } else if (EPI == EPI_RESIDUAL) {
+    float *X = reinterpret_cast<float *>(p.out);
+    const int n0 = nt * p.tile_n;
+    for (int c = 0; c < p.tile_n; c += 16) {
+      ptx::tmem_ld_x16(taddr + c, v);
+      ptx::tmem_ld_wait();
+      if (row_ok) {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          const int col = n0 + c + g * 4;
+          if (col < p.N) {
+            float *px = X + (int64_t)row * p.N + col;
+            if (atomic) {
+              ptx::red_add_v4(px, __uint_as_float(v[4 * g + 0]), __uint_as_float(v[4 * g + 1]),
+                              __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3]));
+            } else {
+              float4 x = *reinterpret_cast<float4 *>(px);
+              x.x += __uint_as_float(v[4 * g + 0]);
+              x.y += __uint_as_float(v[4 * g + 1]);
+              x.z += __uint_as_float(v[4 * g + 2]);
+              x.w += __uint_as_float(v[4 * g + 3]);
+              *reinterpret_cast<float4 *>(px) = x;
+            }
+          }
+        }
+      }
+    }
+  } else if (EPI == EPI_SWIGLU) {
+    bf16 *H = reinterpret_cast<bf16 *>(p.out);
+    const int n0 = nt * half_n;
+    uint32_t u[16];
+    for (int c = 0; c < half_n; c += 16) {
+      ptx::tmem_ld_x16(taddr + c, v);
+      ptx::tmem_ld_x16(taddr + half_n + c, u);
+      ptx::tmem_ld_wait();
+      if (row_ok) {
+#pragma unroll
+        for (int hseg = 0; hseg < 2; ++hseg) {
+          const int col = n0 + c + hseg * 8;
+          if (col < p.N) {
+            uint4 pk;
+            uint32_t *pw = reinterpret_cast<uint32_t *>(&pk);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              float g0 = __uint_as_float(v[hseg * 8 + 2 * i]), g1 = __uint_as_float(v[hseg * 8 + 2 * i + 1]);
+              float u0 = __uint_as_float(u[hseg * 8 + 2 * i]), u1 = __uint_as_float(u[hseg * 8 + 2 * i + 1]);
+              float h0 = g0 / (1.0f + __expf(-g0)) * u0;
+              float h1 = g1 / (1.0f + __expf(-g1)) * u1;
+              __nv_bfloat162 t = __floats2bfloat162_rn(h0, h1);
+              pw[i] = *reinterpret_cast<uint32_t *>(&t);
+            }
+            *reinterpret_cast<uint4 *>(H + (int64_t)row * p.N + col) = pk;
+          }
+        }
+      }
+    }
+  } else {  // EPI_LMHEAD
+    const float L2E = 1.4426950408889634f;
+    const int n0 = nt * p.tile_n;
+    float m_run = -INFINITY, s_run = 0.f;
+    int i_run = 0x7fffffff;
+    for (int c = 0; c < p.tile_n; c += 16) {
+      ptx::tmem_ld_x16(taddr + c, v);
+      ptx::tmem_ld_wait();
+      if (row_ok && n0 + c < p.N) {
+        float f[16];
+        float cm = -INFINITY;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const int col = n0 + c + i;
+          float val = __uint_as_float(v[i]);
+          if (col < p.N) { if (p.bias) val += __ldg(p.bias + col); }
+          else val = -INFINITY;
+          f[i] = val;
+          cm = fmaxf(cm, val);
+        }
+        if (p.logits) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            if (n0 + c + i < p.N) p.logits[(int64_t)row * p.N + n0 + c + i] = f[i];
+        }
+        if (cm > m_run) {
+          s_run *= exp2f((m_run - cm) * L2E);
+          m_run = cm;
+          int ci = 0;
+#pragma unroll
+          for (int i = 15; i >= 0; --i) if (f[i] == cm) ci = i;   // lowest index holding the max
+          i_run = n0 + c + ci;
+        }
+        float add = 0.f;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) add += exp2f((f[i] - m_run) * L2E);
+        s_run += add;
+      }
+    }
+    if (row_ok) {
+      const int64_t o = (int64_t)nt * p.rows_padded + row;
+      p.part_m[o] = m_run;
+      p.part_s[o] = s_run;
+      p.part_i[o] = i_run;
+    }
+  }
+}
 
+// CG = 1: one CTA per 128 x tile_n output tile.
+// CG = 2: a cluster of two CTAs per 256 x tile_n tile (cta_group::2).  CTA r loads A rows
+//         [128 r, 128 r + 128) and the r-th half of the B tile (for SwiGLU: CTA 0 the gate rows,
+//         CTA 1 the up rows), so each SM takes in half of the weight tile; the leader CTA (rank 0)
+//         issues the MMAs, which read both CTAs' shared memory and write both CTAs' tensor memory.
+//         All load-completion bytes are counted on the leader's `full` barriers; `empty` and
+//         `tmem full` are signalled in both CTAs by a multicast commit; the peer's epilogue warps
+//         release the accumulator on the leader's `tmem empty` barrier.
+template <int EPI, int CG>
+__device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensorMap *tmB, const CUtensorMap *tmB2,
+                                          const KParams &p, uint8_t *smem_raw, uint64_t *bars, uint32_t *tmem_slot,
+                                          int *abort_flag) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;
+  const bool leader = rank == 0;
+  const int group = (CG == 2) ? (blockIdx.x >> 1) : blockIdx.x;
+  const int n_groups = (CG == 2) ? (gridDim.x >> 1) : gridDim.x;
+
   const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sA = base;
   const uint32_t sB = base + p.n_stages * A_STAGE_BYTES;
@@ -69,244 +212,182 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.n_stages; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { ptx::mbar_init(tfull_bar(b), 1); ptx::mbar_init(tempty_bar(b), 4); }
-    abort_flag = 0;
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(tfull_bar(b), 1); ptx::mbar_init(tempty_bar(b), 4 * CG); }
+    *abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
   }
   if (warp == 0 && lane == 0) {
-    ptx::prefetch_tensormap(&tmA);
-    ptx::prefetch_tensormap(&tmB);
-    if (EPI == EPI_SWIGLU) ptx::prefetch_tensormap(&tmB2);
+    ptx::prefetch_tensormap(tmA);
+    ptx::prefetch_tensormap(tmB);
+    if (EPI == EPI_SWIGLU) ptx::prefetch_tensormap(tmB2);
   }
   if (warp == 1) {
-    ptx::tmem_alloc(ptx::smem_u32(&tmem_slot), TMEM_COLS);
-    ptx::tmem_relinquish();
+    if (CG == 2) { ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), TMEM_COLS); ptx::tmem_relinquish_pair(); }
+    else { ptx::tmem_alloc(ptx::smem_u32(tmem_slot), TMEM_COLS); ptx::tmem_relinquish(); }
   }
   ptx::tc_fence_before_sync();
   __syncthreads();
+  if (CG == 2) ptx::cluster_sync();     // the peer's barriers exist before anything arrives on them
   ptx::tc_fence_after_sync();
-  const uint32_t tmem_base = tmem_slot;
+  const uint32_t tmem_base = *tmem_slot;
 
-  const int num_tiles = p.m_tiles * p.n_tiles;
+  const int num_units = p.m_tiles * p.n_tiles * p.k_splits;
   const int num_kb = (p.K + TILE_K - 1) / TILE_K;
+  const int kb_per = (num_kb + p.k_splits - 1) / p.k_splits;
   const int half_n = p.tile_n >> 1;
+  // unit -> (row tile, column tile, K slice); row tiles of one column tile are adjacent so that the
+  // CTAs running at the same time share the weight tile in L2
+  auto decode = [&](int u, int &mt, int &nt, int &kb0, int &kb1) {
+    mt = u % p.m_tiles;
+    const int r = u / p.m_tiles;
+    nt = r % p.n_tiles;
+    const int ks = r / p.n_tiles;
+    kb0 = ks * kb_per;
+    kb1 = min(num_kb, kb0 + kb_per);
+  };
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       const uint64_t pol_w = ptx::policy_evict_first();   // weights are read once per step
-      const uint64_t pol_a = ptx::policy_evict_last();    // activations are re-read by every N tile
-      const uint32_t tx = A_STAGE_BYTES + (uint32_t)p.tile_n * 128u;
+      const uint64_t pol_a = ptx::policy_evict_last();    // activations are re-read by every column tile
+      const uint32_t b_bytes = (CG == 2) ? (uint32_t)half_n * 128u : (uint32_t)p.tile_n * 128u;
+      const uint32_t tx = CG * (A_STAGE_BYTES + b_bytes);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
-        const int m0 = mt * TILE_M;
-        for (int kb = 0; kb < num_kb; ++kb) {
+      for (int u = group; u < num_units && ok; u += n_groups) {
+        int mt, nt, kb0, kb1;
+        decode(u, mt, nt, kb0, kb1);
+        const int m0 = mt * (TILE_M * CG) + (int)rank * TILE_M;
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
-          ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
-          ptx::tma_load_2d_hint(sA + stage * A_STAGE_BYTES, &tmA, full_bar(stage), kb * TILE_K, m0, pol_a);
-          const uint32_t dstB = sB + stage * p.b_stage_bytes;
-          if (EPI == EPI_SWIGLU) {
-            ptx::tma_load_2d_hint(dstB, &tmB, full_bar(stage), kb * TILE_K, nt * half_n, pol_w);
-            ptx::tma_load_2d_hint(dstB + half_n * 128, &tmB2, full_bar(stage), kb * TILE_K, nt * half_n, pol_w);
+          const uint32_t dstA = sA + stage * A_STAGE_BYTES, dstB = sB + stage * p.b_stage_bytes;
+          if (CG == 1) {
+            ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
+            ptx::tma_load_2d_hint(dstA, tmA, full_bar(stage), kb * TILE_K, m0, pol_a);
+            if (EPI == EPI_SWIGLU) {
+              ptx::tma_load_2d_hint(dstB, tmB, full_bar(stage), kb * TILE_K, nt * half_n, pol_w);
+              ptx::tma_load_2d_hint(dstB + half_n * 128, tmB2, full_bar(stage), kb * TILE_K, nt * half_n, pol_w);
+            } else {
+              ptx::tma_load_2d_hint(dstB, tmB, full_bar(stage), kb * TILE_K, nt * p.tile_n, pol_w);
+            }
           } else {
-            ptx::tma_load_2d_hint(dstB, &tmB, full_bar(stage), kb * TILE_K, nt * p.tile_n, pol_w);
+            if (leader) ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
+            const uint32_t lead_full = ptx::mapa(full_bar(stage), 0);
+            ptx::tma_load_2d_pair_hint(dstA, tmA, lead_full, kb * TILE_K, m0, pol_a);
+            if (EPI == EPI_SWIGLU)
+              ptx::tma_load_2d_pair_hint(dstB, leader ? tmB : tmB2, lead_full, kb * TILE_K, nt * half_n, pol_w);
+            else
+              ptx::tma_load_2d_pair_hint(dstB, tmB, lead_full, kb * TILE_K, nt * p.tile_n + (int)rank * half_n, pol_w);
           }
           if (++stage == p.n_stages) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) abort_flag = 1;
+      if (!ok) *abort_flag = 1;
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      const uint32_t idesc = ptx::idesc_bf16_m128((uint32_t)p.tile_n);
+    // ------------------------------------------------------------------ MMA issuer (leader CTA only when paired)
+    if (lane == 0 && leader) {
+      const uint32_t idesc = ptx::idesc_bf16(TILE_M * CG, (uint32_t)p.tile_n);
       int stage = 0;
       uint32_t phase = 0;
       int lt = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
+      for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
+        int mt, nt, kb0, kb1;
+        decode(u, mt, nt, kb0, kb1);
         const int ab = lt & 1;
         const uint32_t aphase = (lt >> 1) & 1;
         if (!ptx::mbar_wait(tempty_bar(ab), aphase ^ 1u)) { fail(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + ab * ACC_COLS;
-        for (int kb = 0; kb < num_kb; ++kb) {
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!ptx::mbar_wait(full_bar(stage), phase)) { fail(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
           ptx::tc_fence_after_sync();
           const uint64_t a_desc = ptx::smem_desc_sw128(sA + stage * A_STAGE_BYTES);
           const uint64_t b_desc = ptx::smem_desc_sw128(sB + stage * p.b_stage_bytes);
 #pragma unroll
-          for (int k = 0; k < TILE_K / 16; ++k)   // 16 bf16 = 32 bytes per MMA: descriptor address += 2
-            ptx::mma_bf16_ss(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
-          ptx::mma_commit(empty_bar(stage));
+          for (int k = 0; k < TILE_K / 16; ++k) {   // 16 bf16 = 32 bytes per MMA: descriptor address += 2
+            const uint32_t acc = (kb > kb0 || k > 0) ? 1u : 0u;
+            if (CG == 2) ptx::mma_bf16_ss_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, acc);
+            else ptx::mma_bf16_ss(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, acc);
+          }
+          if (CG == 2) ptx::mma_commit_pair(empty_bar(stage), 3);
+          else ptx::mma_commit(empty_bar(stage));
           if (++stage == p.n_stages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) ptx::mma_commit(tfull_bar(ab));
+        if (ok) {
+          if (CG == 2) ptx::mma_commit_pair(tfull_bar(ab), 3);
+          else ptx::mma_commit(tfull_bar(ab));
+        }
       }
-      if (!ok) abort_flag = 1;
+      if (!ok) *abort_flag = 1;
     }
   } else {
     // ------------------------------------------------------------------ epilogue
     const int q = warp & 3;
     int lt = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++lt) {
-      const int mt = tile % p.m_tiles, nt = tile / p.m_tiles;
+    for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
+      int mt, nt, kb0, kb1;
+      decode(u, mt, nt, kb0, kb1);
       const int ab = lt & 1;
       const uint32_t aphase = (lt >> 1) & 1;
       if (!ptx::mbar_wait(tfull_bar(ab), aphase)) { fail(p.status, DEV_TIMEOUT_EPILOGUE); ok = false; break; }
       ptx::tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ab * ACC_COLS;
-      const int row = mt * TILE_M + q * 32 + lane;
-      const bool row_ok = row < p.M;
-      uint32_t v[16];
-
-      if (EPI == EPI_STORE) {
-        bf16 *C = reinterpret_cast<bf16 *>(p.out);
-        const int n0 = nt * p.tile_n;
-        for (int c = 0; c < p.tile_n; c += 16) {
-          ptx::tmem_ld_x16(taddr + c, v);
-          ptx::tmem_ld_wait();
-          if (row_ok) {
-#pragma unroll
-            for (int hseg = 0; hseg < 2; ++hseg) {
-              const int col = n0 + c + hseg * 8;
-              if (col < p.N) {
-                uint4 pk;
-                uint32_t *pw = reinterpret_cast<uint32_t *>(&pk);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(v[hseg * 8 + 2 * i]),
-                                                           __uint_as_float(v[hseg * 8 + 2 * i + 1]));
-                  pw[i] = *reinterpret_cast<uint32_t *>(&t);
-                }
-                *reinterpret_cast<uint4 *>(C + (int64_t)row * p.N + col) = pk;
-              }
-            }
-          }
-        }
-      } else if (EPI == EPI_RESIDUAL) {
-        float *X = reinterpret_cast<float *>(p.out);
-        const int n0 = nt * p.tile_n;
-        for (int c = 0; c < p.tile_n; c += 16) {
-          ptx::tmem_ld_x16(taddr + c, v);
-          ptx::tmem_ld_wait();
-          if (row_ok) {
-#pragma unroll
-            for (int g = 0; g < 4; ++g) {
-              const int col = n0 + c + g * 4;
-              if (col < p.N) {
-                float4 *px = reinterpret_cast<float4 *>(X + (int64_t)row * p.N + col);
-                float4 x = *px;
-                x.x += __uint_as_float(v[4 * g + 0]);
-                x.y += __uint_as_float(v[4 * g + 1]);
-                x.z += __uint_as_float(v[4 * g + 2]);
-                x.w += __uint_as_float(v[4 * g + 3]);
-                *px = x;
-              }
-            }
-          }
-        }
-      } else if (EPI == EPI_SWIGLU) {
-        bf16 *H = reinterpret_cast<bf16 *>(p.out);
-        const int n0 = nt * half_n;
-        uint32_t u[16];
-        for (int c = 0; c < half_n; c += 16) {
-          ptx::tmem_ld_x16(taddr + c, v);
-          ptx::tmem_ld_x16(taddr + half_n + c, u);
-          ptx::tmem_ld_wait();
-          if (row_ok) {
-#pragma unroll
-            for (int hseg = 0; hseg < 2; ++hseg) {
-              const int col = n0 + c + hseg * 8;
-              if (col < p.N) {
-                uint4 pk;
-                uint32_t *pw = reinterpret_cast<uint32_t *>(&pk);
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  float g0 = __uint_as_float(v[hseg * 8 + 2 * i]), g1 = __uint_as_float(v[hseg * 8 + 2 * i + 1]);
-                  float u0 = __uint_as_float(u[hseg * 8 + 2 * i]), u1 = __uint_as_float(u[hseg * 8 + 2 * i + 1]);
-                  float h0 = g0 / (1.0f + __expf(-g0)) * u0;
-                  float h1 = g1 / (1.0f + __expf(-g1)) * u1;
-                  __nv_bfloat162 t = __floats2bfloat162_rn(h0, h1);
-                  pw[i] = *reinterpret_cast<uint32_t *>(&t);
-                }
-                *reinterpret_cast<uint4 *>(H + (int64_t)row * p.N + col) = pk;
-              }
-            }
-          }
-        }
-      } else {  // EPI_LMHEAD
-        const float L2E = 1.4426950408889634f;
-        const int n0 = nt * p.tile_n;
-        float m_run = -INFINITY, s_run = 0.f;
-        int i_run = 0x7fffffff;
-        for (int c = 0; c < p.tile_n; c += 16) {
-          ptx::tmem_ld_x16(taddr + c, v);
-          ptx::tmem_ld_wait();
-          if (row_ok && n0 + c < p.N) {
-            float f[16];
-            float cm = -INFINITY;
-#pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const int col = n0 + c + i;
-              float val = __uint_as_float(v[i]);
-              if (col < p.N) { if (p.bias) val += __ldg(p.bias + col); }
-              else val = -INFINITY;
-              f[i] = val;
-              cm = fmaxf(cm, val);
-            }
-            if (p.logits) {
-#pragma unroll
-              for (int i = 0; i < 16; ++i)
-                if (n0 + c + i < p.N) p.logits[(int64_t)row * p.N + n0 + c + i] = f[i];
-            }
-            if (cm > m_run) {
-              s_run *= exp2f((m_run - cm) * L2E);
-              m_run = cm;
-              int ci = 0;
-#pragma unroll
-              for (int i = 15; i >= 0; --i) if (f[i] == cm) ci = i;   // lowest index holding the max
-              i_run = n0 + c + ci;
-            }
-            float add = 0.f;
-#pragma unroll
-            for (int i = 0; i < 16; ++i) add += exp2f((f[i] - m_run) * L2E);
-            s_run += add;
-          }
-        }
-        if (row_ok) {
-          const int64_t o = (int64_t)nt * p.rows_padded + row;
-          p.part_m[o] = m_run;
-          p.part_s[o] = s_run;
-          p.part_i[o] = i_run;
-        }
-      }
+      const int row = mt * (TILE_M * CG) + (int)rank * TILE_M + q * 32 + lane;
+      drain_tile<EPI>(p, taddr, row, nt, p.k_splits > 1);
       ptx::tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(tempty_bar(ab));
+      if (lane == 0) {
+        if (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(tempty_bar(ab), 0));
+        else ptx::mbar_arrive(tempty_bar(ab));
+      }
     }
-    if (!ok) abort_flag = 1;
+    if (!ok) *abort_flag = 1;
   }
 
   // ---------------------------------------------------------------------- teardown
   __syncwarp();
   ptx::tc_fence_before_sync();
   __syncthreads();
-  if (abort_flag) {
+  if (*abort_flag) {
     // A wait ran out: give copies still in flight time to land before the CTA's shared memory goes away.
     const uint64_t t0 = ptx::globaltimer();
     while (ptx::globaltimer() - t0 < 200000ull) __nanosleep(1000);
     __syncthreads();
   }
+  if (CG == 2) ptx::cluster_sync();     // neither CTA leaves while the other may still touch its memory
   if (warp == 1) {
     ptx::tc_fence_after_sync();
-    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+    if (CG == 2) ptx::tmem_dealloc_pair(tmem_base, TMEM_COLS);
+    else ptx::tmem_dealloc(tmem_base, TMEM_COLS);
   }
+}
+
+template <int EPI>
+__global__ void __launch_bounds__(192, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const __grid_constant__ CUtensorMap tmB2, const KParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  gemm_body<EPI, 1>(&tmA, &tmB, &tmB2, p, smem_raw, bars, &tmem_slot, &abort_flag);
+}
+
+template <int EPI>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1)
+gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                         const __grid_constant__ CUtensorMap tmB2, const KParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
+  __shared__ uint32_t tmem_slot;
+  __shared__ int abort_flag;
+  gemm_body<EPI, 2>(&tmA, &tmB, &tmB2, p, smem_raw, bars, &tmem_slot, &abort_flag);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -368,52 +449,96 @@ l2pd_status make_tma_2d_bf16(TmaDesc *out, const void *ptr, int64_t rows, int64_
   return r == CUDA_SUCCESS ? L2PD_OK : L2PD_ERR_CUDA;
 }
 
-// Tile width that minimises (waves x per-tile cost) for m_tiles row tiles over num_sms persistent
-// CTAs.  `unit` is the granularity of the returned width, `max_tile` its largest value.
-int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile) {
-  const int m_tiles = ceil_div(M, TILE_M);
-  int best = max_tile;
-  double best_cost = 1e30;
-  for (int tn = max_tile; tn >= 64 && tn >= multiple; tn -= multiple) {
-    const int tiles = m_tiles * ceil_div(N, tn);
-    const int waves = ceil_div(tiles, num_sms);
-    const double cost = (double)waves * (tn + 12);   // per-tile main loop ~ tn, plus a fixed part
-    if (cost < best_cost - 1e-9) { best_cost = cost; best = tn; }
+// Modelled cycles of one GEMM for a tile width / K split: per 64-deep k-block a CTA needs
+// max(2 * tile_n MMA cycles, bytes it must take in / ~70 B per cycle), plus a fixed fill/drain part
+// per unit, times the number of waves over the SMs (or SM pairs).
+static double plan_cost(int M, int N, int K, int num_sms, int cg, int unit_n, int tile_n, int ks) {
+  const int groups = num_sms / cg;
+  const int m_tiles = ceil_div(M, TILE_M * cg);
+  const int n_tiles = ceil_div(N, unit_n);
+  const int units = m_tiles * n_tiles * ks;
+  const int waves = ceil_div(units, groups);
+  const int kb = ceil_div(ceil_div(K, TILE_K), ks);
+  const double bytes = A_STAGE_BYTES + 128.0 * tile_n / cg;
+  const double per_kb = fmax(2.0 * tile_n, bytes / 70.0);
+  return waves * (kb * per_kb + 1500.0 + 4.0 * tile_n + (ks > 1 ? 2.0 * tile_n : 0.0));
+}
+
+GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n) {
+  GemmPlan best{1, 256, 1};
+  double best_cost = 1e300;
+  const bool swiglu = epi == EPI_SWIGLU;
+  const int step = swiglu ? 32 : 16;
+  for (int cg = 1; cg <= 2; ++cg) {
+    if (cg == 2 && (M <= TILE_M || epi == EPI_LMHEAD || num_sms < 2)) continue;
+    for (int tn = 256; tn >= 64; tn -= step) {
+      if (force_tile_n && tn != force_tile_n) continue;
+      const int unit_n = swiglu ? tn / 2 : tn;
+      const int max_ks = (epi == EPI_RESIDUAL) ? 4 : 1;
+      for (int ks = 1; ks <= max_ks; ++ks) {
+        if (ceil_div(K, TILE_K) < 8 * ks) break;
+        const double c = plan_cost(M, N, K, num_sms, cg, unit_n, tn, ks);
+        if (c < best_cost - 1e-9) { best_cost = c; best = GemmPlan{cg, tn, ks}; }
+      }
+    }
   }
+  if (force_tile_n && best_cost > 1e299) best.tile_n = force_tile_n;
   return best;
 }
 
+int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile) {
+  (void)multiple; (void)max_tile;
+  return plan_gemm(EPI_LMHEAD, M, N, 4096, num_sms, 0).tile_n;
+}
+
 cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms) {
+  const int cg = g.cta_group == 2 ? 2 : 1;
+  int ks = g.k_splits > 1 ? g.k_splits : 1;
+  if (ks > 1 && g.epi != EPI_RESIDUAL) return cudaErrorInvalidValue;
+  {   // every K slice must hold at least one k-block (an empty slice would add an unwritten accumulator)
+    const int num_kb = ceil_div(g.K, TILE_K);
+    while (ks > 1 && ceil_div(num_kb, ks) * (ks - 1) >= num_kb) --ks;
+  }
   KParams p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.tile_n = g.tile_n;
-  p.b_stage_bytes = g.tile_n * 128;
+  p.b_stage_bytes = g.tile_n * 128 / cg;
   const int stage_bytes = A_STAGE_BYTES + p.b_stage_bytes;
   int stages = (SMEM_BUDGET - 2048) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) return cudaErrorInvalidValue;
   p.n_stages = stages;
-  p.m_tiles = ceil_div(g.M, TILE_M);
+  p.m_tiles = ceil_div(g.M, TILE_M * cg);
   const int n_per_tile = (g.epi == EPI_SWIGLU) ? g.tile_n / 2 : g.tile_n;
   p.n_tiles = ceil_div(g.N, n_per_tile);
+  p.k_splits = ks;
   p.out = g.out; p.bias = g.bias; p.part_m = g.part_m; p.part_s = g.part_s; p.part_i = g.part_i;
   p.rows_padded = g.rows_padded; p.logits = g.logits; p.status = g.status;
-  const int tiles = p.m_tiles * p.n_tiles;
-  if (tiles <= 0) return cudaSuccess;
-  const int grid = tiles < num_sms ? tiles : num_sms;
+  const int units = p.m_tiles * p.n_tiles * ks;
+  if (units <= 0) return cudaSuccess;
+  const int groups = num_sms / cg;
+  const int grid = cg * (units < groups ? units : groups);
   const size_t smem = (size_t)stages * stage_bytes + 1024;
   const CUtensorMap &b2 = g.b2 ? g.b2->map : g.b->map;
   cudaError_t e;
-#define L2PD_LAUNCH(EPI)                                                                              \
-  e = cudaFuncSetAttribute(gemm_tcgen05_kernel<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize,    \
-                           SMEM_BUDGET - 1024);                                                      \
+#define L2PD_LAUNCH(KERNEL, EPI)                                                                      \
+  e = cudaFuncSetAttribute(KERNEL<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET - 1024); \
   if (e != cudaSuccess) return e;                                                                    \
-  gemm_tcgen05_kernel<EPI><<<grid, 192, smem, st>>>(g.a->map, g.b->map, b2, p);
-  switch (g.epi) {
-    case EPI_STORE: L2PD_LAUNCH(EPI_STORE) break;
-    case EPI_RESIDUAL: L2PD_LAUNCH(EPI_RESIDUAL) break;
-    case EPI_SWIGLU: L2PD_LAUNCH(EPI_SWIGLU) break;
-    case EPI_LMHEAD: L2PD_LAUNCH(EPI_LMHEAD) break;
-    default: return cudaErrorInvalidValue;
+  KERNEL<EPI><<<grid, 192, smem, st>>>(g.a->map, g.b->map, b2, p);
+  if (cg == 1) {
+    switch (g.epi) {
+      case EPI_STORE: L2PD_LAUNCH(gemm_tcgen05_kernel, EPI_STORE) break;
+      case EPI_RESIDUAL: L2PD_LAUNCH(gemm_tcgen05_kernel, EPI_RESIDUAL) break;
+      case EPI_SWIGLU: L2PD_LAUNCH(gemm_tcgen05_kernel, EPI_SWIGLU) break;
+      case EPI_LMHEAD: L2PD_LAUNCH(gemm_tcgen05_kernel, EPI_LMHEAD) break;
+      default: return cudaErrorInvalidValue;
+    }
+  } else {
+    switch (g.epi) {
+      case EPI_STORE: L2PD_LAUNCH(gemm_tcgen05_pair_kernel, EPI_STORE) break;
+      case EPI_RESIDUAL: L2PD_LAUNCH(gemm_tcgen05_pair_kernel, EPI_RESIDUAL) break;
+      case EPI_SWIGLU: L2PD_LAUNCH(gemm_tcgen05_pair_kernel, EPI_SWIGLU) break;
+      default: return cudaErrorInvalidValue;
+    }
   }
 #undef L2PD_LAUNCH
   return cudaGetLastError();

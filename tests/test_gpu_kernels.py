@@ -44,6 +44,11 @@ GEMM_SHAPES = [
     (300, 528, 1032, 176),  # odd tile width (multiple of 16), K tail
     (1, 64, 64, 0),
     (640, 2048, 256, 112),  # many tiles per CTA: accumulator double-buffering, ring wrap-around
+    (512, 1024, 512, 2000),  # pair of SMs per 256-row tile (cta_group::2), automatic width
+    (300, 528, 1032, 2176),  # pair: ragged M (second half-tile partly empty), N and K tails
+    (640, 2048, 256, 2112),  # pair: several tiles per pair
+    (129, 256, 128, 2256),   # pair: second CTA holds a single live row
+    (4000, 4608, 320, 0),    # many row tiles: automatic plan
 ]
 
 
@@ -57,7 +62,15 @@ def test_gemm_bf16_store(M, N, K, tile_n):
     _close_bf16(got, want)
 
 
-@pytest.mark.parametrize("M,N,K,tile_n", GEMM_SHAPES[:5])
+RESIDUAL_SHAPES = GEMM_SHAPES[:5] + [
+    (512, 1024, 2048, 22128),   # pair + K split in two: slices add into X with reductions
+    (300, 528, 4104, 31064),    # single CTA, three K slices, K tail in the last slice
+    (512, 512, 12288, 0),       # automatic plan for a narrow, deep projection
+    (512, 4096, 1024, 2240),    # pair, width 240
+]
+
+
+@pytest.mark.parametrize("M,N,K,tile_n", RESIDUAL_SHAPES)
 def test_gemm_bf16_residual(M, N, K, tile_n):
     b = _b()
     A = _bf16(2, 0, (M, K), 1.0)
@@ -71,7 +84,8 @@ def test_gemm_bf16_residual(M, N, K, tile_n):
 
 
 @pytest.mark.parametrize("M,F,K,tile_n", [(128, 128, 64, 0), (200, 336, 192, 0), (512, 1408, 512, 224),
-                                          (77, 136, 72, 64), (640, 2048, 256, 96)])
+                                          (77, 136, 72, 64), (640, 2048, 256, 96), (512, 1408, 512, 2224),
+                                          (200, 336, 192, 2064), (1000, 2048, 256, 2256)])
 def test_gemm_bf16_swiglu(M, F, K, tile_n):
     b = _b()
     A = _bf16(3, 0, (M, K), 1.0)
