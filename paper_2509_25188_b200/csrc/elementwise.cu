@@ -43,33 +43,131 @@ __global__ void embed_rmsnorm_kernel(const int32_t *tokens, int64_t tok_stride, 
     nr[i] = from_f32<T>(to_f32(e[i]) * gain[i] * inv);
 }
 
+__device__ __forceinline__ void store4(float *p, float a, float b, float c, float d) {
+  *reinterpret_cast<float4 *>(p) = make_float4(a, b, c, d);
+}
+__device__ __forceinline__ void store4(bf16 *p, float a, float b, float c, float d) {
+  __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+  uint2 u;
+  u.x = *reinterpret_cast<uint32_t *>(&lo);
+  u.y = *reinterpret_cast<uint32_t *>(&hi);
+  *reinterpret_cast<uint2 *>(p) = u;
+}
+
+// One block per row; rows up to 4 * 4 * blockDim floats stay in registers between the two passes.
 template <typename T>
-__global__ void rmsnorm_kernel(const float *x, const float *gain, float eps, T *n, int d) {
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const float *x, const float *gain, float eps, T *n, int d) {
   __shared__ float red[32];
-  int row = blockIdx.x;
+  const int row = blockIdx.x;
   const float4 *xr = reinterpret_cast<const float4 *>(x + (int64_t)row * d);
-  int d4 = d >> 2;
+  const int d4 = d >> 2;
+  constexpr int CACHE = 4;
+  float4 v[CACHE];
   float ss = 0.f;
-  for (int i = threadIdx.x; i < d4; i += blockDim.x) {
-    float4 v = xr[i];
-    ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+#pragma unroll
+  for (int k = 0; k < CACHE; ++k) {
+    const int i = threadIdx.x + k * blockDim.x;
+    v[k] = (i < d4) ? xr[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
   }
-  float tot = block_sum(ss, red);
-  float inv = 1.0f / sqrtf(tot / (float)d + eps);
+  for (int i = threadIdx.x + CACHE * blockDim.x; i < d4; i += blockDim.x) {
+    float4 w = xr[i];
+    ss += w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w;
+  }
+  const float tot = block_sum(ss, red);
+  const float inv = 1.0f / sqrtf(tot / (float)d + eps);
   const float4 *g4 = reinterpret_cast<const float4 *>(gain);
   T *nr = n + (int64_t)row * d;
-  for (int i = threadIdx.x; i < d4; i += blockDim.x) {
-    float4 v = xr[i];
-    float4 g = g4[i];
-    nr[4 * i + 0] = from_f32<T>(v.x * g.x * inv);
-    nr[4 * i + 1] = from_f32<T>(v.y * g.y * inv);
-    nr[4 * i + 2] = from_f32<T>(v.z * g.z * inv);
-    nr[4 * i + 3] = from_f32<T>(v.w * g.w * inv);
+#pragma unroll
+  for (int k = 0; k < CACHE; ++k) {
+    const int i = threadIdx.x + k * blockDim.x;
+    if (i < d4) {
+      const float4 g = g4[i];
+      store4(nr + 4 * i, v[k].x * g.x * inv, v[k].y * g.y * inv, v[k].z * g.z * inv, v[k].w * g.w * inv);
+    }
+  }
+  for (int i = threadIdx.x + CACHE * blockDim.x; i < d4; i += blockDim.x) {
+    const float4 w = xr[i];
+    const float4 g = g4[i];
+    store4(nr + 4 * i, w.x * g.x * inv, w.y * g.y * inv, w.z * g.z * inv, w.w * g.w * inv);
   }
 }
 
+template <typename T> struct Vec8;
+template <> struct Vec8<bf16> {
+  uint4 raw;
+  __device__ __forceinline__ void load(const bf16 *p) { raw = *reinterpret_cast<const uint4 *>(p); }
+  __device__ __forceinline__ void store(bf16 *p) const { *reinterpret_cast<uint4 *>(p) = raw; }
+  __device__ __forceinline__ float get(int i) const {
+    const __nv_bfloat16 *h = reinterpret_cast<const __nv_bfloat16 *>(&raw);
+    return __bfloat162float(h[i]);
+  }
+  __device__ __forceinline__ void set(int i, float f) {
+    __nv_bfloat16 *h = reinterpret_cast<__nv_bfloat16 *>(&raw);
+    h[i] = __float2bfloat16_rn(f);
+  }
+};
+template <> struct Vec8<float> {
+  float4 a, b;
+  __device__ __forceinline__ void load(const float *p) {
+    a = *reinterpret_cast<const float4 *>(p);
+    b = *reinterpret_cast<const float4 *>(p + 4);
+  }
+  __device__ __forceinline__ void store(float *p) const {
+    *reinterpret_cast<float4 *>(p) = a;
+    *reinterpret_cast<float4 *>(p + 4) = b;
+  }
+  __device__ __forceinline__ float get(int i) const { return reinterpret_cast<const float *>(&a)[i]; }
+  __device__ __forceinline__ void set(int i, float f) { reinterpret_cast<float *>(&a)[i] = f; }
+};
+
 // Rotates q and k (pair (i, i+dh/2) by the tabulated angle of the row's position) and writes
 // q to the packed query buffer and k, v to the key/value store at [sequence, position].
+// One work item = 8 consecutive pair indices of one head (16-byte accesses); needs dh % 16 == 0.
+template <typename T>
+__global__ void __launch_bounds__(256) rope_scatter_vec_kernel(const T *qkv, const SeqMeta *meta,
+                                                                const int32_t *row_slot, const float2 *cs_table,
+                                                                T *q, T *kc, T *vc, int64_t kv_seq_stride, int H,
+                                                                int dh) {
+  const int row = blockIdx.x;
+  const SeqMeta m = meta[row_slot[row]];
+  const int pos = m.pos0 + (row - m.row0);
+  const int half = dh >> 1, hd = H * dh, per_head = half >> 3;
+  const T *src = qkv + (int64_t)row * 3 * hd;
+  T *qd = q + (int64_t)row * hd;
+  T *kd = kc + (int64_t)m.seq * kv_seq_stride + (int64_t)pos * hd;
+  T *vd = vc + (int64_t)m.seq * kv_seq_stride + (int64_t)pos * hd;
+  const float2 *cs = cs_table + (int64_t)pos * half;
+  for (int item = threadIdx.x; item < H * per_head; item += blockDim.x) {
+    const int h = item / per_head, c = item - h * per_head;
+    const int a = h * dh + c * 8, b = a + half;
+    float2 t[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+      *reinterpret_cast<float4 *>(&t[2 * i]) = *reinterpret_cast<const float4 *>(&cs[c * 8 + 2 * i]);
+    Vec8<T> x1, x2, y1, y2;
+    x1.load(src + a); x2.load(src + b);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float u = x1.get(i), w = x2.get(i);
+      y1.set(i, u * t[i].x - w * t[i].y);
+      y2.set(i, w * t[i].x + u * t[i].y);
+    }
+    y1.store(qd + a); y2.store(qd + b);
+    x1.load(src + hd + a); x2.load(src + hd + b);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const float u = x1.get(i), w = x2.get(i);
+      y1.set(i, u * t[i].x - w * t[i].y);
+      y2.set(i, w * t[i].x + u * t[i].y);
+    }
+    y1.store(kd + a); y2.store(kd + b);
+    x1.load(src + 2 * hd + a); x2.load(src + 2 * hd + b);
+    x1.store(vd + a); x2.store(vd + b);
+  }
+}
+
+// Scalar form for head sizes that are not a multiple of 16.
 template <typename T>
 __global__ void rope_scatter_kernel(const T *qkv, const SeqMeta *meta, const int32_t *row_slot,
                                     const float2 *cs_table, T *q, T *kc, T *vc,
@@ -176,7 +274,10 @@ template <typename T>
 cudaError_t launch_rope_scatter(cudaStream_t st, const T *qkv, const SeqMeta *meta,
                                 const int32_t *row_slot, const float2 *cs_table, T *q, T *kc, T *vc,
                                 int64_t kv_seq_stride, int rows, int H, int dh) {
-  rope_scatter_kernel<T><<<rows, 256, 0, st>>>(qkv, meta, row_slot, cs_table, q, kc, vc, kv_seq_stride, H, dh);
+  if (dh % 16 == 0 && (H * dh) % 8 == 0)
+    rope_scatter_vec_kernel<T><<<rows, 256, 0, st>>>(qkv, meta, row_slot, cs_table, q, kc, vc, kv_seq_stride, H, dh);
+  else
+    rope_scatter_kernel<T><<<rows, 256, 0, st>>>(qkv, meta, row_slot, cs_table, q, kc, vc, kv_seq_stride, H, dh);
   return cudaGetLastError();
 }
 template <typename T>

@@ -36,6 +36,7 @@ def main():
     ap.add_argument("--ff", type=int, default=12288)
     ap.add_argument("--vocab", type=int, default=126464)
     ap.add_argument("--heads", type=int, default=32)
+    ap.add_argument("--ring", type=int, default=0, help="number of weight buffers to rotate through (0 = enough to exceed L2)")
     a = ap.parse_args()
     dev = "cuda:0"
     torch.manual_seed(0)
@@ -46,7 +47,7 @@ def main():
         return (torch.randn(r, c, device=dev) * std).to(torch.bfloat16)
 
     def ring(r, c, min_bytes=400e6):
-        n = max(2, int(min_bytes // (r * c * 2)) + 1)
+        n = a.ring if a.ring > 0 else max(2, int(min_bytes // (r * c * 2)) + 1)
         return [rnd(r, c) for _ in range(n)]
 
     if a.case == "qkv":
@@ -101,7 +102,14 @@ def main():
         torch.cuda.synchronize()
         tot += e0.elapsed_time(e1)
     ms = tot / a.iters
-    print(json.dumps({"case": a.case, "rows": T, "tile_n": a.tile_n, "ms": ms, "tflops": flops / ms / 1e9,
+    # the same launches back to back (no host synchronisation in between)
+    e0.record()
+    for i in range(a.iters):
+        run(i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms_b2b = e0.elapsed_time(e1) / a.iters
+    print(json.dumps({"case": a.case, "rows": T, "tile_n": a.tile_n, "ms": ms, "ms_back_to_back": ms_b2b, "tflops_b2b": flops / ms_b2b / 1e9, "tflops": flops / ms / 1e9,
                       "gbs": byts / ms / 1e6, "flops": flops, "bytes": byts}))
 
 
