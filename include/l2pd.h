@@ -245,6 +245,28 @@ l2pd_status l2pd_lm_head_bf16(void *stream, const void *A, const void *W, const 
                               int32_t *d_pred, float *d_conf, float *d_logits, int32_t check);
 int64_t l2pd_lm_head_scratch_elems(int32_t R, int32_t V);
 
+/*
+ * The same LM head + confidence head for callers that cannot allocate device memory.  (The paper
+ * has no counterpart to this entry point; it exists for deployment reasons only.)  Some hosts run
+ * this library where cudaMalloc is off limits at call time: inside a serving loop whose memory is
+ * carved up front and handed out by the host's own arena, under a framework that forbids driver
+ * allocations once a stream is being captured, or in a process whose device memory is fully
+ * committed to weights and caches.  Those callers still pass inputs (A, W, bias) and outputs
+ * (d_pred, d_conf) as DEVICE pointers, but no scratch: the per-tile reduction records go to a
+ * fixed 3 MiB array compiled into the library, which every GPU that loads the library holds until
+ * the process exits.  Limits: R <= 128 rows, V <= 131072; larger sizes return L2PD_ERR_SHAPE and
+ * launch nothing.  The call makes no cudaMalloc/cudaFree and calls no allocating routine.
+ * The first call on each device looks up the array's device address (the calling thread's current
+ * device must be the one the pointers belong to); make that first call before any stream capture.
+ * All calls on a device share the one array and its contents persist between calls: the call
+ * clears the status word it needs at zero and rewrites every record it later reads, so stale
+ * contents are harmless, but two calls that overlap on the GPU (different streams, or threads)
+ * race on it — serialise them.  Results equal l2pd_lm_head_bf16's.
+ */
+l2pd_status l2pd_lm_head_bf16_static(void *stream, const void *A, const void *W, const float *bias,
+                                     int32_t R, int32_t V, int32_t K, int32_t *d_pred, float *d_conf,
+                                     int32_t check);
+
 /* Bidirectional attention, bf16: q [Tq, H*dh], k and v [Tk, H*dh] (row stride given in
  * elements), out [Tq, H*dh]; softmax(q k^T / sqrt(dh)) v per head, no mask. dh 64 or 128. */
 l2pd_status l2pd_attention_bf16(void *stream, const void *q, const void *k, const void *v,

@@ -58,7 +58,7 @@ EXPORTS = ["l2pd_init", "l2pd_state_reset", "l2pd_denoise_step", "l2pd_decode", 
            "l2pd_state_tokens", "l2pd_state_masked", "l2pd_set_capture", "l2pd_last_step_rows",
            "l2pd_launch_count", "l2pd_last_step_ms", "l2pd_profile_enable", "l2pd_profile_read", "l2pd_last_error", "l2pd_destroy",
            "l2pd_gemm_bf16", "l2pd_gemm_bf16_residual", "l2pd_gemm_bf16_swiglu", "l2pd_lm_head_bf16",
-           "l2pd_lm_head_scratch_elems", "l2pd_attention_bf16"]
+           "l2pd_lm_head_scratch_elems", "l2pd_attention_bf16", "l2pd_lm_head_bf16_static"]
 
 
 KINDS = ["embed", "gemm_qkv", "rope", "attention", "gemm_o", "rmsnorm", "gemm_gate_up", "gemm_down",
@@ -98,6 +98,7 @@ def _load() -> C.CDLL:
     lib.l2pd_lm_head_bf16.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, i32]
     lib.l2pd_lm_head_scratch_elems.argtypes = [i32, i32]
     lib.l2pd_lm_head_scratch_elems.restype = i64
+    lib.l2pd_lm_head_bf16_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, i32]
     lib.l2pd_attention_bf16.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, i64]
     return lib
 
@@ -352,6 +353,20 @@ def lm_head_bf16(A: torch.Tensor, W: torch.Tensor, bias: Optional[torch.Tensor] 
                                  R, V, K, scratch.data_ptr(), pred.data_ptr(), conf.data_ptr(),
                                  logits.data_ptr() if want_logits else None, 1))
     return pred, conf, logits
+
+
+def lm_head_bf16_static(A: torch.Tensor, W: torch.Tensor, bias: Optional[torch.Tensor], pred: torch.Tensor,
+                        conf: torch.Tensor):
+    """LM head + confidence head through the entry point that allocates nothing: for callers whose
+    device memory is handed out by their own arena (or is fully committed) and who therefore pass
+    only inputs and outputs; the scratch is a fixed array inside the library (R <= 128, V <= 131072).
+    `pred` (int32 [R]) and `conf` (float32 [R]) are caller-owned device tensors."""
+    R, K = A.shape
+    V = W.shape[0]
+    _check(lib.l2pd_lm_head_bf16_static(_stream(), A.data_ptr(), W.data_ptr(),
+                                        bias.data_ptr() if bias is not None else None, R, V, K,
+                                        pred.data_ptr(), conf.data_ptr(), 1))
+    return pred, conf
 
 
 def attention_bf16(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, H: int, dh: int) -> torch.Tensor:
