@@ -277,12 +277,10 @@ def run_ours(args):
     clocks = sampler.stop() if sampler else None
 
     if world > 1:
-        t = torch.tensor([ms, ms_e2e], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, ms_e2e = float(t[0]), float(t[1])
-        c = torch.tensor([tokens, tokens_e2e, launches], device=dev, dtype=torch.float64)
-        dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        tokens, tokens_e2e, launches = int(c[0]), int(c[1]), int(c[2])
+        from paper_2509_25188_b200 import replicas
+        ms, (tokens, launches) = replicas.reduce_timing(ms, [tokens, launches], device=dev)
+        ms_e2e, (tokens_e2e,) = replicas.reduce_timing(ms_e2e, [tokens_e2e], device=dev)
+        tokens, tokens_e2e, launches = int(tokens), int(tokens_e2e), int(launches)
 
     # ---- untimed: per-kernel breakdown of one step
     breakdown = {}

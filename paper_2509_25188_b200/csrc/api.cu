@@ -78,6 +78,13 @@ struct l2pd_ctx {
   std::string err;
 };
 
+namespace l2pd {
+bool pdl_enabled() {
+  static const bool on = [] { const char *e = getenv("L2PD_NO_PDL"); return !(e && e[0] == '1'); }();
+  return on;
+}
+}  // namespace l2pd
+
 namespace {
 
 l2pd_status set_err(l2pd_ctx *c, l2pd_status s, const char *fmt, ...) {

@@ -81,6 +81,8 @@ __global__ void __launch_bounds__(128) attention_bf16_kernel(const AttnParams p)
   const uint32_t sK = sQ + BQ * DH * 2;
   const uint32_t sV = sK + 2 * TILE_BYTES;
 
+  grid_dep_launch();
+  grid_dep_wait();
   const SeqMeta m = p.use_single ? p.single : p.meta[blockIdx.z];
   const int q0 = blockIdx.x * BQ;
   if (q0 >= m.n_rows) return;
@@ -225,8 +227,7 @@ cudaError_t launch(cudaStream_t st, const AttnParams &p, dim3 grid) {
   const int smem = (BQ + 4 * BKV) * DH * 2;
   cudaError_t e = cudaFuncSetAttribute(attention_bf16_kernel<DH>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
   if (e != cudaSuccess) return e;
-  attention_bf16_kernel<DH><<<grid, 128, smem, st>>>(p);
-  return cudaGetLastError();
+  return launch_kernel(attention_bf16_kernel<DH>, grid, dim3(128), (size_t)smem, st, p);
 }
 
 }  // namespace

@@ -27,6 +27,8 @@ __global__ void __launch_bounds__(256) decide_kernel(DecideArgs a) {
   __shared__ int s_unmask[MAX_S];
   __shared__ int s_any, s_e, s_left;
 
+  grid_dep_launch();
+  grid_dep_wait();
   const int slot = blockIdx.x;
   const SeqMeta m = a.meta[slot];
   const int s = a.s;
@@ -172,8 +174,7 @@ __global__ void __launch_bounds__(256) decide_kernel(DecideArgs a) {
 }  // namespace
 
 cudaError_t launch_decide(cudaStream_t st, const DecideArgs &a, int n_slots) {
-  decide_kernel<<<n_slots, 256, 0, st>>>(a);
-  return cudaGetLastError();
+  return launch_kernel(decide_kernel, dim3(n_slots), dim3(256), 0, st, a);
 }
 
 }  // namespace l2pd

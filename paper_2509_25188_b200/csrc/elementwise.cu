@@ -23,6 +23,8 @@ template <typename T>
 __global__ void embed_rmsnorm_kernel(const int32_t *tokens, int64_t tok_stride, const SeqMeta *meta,
                                      const int32_t *row_slot, const T *emb, const float *gain,
                                      float eps, float *x, T *n, int d) {
+  grid_dep_launch();
+  grid_dep_wait();
   __shared__ float red[32];
   int row = blockIdx.x;
   SeqMeta m = meta[row_slot[row]];
@@ -57,6 +59,8 @@ __device__ __forceinline__ void store4(bf16 *p, float a, float b, float c, float
 // One block per row; rows up to 4 * 4 * blockDim floats stay in registers between the two passes.
 template <typename T>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *x, const float *gain, float eps, T *n, int d) {
+  grid_dep_launch();
+  grid_dep_wait();
   __shared__ float red[32];
   const int row = blockIdx.x;
   const float4 *xr = reinterpret_cast<const float4 *>(x + (int64_t)row * d);
@@ -129,6 +133,8 @@ __global__ void __launch_bounds__(256) rope_scatter_vec_kernel(const T *qkv, con
                                                                 const int32_t *row_slot, const float2 *cs_table,
                                                                 T *q, T *kc, T *vc, int64_t kv_seq_stride, int H,
                                                                 int dh) {
+  grid_dep_launch();
+  grid_dep_wait();
   const int row = blockIdx.x;
   const SeqMeta m = meta[row_slot[row]];
   const int pos = m.pos0 + (row - m.row0);
@@ -172,6 +178,8 @@ template <typename T>
 __global__ void rope_scatter_kernel(const T *qkv, const SeqMeta *meta, const int32_t *row_slot,
                                     const float2 *cs_table, T *q, T *kc, T *vc,
                                     int64_t kv_seq_stride, int H, int dh) {
+  grid_dep_launch();
+  grid_dep_wait();
   int row = blockIdx.x;
   SeqMeta m = meta[row_slot[row]];
   int pos = m.pos0 + (row - m.row0);
@@ -202,6 +210,8 @@ __global__ void rope_scatter_kernel(const T *qkv, const SeqMeta *meta, const int
 template <typename T>
 __global__ void final_norm_gather_kernel(const float *x, const SeqMeta *meta, const float *gain,
                                          float eps, T *nf, int n_slots, int s, int d) {
+  grid_dep_launch();
+  grid_dep_wait();
   __shared__ float red[32];
   int r = blockIdx.x;
   int slot = r / s, j = r - slot * s;
@@ -226,6 +236,8 @@ __global__ void final_norm_gather_kernel(const float *x, const SeqMeta *meta, co
 }
 
 __global__ void build_row_map_kernel(const SeqMeta *meta, int32_t *row_slot) {
+  grid_dep_launch();
+  grid_dep_wait();
   SeqMeta m = meta[blockIdx.x];
   for (int i = threadIdx.x; i < m.n_rows; i += blockDim.x) row_slot[m.row0 + i] = blockIdx.x;
 }
@@ -233,6 +245,8 @@ __global__ void build_row_map_kernel(const SeqMeta *meta, int32_t *row_slot) {
 // Algorithm 2: X <- concat(prompt, [MASK]^G); all generation positions masked.
 __global__ void state_reset_kernel(const int32_t *prompts, int P, int G, int vocab, int mask_id,
                                    int32_t *tokens, uint8_t *masked, SeqState s, int32_t *bad) {
+  grid_dep_launch();
+  grid_dep_wait();
   int b = blockIdx.x;
   int L = P + G;
   for (int i = threadIdx.x; i < L; i += blockDim.x) {
@@ -250,6 +264,8 @@ __global__ void state_reset_kernel(const int32_t *prompts, int P, int G, int voc
 }
 
 __global__ void gather_response_kernel(const int32_t *tokens, int P, int G, int32_t *out) {
+  grid_dep_launch();
+  grid_dep_wait();
   int b = blockIdx.x;
   for (int i = threadIdx.x; i < G; i += blockDim.x)
     out[(int64_t)b * G + i] = tokens[(int64_t)b * (P + G) + P + i];
@@ -261,45 +277,39 @@ template <typename T>
 cudaError_t launch_embed_rmsnorm(cudaStream_t st, const int32_t *tokens, int64_t tok_stride,
                                  const SeqMeta *meta, const int32_t *row_slot, const T *emb,
                                  const float *gain, float eps, float *x, T *n, int rows, int d) {
-  embed_rmsnorm_kernel<T><<<rows, 256, 0, st>>>(tokens, tok_stride, meta, row_slot, emb, gain, eps, x, n, d);
-  return cudaGetLastError();
+  return launch_kernel(embed_rmsnorm_kernel<T>, dim3(rows), dim3(256), 0, st, tokens, tok_stride, meta, row_slot, emb, gain, eps, x, n, d);
 }
 template <typename T>
 cudaError_t launch_rmsnorm(cudaStream_t st, const float *x, const float *gain, float eps, T *n,
                            int rows, int d) {
-  rmsnorm_kernel<T><<<rows, 256, 0, st>>>(x, gain, eps, n, d);
-  return cudaGetLastError();
+  return launch_kernel(rmsnorm_kernel<T>, dim3(rows), dim3(256), 0, st, x, gain, eps, n, d);
 }
 template <typename T>
 cudaError_t launch_rope_scatter(cudaStream_t st, const T *qkv, const SeqMeta *meta,
                                 const int32_t *row_slot, const float2 *cs_table, T *q, T *kc, T *vc,
                                 int64_t kv_seq_stride, int rows, int H, int dh) {
   if (dh % 16 == 0 && (H * dh) % 8 == 0)
-    rope_scatter_vec_kernel<T><<<rows, 256, 0, st>>>(qkv, meta, row_slot, cs_table, q, kc, vc, kv_seq_stride, H, dh);
-  else
-    rope_scatter_kernel<T><<<rows, 256, 0, st>>>(qkv, meta, row_slot, cs_table, q, kc, vc, kv_seq_stride, H, dh);
-  return cudaGetLastError();
+    return launch_kernel(rope_scatter_vec_kernel<T>, dim3(rows), dim3(256), 0, st, qkv, meta, row_slot, cs_table, q, kc, vc,
+                         kv_seq_stride, H, dh);
+  return launch_kernel(rope_scatter_kernel<T>, dim3(rows), dim3(256), 0, st, qkv, meta, row_slot, cs_table, q, kc, vc,
+                       kv_seq_stride, H, dh);
 }
 template <typename T>
 cudaError_t launch_final_norm_gather(cudaStream_t st, const float *x, const SeqMeta *meta,
                                      const float *gain, float eps, T *nf, int n_slots, int s,
                                      int rows_padded, int d) {
-  final_norm_gather_kernel<T><<<rows_padded, 256, 0, st>>>(x, meta, gain, eps, nf, n_slots, s, d);
-  return cudaGetLastError();
+  return launch_kernel(final_norm_gather_kernel<T>, dim3(rows_padded), dim3(256), 0, st, x, meta, gain, eps, nf, n_slots, s, d);
 }
 cudaError_t launch_build_row_map(cudaStream_t st, const SeqMeta *meta, int n_slots, int32_t *row_slot) {
-  build_row_map_kernel<<<n_slots, 256, 0, st>>>(meta, row_slot);
-  return cudaGetLastError();
+  return launch_kernel(build_row_map_kernel, dim3(n_slots), dim3(256), 0, st, meta, row_slot);
 }
 cudaError_t launch_state_reset(cudaStream_t st, const int32_t *prompts, int B, int P, int G, int vocab,
                                int mask_id, int32_t *tokens, uint8_t *masked, SeqState s, int32_t *bad) {
-  state_reset_kernel<<<B, 256, 0, st>>>(prompts, P, G, vocab, mask_id, tokens, masked, s, bad);
-  return cudaGetLastError();
+  return launch_kernel(state_reset_kernel, dim3(B), dim3(256), 0, st, prompts, P, G, vocab, mask_id, tokens, masked, s, bad);
 }
 cudaError_t launch_gather_response(cudaStream_t st, const int32_t *tokens, int B, int P, int G,
                                    int32_t *out) {
-  gather_response_kernel<<<B, 256, 0, st>>>(tokens, P, G, out);
-  return cudaGetLastError();
+  return launch_kernel(gather_response_kernel, dim3(B), dim3(256), 0, st, tokens, P, G, out);
 }
 
 #define INSTANTIATE(T)                                                                              \

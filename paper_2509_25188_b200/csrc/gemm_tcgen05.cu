@@ -231,6 +231,9 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
   if (CG == 2) ptx::cluster_sync();     // the peer's barriers exist before anything arrives on them
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  // set-up above overlaps the previous kernel's tail; from here on its results are needed
+  grid_dep_launch();
+  grid_dep_wait();
 
   const int num_units = p.m_tiles * p.n_tiles * p.k_splits;
   const int num_kb = (p.K + TILE_K - 1) / TILE_K;
@@ -411,6 +414,8 @@ EncodeTiledFn get_encode_fn() {
 
 __global__ void merge_partials_kernel(const float *part_m, const float *part_s, const int32_t *part_i,
                                       int n_tiles, int rows_padded, int32_t *pred, float *conf) {
+  grid_dep_launch();
+  grid_dep_wait();
   const int r = blockIdx.x, lane = threadIdx.x;
   float mx = -INFINITY, sum = 0.f;
   int ix = 0x7fffffff;
@@ -523,7 +528,8 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
 #define L2PD_LAUNCH(KERNEL, EPI)                                                                      \
   e = cudaFuncSetAttribute(KERNEL<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET - 1024); \
   if (e != cudaSuccess) return e;                                                                    \
-  KERNEL<EPI><<<grid, 192, smem, st>>>(g.a->map, g.b->map, b2, p);
+  e = launch_kernel(KERNEL<EPI>, dim3(grid), dim3(192), smem, st, g.a->map, g.b->map, b2, p);                \
+  if (e != cudaSuccess) return e;
   if (cg == 1) {
     switch (g.epi) {
       case EPI_STORE: L2PD_LAUNCH(gemm_tcgen05_kernel, EPI_STORE) break;
@@ -547,8 +553,8 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
 cudaError_t launch_merge_partials(cudaStream_t st, const float *part_m, const float *part_s,
                                   const int32_t *part_i, int n_tiles, int rows_padded, int R,
                                   int32_t *pred, float *conf) {
-  merge_partials_kernel<<<R, 32, 0, st>>>(part_m, part_s, part_i, n_tiles, rows_padded, pred, conf);
-  return cudaGetLastError();
+  return launch_kernel(merge_partials_kernel, dim3(R), dim3(32), 0, st, part_m, part_s, part_i, n_tiles, rows_padded, pred,
+                       conf);
 }
 
 }  // namespace l2pd

@@ -19,6 +19,8 @@ template <typename T, int EPI>
 __global__ void __launch_bounds__(256) simt_gemm_kernel(const T *__restrict__ A, const T *__restrict__ W,
                                                         const T *__restrict__ W2, void *Cv,
                                                         const float *__restrict__ bias, int M, int N, int K) {
+  grid_dep_launch();
+  grid_dep_wait();
   __shared__ float As[BK][BM + 1];
   __shared__ float Ws[BK][BN + 1];
   __shared__ float W2s[EPI == EPI_SWIGLU ? BK : 1][BN + 1];
@@ -85,6 +87,8 @@ __global__ void simt_attention_kernel(const T *__restrict__ q, const T *__restri
                                       const T *__restrict__ vc, const SeqMeta *meta,
                                       const int32_t *row_slot, T *out, int64_t kv_seq_stride, int H,
                                       int dh) {
+  grid_dep_launch();
+  grid_dep_wait();
   extern __shared__ float sm[];
   float *qs = sm;          // [dh]
   float *sc = sm + dh;     // [kv_len]
@@ -137,6 +141,8 @@ __global__ void simt_attention_kernel(const T *__restrict__ q, const T *__restri
 // Per-row max, sum of exp and argmax (lowest id on ties) of stored fp32 logits: one tile.
 __global__ void row_softmax_partials_kernel(const float *logits, int V, float *part_m, float *part_s,
                                             int32_t *part_i) {
+  grid_dep_launch();
+  grid_dep_wait();
   __shared__ float rm[32];
   __shared__ int ri[32];
   __shared__ float rs[32];
@@ -180,13 +186,12 @@ cudaError_t launch_simt_gemm(cudaStream_t st, int epi, const T *A, const T *W, c
                              const float *bias, int M, int N, int K) {
   dim3 grid(ceil_div(N, BN), ceil_div(M, BM));
   switch (epi) {
-    case EPI_STORE: simt_gemm_kernel<T, EPI_STORE><<<grid, 256, 0, st>>>(A, W, W2, C, bias, M, N, K); break;
-    case EPI_RESIDUAL: simt_gemm_kernel<T, EPI_RESIDUAL><<<grid, 256, 0, st>>>(A, W, W2, C, bias, M, N, K); break;
-    case EPI_SWIGLU: simt_gemm_kernel<T, EPI_SWIGLU><<<grid, 256, 0, st>>>(A, W, W2, C, bias, M, N, K); break;
-    case EPI_STORE_F32: simt_gemm_kernel<T, EPI_STORE_F32><<<grid, 256, 0, st>>>(A, W, W2, C, bias, M, N, K); break;
+    case EPI_STORE: return launch_kernel(simt_gemm_kernel<T, EPI_STORE>, grid, dim3(256), 0, st, A, W, W2, C, bias, M, N, K);
+    case EPI_RESIDUAL: return launch_kernel(simt_gemm_kernel<T, EPI_RESIDUAL>, grid, dim3(256), 0, st, A, W, W2, C, bias, M, N, K);
+    case EPI_SWIGLU: return launch_kernel(simt_gemm_kernel<T, EPI_SWIGLU>, grid, dim3(256), 0, st, A, W, W2, C, bias, M, N, K);
+    case EPI_STORE_F32: return launch_kernel(simt_gemm_kernel<T, EPI_STORE_F32>, grid, dim3(256), 0, st, A, W, W2, C, bias, M, N, K);
     default: return cudaErrorInvalidValue;
   }
-  return cudaGetLastError();
 }
 
 template <typename T>
@@ -199,15 +204,13 @@ cudaError_t launch_simt_attention(cudaStream_t st, const T *q, const T *kc, cons
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
   }
-  simt_attention_kernel<T><<<dim3(rows, H), 128, smem, st>>>(q, kc, vc, meta, row_slot, out,
-                                                            kv_seq_stride, H, dh);
-  return cudaGetLastError();
+  return launch_kernel(simt_attention_kernel<T>, dim3(rows, H), dim3(128), smem, st, q, kc, vc, meta, row_slot, out,
+                       kv_seq_stride, H, dh);
 }
 
 cudaError_t launch_row_softmax_partials(cudaStream_t st, const float *logits, int R, int V,
                                         float *part_m, float *part_s, int32_t *part_i) {
-  row_softmax_partials_kernel<<<R, 256, 0, st>>>(logits, V, part_m, part_s, part_i);
-  return cudaGetLastError();
+  return launch_kernel(row_softmax_partials_kernel, dim3(R), dim3(256), 0, st, logits, V, part_m, part_s, part_i);
 }
 
 template cudaError_t launch_simt_gemm<float>(cudaStream_t, int, const float *, const float *,
