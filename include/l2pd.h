@@ -267,11 +267,17 @@ l2pd_status l2pd_lm_head_bf16_static(void *stream, const void *A, const void *W,
                                      int32_t R, int32_t V, int32_t K, int32_t *d_pred, float *d_conf,
                                      int32_t check);
 
-/* Bidirectional attention, bf16: q [Tq, H*dh], k and v [Tk, H*dh] (row stride given in
- * elements), out [Tq, H*dh]; softmax(q k^T / sqrt(dh)) v per head, no mask. dh 64 or 128. */
+/* Bidirectional attention, bf16 (the mask predictor of Section 3.1 attends over the whole
+ * sequence: no causal mask): q [Tq, H*dh], k and v [Tk, H*dh] (row stride given in elements),
+ * out [Tq, H*dh]; softmax(q k^T / sqrt(dh)) v per head. dh 64 or 128.  All pointers are device
+ * memory owned by the caller and 16-byte aligned.  impl: 0 = tensor-memory kernel (tcgen05) when
+ * dh is 128 and the strides are multiples of 8, else the warp-level kernel; 1 = always the
+ * warp-level (mma.sync) kernel.  check != 0 synchronises the stream and turns a device wait that
+ * ran out into L2PD_ERR_TIMEOUT. */
 l2pd_status l2pd_attention_bf16(void *stream, const void *q, const void *k, const void *v,
                                 void *out, int32_t Tq, int32_t Tk, int32_t H, int32_t dh,
-                                int64_t q_stride, int64_t kv_stride, int64_t out_stride);
+                                int64_t q_stride, int64_t kv_stride, int64_t out_stride,
+                                int32_t impl, int32_t check);
 
 #ifdef __cplusplus
 }

@@ -99,7 +99,7 @@ def _load() -> C.CDLL:
     lib.l2pd_lm_head_scratch_elems.argtypes = [i32, i32]
     lib.l2pd_lm_head_scratch_elems.restype = i64
     lib.l2pd_lm_head_bf16_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, i32]
-    lib.l2pd_attention_bf16.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, i64]
+    lib.l2pd_attention_bf16.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, i64, i32, i32]
     return lib
 
 
@@ -369,9 +369,10 @@ def lm_head_bf16_static(A: torch.Tensor, W: torch.Tensor, bias: Optional[torch.T
     return pred, conf
 
 
-def attention_bf16(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, H: int, dh: int) -> torch.Tensor:
+def attention_bf16(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, H: int, dh: int, impl: int = 0) -> torch.Tensor:
+    """impl 0: tensor-memory kernel where it applies (dh 128), 1: the warp-level kernel."""
     Tq, Tk = q.shape[0], k.shape[0]
     out = torch.empty(Tq, H * dh, dtype=torch.bfloat16, device=q.device)
     _check(lib.l2pd_attention_bf16(_stream(), q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
-                                   Tq, Tk, H, dh, q.stride(0), k.stride(0), out.stride(0)))
+                                   Tq, Tk, H, dh, q.stride(0), k.stride(0), out.stride(0), impl, 1))
     return out

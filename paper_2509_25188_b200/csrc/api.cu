@@ -19,6 +19,7 @@ struct l2pd_ctx {
   l2pd_config cfg;
   int device = 0, num_sms = 148;
   bool force_simt = false;   // L2PD_FORCE_SIMT=1: bf16 GEMMs and attention on the CUDA-core cross-check kernels
+  bool attn_tc = false;      // head size 128: attention on tcgen05 (L2PD_ATTN_WARP=1 keeps the mma.sync kernel)
 
   // weights (borrowed device pointers)
   const void *tok_emb = nullptr, *lm_head = nullptr;
@@ -54,7 +55,7 @@ struct l2pd_ctx {
   float2 *cs_table = nullptr;
 
   // TMA descriptors (bf16 path)
-  TmaDesc ta_n, ta_att, ta_h, ta_nf;
+  TmaDesc ta_n, ta_att, ta_h, ta_nf, ta_q, t_kstore, t_vstore;
   std::vector<TmaDesc> tb_qkv, tb_o, tb_gate, tb_up, tb_down;
   TmaDesc tb_lm;
   GemmPlan pl_qkv{}, pl_o{}, pl_gu{}, pl_down{};
@@ -178,7 +179,7 @@ l2pd_status run_gemm_tc(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const Tm
                         const TmaDesc *b2, void *out, int M, int N, int K, const GemmPlan &pl) {
   GemmArgs g{};
   g.epi = epi; g.a = a; g.b = b; g.b2 = b2; g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.out = out;
-  g.cta_group = pl.cta_group; g.k_splits = pl.k_splits;
+  g.cta_group = pl.cta_group; g.k_splits = pl.k_splits; g.slabs = pl.slabs;
   g.status = c->d_status;
   CKLK(kind, launch_gemm_tcgen05(s, g, c->num_sms));
   return L2PD_OK;
@@ -226,7 +227,11 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_QKV, EPI_STORE, n, c->wqkv[l], nullptr, qkv, nullptr, T_rows, 3 * hd, d);
     if (r) return r;
     CKLK(L2PD_K_ROPE, launch_rope_scatter<T>(s, qkv, c->d_meta, c->d_row_slot, c->cs_table, q, kc, vc, c->kv_seq_stride, T_rows, H, dh));
-    if (tc) {
+    if (tc && c->attn_tc) {
+      const int kv_row_base = f.kv_cache_mode ? l * f.max_batch * f.max_seq : 0;
+      CKLK(L2PD_K_ATTENTION, launch_attention_tc(s, c->ta_q, c->t_kstore, c->t_vstore, c->d_meta, (bf16 *)att, hd, f.max_seq,
+                                kv_row_base, n_slots, max_q_rows, H, c->d_status));
+    } else if (tc) {
       CKLK(L2PD_K_ATTENTION, launch_attention_bf16(s, (const bf16 *)q, (const bf16 *)kc, (const bf16 *)vc, c->d_meta, (bf16 *)att, hd, hd,
                                 c->kv_seq_stride, hd, n_slots, max_q_rows, H, dh));
     } else {
@@ -421,7 +426,13 @@ l2pd_status l2pd_init(const l2pd_config *cfg, const l2pd_weights *w, int device,
   if (cudaMemset(c->d_status, 0, 4) != cudaSuccess) return fail(L2PD_ERR_CUDA);
   // the activation buffers back TMA boxes that reach past the live rows: start them defined
   if (cudaMemset(c->n, 0, mr * d * es) != cudaSuccess || cudaMemset(c->att, 0, mr * hd * es) != cudaSuccess ||
-      cudaMemset(c->h, 0, mr * F * es) != cudaSuccess || cudaMemset(c->nf, 0, c->max_lm_rows * d * es) != cudaSuccess)
+      cudaMemset(c->h, 0, mr * F * es) != cudaSuccess || cudaMemset(c->nf, 0, c->max_lm_rows * d * es) != cudaSuccess ||
+      cudaMemset(c->q, 0, mr * hd * es) != cudaSuccess)
+    return fail(L2PD_ERR_CUDA);
+  // key tiles reach past a sequence's last key: what lies there is masked out of the scores, but
+  // the value rows are multiplied by a probability of zero, so they must never hold NaN or Inf
+  if (cudaMemset(c->kc, 0, c->kv_layer_stride * kv_layers * es) != cudaSuccess ||
+      cudaMemset(c->vc, 0, c->kv_layer_stride * kv_layers * es) != cudaSuccess)
     return fail(L2PD_ERR_CUDA);
   c->st.cur_block = c->d_state_ints; c->st.l_eff = c->d_state_ints + f.max_batch;
   c->st.done = c->d_state_ints + 2 * f.max_batch; c->st.steps = c->d_state_ints + 3 * f.max_batch;
@@ -445,6 +456,14 @@ l2pd_status l2pd_init(const l2pd_config *cfg, const l2pd_weights *w, int device,
     l2pd_status s3 = make_tma_2d_bf16(&c->ta_h, c->h, mr, F, 128);
     l2pd_status s4 = make_tma_2d_bf16(&c->ta_nf, c->nf, c->max_lm_rows, d, 128);
     if (s1 || s2 || s3 || s4) return fail(L2PD_ERR_CUDA);
+    const char *aw = getenv("L2PD_ATTN_WARP");
+    c->attn_tc = attention_tc_supported(f.head_dim, hd, hd, hd) && !(aw && aw[0] == '1');
+    if (c->attn_tc) {
+      const int64_t store_rows = (int64_t)kv_layers * f.max_batch * f.max_seq;
+      if (make_tma_2d_bf16(&c->ta_q, c->q, mr, hd, 128) || make_tma_2d_bf16(&c->t_kstore, c->kc, store_rows, hd, 128) ||
+          make_tma_2d_bf16(&c->t_vstore, c->vc, store_rows, hd, 128))
+        return fail(L2PD_ERR_CUDA);
+    }
   }
   if (cudaEventCreate(&c->ev0) != cudaSuccess || cudaEventCreate(&c->ev1) != cudaSuccess) return fail(L2PD_ERR_CUDA);
   c->h_cur_block.assign(f.max_batch, 0); c->h_l_eff.assign(f.max_batch, 0); c->h_done.assign(f.max_batch, 1);
@@ -626,15 +645,18 @@ static l2pd_status gemm_common(void *stream, int epi, const void *A, const void 
   if (M < 1 || N < 8 || K < 8 || (N % 8) || (K % 8)) return L2PD_ERR_SHAPE;
   if (tile_n < 0) return L2PD_ERR_SHAPE;
   const int sms = device_sms();
-  // tile_n = width + 1000 * cta_group + 10000 * k_splits; any part 0 = chosen automatically
-  const int want_ks = tile_n / 10000, want_cg = (tile_n % 10000) / 1000, want_tn = tile_n % 1000;
+  // tile_n = width + 1000 * cta_group + 10000 * k_splits + 100000 * slabs; any part 0 = chosen automatically
+  const int want_sl = tile_n / 100000, want_ks = (tile_n % 100000) / 10000, want_cg = (tile_n % 10000) / 1000,
+            want_tn = tile_n % 1000;
   const int unit = epi == EPI_SWIGLU ? 32 : 16;
   if (want_tn && (want_tn < 32 || want_tn > 256 || (want_tn % unit))) return L2PD_ERR_SHAPE;
-  if (want_cg > 2 || want_ks > 8 || (want_ks > 1 && epi != EPI_RESIDUAL)) return L2PD_ERR_SHAPE;
+  if (want_cg > 2 || want_ks > 8 || (want_ks > 1 && epi != EPI_RESIDUAL) || want_sl > 2) return L2PD_ERR_SHAPE;
   GemmPlan pl = plan_gemm(epi, M, N, K, sms, want_tn);
   if (want_tn) pl.tile_n = want_tn;
   if (want_cg) pl.cta_group = want_cg;
   if (want_ks) pl.k_splits = want_ks;
+  if (want_sl) pl.slabs = want_sl;
+  if (pl.slabs == 2 && pl.cta_group != 2) return L2PD_ERR_SHAPE;
   if (pl.k_splits > ceil_div(K, 64)) pl.k_splits = ceil_div(K, 64);
   int32_t *status = standalone_status();
   if (!status) return L2PD_ERR_CUDA;
@@ -648,6 +670,7 @@ static l2pd_status gemm_common(void *stream, int epi, const void *A, const void 
   GemmArgs g{};
   g.epi = epi; g.a = &ta; g.b = &tb; g.b2 = epi == EPI_SWIGLU ? &tb2 : nullptr;
   g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.cta_group = pl.cta_group; g.k_splits = pl.k_splits;
+  g.slabs = pl.slabs;
   g.out = out; g.status = status;
   if (launch_gemm_tcgen05((cudaStream_t)stream, g, sms) != cudaSuccess) return L2PD_ERR_CUDA;
   return finish_standalone((cudaStream_t)stream, status, check);
@@ -701,13 +724,32 @@ l2pd_status l2pd_lm_head_bf16(void *stream, const void *A, const void *W, const 
 
 l2pd_status l2pd_attention_bf16(void *stream, const void *q, const void *k, const void *v, void *out, int32_t Tq,
                                 int32_t Tk, int32_t H, int32_t dh, int64_t q_stride, int64_t kv_stride,
-                                int64_t out_stride) {
+                                int64_t out_stride, int32_t impl, int32_t check) {
   if (!q || !k || !v || !out) return L2PD_ERR_ARG;
   if (Tq < 1 || Tk < 1 || H < 1 || (dh != 64 && dh != 128) || (q_stride % 8) || (kv_stride % 8) || (out_stride % 2))
     return L2PD_ERR_SHAPE;
+  if (impl != 0 && impl != 1) return L2PD_ERR_ARG;
+  if (q_stride < (int64_t)H * dh || kv_stride < (int64_t)H * dh || out_stride < (int64_t)H * dh) return L2PD_ERR_SHAPE;
+  if (impl == 0 && attention_tc_supported(dh, q_stride, kv_stride, out_stride)) {
+    int32_t *status = standalone_status();
+    if (!status) return L2PD_ERR_CUDA;
+    TmaDesc tq, tk, tv;
+    l2pd_status r = make_tma_2d_bf16_strided(&tq, q, Tq, (int64_t)H * dh, q_stride, 128);
+    if (r) return r;
+    r = make_tma_2d_bf16_strided(&tk, k, Tk, (int64_t)H * dh, kv_stride, 128);
+    if (r) return r;
+    r = make_tma_2d_bf16_strided(&tv, v, Tk, (int64_t)H * dh, kv_stride, 128);
+    if (r) return r;
+    if (launch_attention_tc((cudaStream_t)stream, tq, tk, tv, nullptr, (bf16 *)out, out_stride, 0, 0, Tk, Tq, H, status) !=
+        cudaSuccess)
+      return L2PD_ERR_CUDA;
+    return finish_standalone((cudaStream_t)stream, status, check);
+  }
   cudaError_t e = launch_attention_bf16((cudaStream_t)stream, (const bf16 *)q, (const bf16 *)k, (const bf16 *)v,
                                         nullptr, (bf16 *)out, q_stride, kv_stride, 0, out_stride, Tk, Tq, H, dh);
-  return e == cudaSuccess ? L2PD_OK : L2PD_ERR_CUDA;
+  if (e != cudaSuccess) return L2PD_ERR_CUDA;
+  if (check && cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return L2PD_ERR_CUDA;
+  return L2PD_OK;
 }
 
 }  // extern "C"

@@ -130,17 +130,24 @@ cudaError_t launch_decide(cudaStream_t st, const DecideArgs &a, int n_slots);
 struct TmaDesc { CUtensorMap map; };
 // Encodes a 2-D bf16 row-major tensor [rows, cols] with a box of [box_rows, 64] and 128-byte swizzle.
 l2pd_status make_tma_2d_bf16(TmaDesc *out, const void *ptr, int64_t rows, int64_t cols, int box_rows);
+// The same for rows that are `row_stride` elements apart (a multiple of 8).
+l2pd_status make_tma_2d_bf16_strided(TmaDesc *out, const void *ptr, int64_t rows, int64_t cols, int64_t row_stride,
+                                     int box_rows);
 int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile);
 // How one GEMM is laid over the SMs: CTAs per tile (1, or 2 = a cta_group::2 pair on a 256-row tile),
-// tile width, and K slices (residual epilogue only: slices add into X with vector reductions).
+// tile width, K slices (residual epilogue only: slices add into X with vector reductions), and row
+// slabs per unit (2 = a unit covers two 128 * cta_group row slabs against one load of the weight
+// tile, each slab with its own MMA-issuing thread; its accumulators fill tensor memory, so the
+// drain is not overlapped with the next unit).
 // The B tensor map's box must be tile_n / cta_group rows (SwiGLU: tile_n / 2 for either group size).
-struct GemmPlan { int cta_group, tile_n, k_splits; };
+struct GemmPlan { int cta_group, tile_n, k_splits, slabs; };
 GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n);
 struct GemmArgs {
   int epi;                 // EPI_STORE, EPI_RESIDUAL, EPI_SWIGLU, or EPI_LMHEAD
   const TmaDesc *a, *b, *b2;
   int M, N, K, tile_n;
   int cta_group, k_splits; // 0 / 1 = single CTA, no split
+  int slabs;               // 0 / 1 = one row slab per unit, 2 = two
   void *out;               // bf16 C, fp32 X, or bf16 H
   // LM head
   const float *bias; float *part_m, *part_s; int32_t *part_i; int rows_padded; float *logits;
@@ -156,5 +163,13 @@ cudaError_t launch_attention_bf16(cudaStream_t st, const bf16 *q, const bf16 *kc
                                   const SeqMeta *meta, bf16 *out, int64_t q_stride, int64_t kv_row_stride,
                                   int64_t kv_seq_stride, int64_t out_stride, int n_slots, int max_q_rows,
                                   int H, int dh);
+
+
+// attention_tc.cu : head size 128 on tcgen05.  tq covers the packed query rows [rows, H*128], tk / tv the
+// key / value store as one matrix of rows (layer, sequence, position) x H*128; all with a box of 128 rows.
+bool attention_tc_supported(int dh, int64_t q_stride, int64_t kv_row_stride, int64_t out_stride);
+cudaError_t launch_attention_tc(cudaStream_t st, const TmaDesc &tq, const TmaDesc &tk, const TmaDesc &tv,
+                                const SeqMeta *meta, bf16 *out, int64_t out_stride, int kv_rows_per_seq,
+                                int kv_row_base, int n_slots, int max_q_rows, int H, int32_t *status);
 
 }  // namespace l2pd

@@ -12,8 +12,14 @@
 //   EPI_LMHEAD    per-row running (max, sum exp, argmax) over the vocabulary tile, written as one
 //                 record per (tile, row): the logits are never stored (Eq. 3-4 need only these).
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner and MMA issuer,
-// warps 2-5 = epilogue (warp w reads TMEM lanes 32*(w%4) .. +31).
+// Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner and MMA issuer, warp 2 = second MMA
+// issuer (two-slab units only), warps 3-6 (and 7-10 for the second slab) = epilogue; warp w reads
+// TMEM lanes 32*(w%4) .. +31.
+//
+// One thread can issue a tcgen05.mma (K = 16) only every ~132 cycles, whatever its N, while the
+// tensor pipe needs N/2 cycles for it: a single issuer keeps the pipe busy only for N = 256.
+// A unit of two row slabs has two independent accumulators, each fed by its own issuing thread,
+// so the pipe sees two instructions per 132 cycles and stays busy for any N >= 132.
 #include <math.h>
 #include <stdio.h>
 
@@ -34,7 +40,8 @@ constexpr int SMEM_BUDGET = 227 * 1024;
 
 struct KParams {
   int M, N, K, tile_n, n_stages, b_stage_bytes;
-  int m_tiles, n_tiles, k_splits;   // m_tiles counts 128-row tiles (CG = 1) or 256-row pair tiles (CG = 2)
+  int slabs, a_stage_bytes;         // row slabs (of 128 * CG rows) one unit covers: 1, or 2 = accumulators not double-buffered
+  int m_tiles, n_tiles, k_splits;   // m_tiles counts row tiles of 128 * CG * slabs rows
   void *out;
   const float *bias;
   float *part_m, *part_s;
@@ -48,94 +55,117 @@ __device__ __forceinline__ void fail(int32_t *status, int code) {
   if (status) atomicCAS(status, 0, code);
 }
 
+// Emitters: what the epilogue does with 16 consecutive accumulator columns of one row.
+// `valid` = columns left in the row from the first of the 16 (the row length is a multiple of 8).
+__device__ __forceinline__ void emit_store16(bf16 *dst, const uint32_t *v, int valid) {   // 16 fp32 -> 16 bf16, 32 bytes
+#pragma unroll
+  for (int hseg = 0; hseg < 2; ++hseg) {
+    if (hseg * 8 >= valid) break;
+    uint4 pk;
+    uint32_t *pw = reinterpret_cast<uint32_t *>(&pk);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(v[hseg * 8 + 2 * i]), __uint_as_float(v[hseg * 8 + 2 * i + 1]));
+      pw[i] = *reinterpret_cast<uint32_t *>(&t);
+    }
+    *reinterpret_cast<uint4 *>(dst + hseg * 8) = pk;
+  }
+}
+__device__ __forceinline__ void emit_residual16(float *px, const uint32_t *v, bool atomic, int valid) {
+#pragma unroll
+  for (int g = 0; g < 4; ++g) {
+    if (g * 4 >= valid) break;
+    if (atomic) {
+      ptx::red_add_v4(px + 4 * g, __uint_as_float(v[4 * g + 0]), __uint_as_float(v[4 * g + 1]),
+                      __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3]));
+    } else {
+      float4 x = *reinterpret_cast<float4 *>(px + 4 * g);
+      x.x += __uint_as_float(v[4 * g + 0]);
+      x.y += __uint_as_float(v[4 * g + 1]);
+      x.z += __uint_as_float(v[4 * g + 2]);
+      x.w += __uint_as_float(v[4 * g + 3]);
+      *reinterpret_cast<float4 *>(px + 4 * g) = x;
+    }
+  }
+}
+__device__ __forceinline__ void emit_swiglu16(bf16 *dst, const uint32_t *g, const uint32_t *u, int valid) {
+#pragma unroll
+  for (int hseg = 0; hseg < 2; ++hseg) {
+    if (hseg * 8 >= valid) break;
+    uint4 pk;
+    uint32_t *pw = reinterpret_cast<uint32_t *>(&pk);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float g0 = __uint_as_float(g[hseg * 8 + 2 * i]), g1 = __uint_as_float(g[hseg * 8 + 2 * i + 1]);
+      const float u0 = __uint_as_float(u[hseg * 8 + 2 * i]), u1 = __uint_as_float(u[hseg * 8 + 2 * i + 1]);
+      __nv_bfloat162 t = __floats2bfloat162_rn(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
+      pw[i] = *reinterpret_cast<uint32_t *>(&t);
+    }
+    *reinterpret_cast<uint4 *>(dst + hseg * 8) = pk;
+  }
+}
+
 // Drains one 128-row x tile_n accumulator from tensor memory (this warp's 32 lanes) and applies the
-// epilogue.  `atomic` (split-K residual): the partial sum is added to X with a vector reduction.
+// epilogue with per-thread stores (a thread owns one row).  The loads run one step ahead of the
+// arithmetic and stores: while chunk c is converted and written, chunk c + 1 is in flight
+// (tcgen05.wait::ld covers every load issued so far).
+// `atomic` (split-K residual): the partial sum is added to X with a vector reduction.
 template <int EPI>
 __device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int row, int nt, bool atomic) {
   const bool row_ok = row < p.M;
   const int half_n = p.tile_n >> 1;
-  uint32_t v[16];
-  if (EPI == EPI_STORE) {
-    bf16 *C = reinterpret_cast<bf16 *>(p.out);
-    const int n0 = nt * p.tile_n;
-    for (int c = 0; c < p.tile_n; c += 16) {
-      ptx::tmem_ld_x16(taddr + c, v);
-      ptx::tmem_ld_wait();
-      if (row_ok) {
+  if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+    // 32 columns per step (tile_n is a multiple of 16: the last step may hold 16)
+    const int n0 = nt * p.tile_n, n = p.tile_n;
+    uint32_t va[32], vb[32];
+    auto load = [&](uint32_t *v, int c) {
+      if (n - c >= 32) ptx::tmem_ld_x32(taddr + c, v);
+      else ptx::tmem_ld_x16(taddr + c, v);
+    };
+    auto emit = [&](const uint32_t *v, int c) {
+      if (!row_ok) return;
 #pragma unroll
-        for (int hseg = 0; hseg < 2; ++hseg) {
-          const int col = n0 + c + hseg * 8;
-          if (col < p.N) {
-            uint4 pk;
-            uint32_t *pw = reinterpret_cast<uint32_t *>(&pk);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(v[hseg * 8 + 2 * i]),
-                                                       __uint_as_float(v[hseg * 8 + 2 * i + 1]));
-              pw[i] = *reinterpret_cast<uint32_t *>(&t);
-            }
-            *reinterpret_cast<uint4 *>(C + (int64_t)row * p.N + col) = pk;
-          }
+      for (int h16 = 0; h16 < 2; ++h16) {
+        const int col = n0 + c + 16 * h16;
+        if (c + 16 * h16 < n && col < p.N) {
+          if (EPI == EPI_STORE) emit_store16(reinterpret_cast<bf16 *>(p.out) + (int64_t)row * p.N + col, v + 16 * h16, p.N - col);
+          else emit_residual16(reinterpret_cast<float *>(p.out) + (int64_t)row * p.N + col, v + 16 * h16, atomic, p.N - col);
         }
       }
-    }
-  } else if (EPI == EPI_RESIDUAL) {
-    float *X = reinterpret_cast<float *>(p.out);
-    const int n0 = nt * p.tile_n;
-    for (int c = 0; c < p.tile_n; c += 16) {
-      ptx::tmem_ld_x16(taddr + c, v);
+    };
+    load(va, 0);
+    for (int c = 0; c < n; c += 64) {
       ptx::tmem_ld_wait();
-      if (row_ok) {
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-          const int col = n0 + c + g * 4;
-          if (col < p.N) {
-            float *px = X + (int64_t)row * p.N + col;
-            if (atomic) {
-              ptx::red_add_v4(px, __uint_as_float(v[4 * g + 0]), __uint_as_float(v[4 * g + 1]),
-                              __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3]));
-            } else {
-              float4 x = *reinterpret_cast<float4 *>(px);
-              x.x += __uint_as_float(v[4 * g + 0]);
-              x.y += __uint_as_float(v[4 * g + 1]);
-              x.z += __uint_as_float(v[4 * g + 2]);
-              x.w += __uint_as_float(v[4 * g + 3]);
-              *reinterpret_cast<float4 *>(px) = x;
-            }
-          }
-        }
-      }
+      if (c + 32 < n) load(vb, c + 32);
+      emit(va, c);
+      if (c + 32 >= n) break;
+      ptx::tmem_ld_wait();
+      if (c + 64 < n) load(va, c + 64);
+      emit(vb, c + 32);
     }
   } else if (EPI == EPI_SWIGLU) {
     bf16 *H = reinterpret_cast<bf16 *>(p.out);
     const int n0 = nt * half_n;
-    uint32_t u[16];
-    for (int c = 0; c < half_n; c += 16) {
-      ptx::tmem_ld_x16(taddr + c, v);
+    uint32_t ga[16], ua[16], gb[16], ub[16];
+    auto load = [&](uint32_t *g, uint32_t *u, int c) {
+      ptx::tmem_ld_x16(taddr + c, g);
       ptx::tmem_ld_x16(taddr + half_n + c, u);
+    };
+    auto emit = [&](const uint32_t *g, const uint32_t *u, int c) {
+      if (row_ok && n0 + c < p.N) emit_swiglu16(H + (int64_t)row * p.N + n0 + c, g, u, p.N - n0 - c);
+    };
+    load(ga, ua, 0);
+    for (int c = 0; c < half_n; c += 32) {
       ptx::tmem_ld_wait();
-      if (row_ok) {
-#pragma unroll
-        for (int hseg = 0; hseg < 2; ++hseg) {
-          const int col = n0 + c + hseg * 8;
-          if (col < p.N) {
-            uint4 pk;
-            uint32_t *pw = reinterpret_cast<uint32_t *>(&pk);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              float g0 = __uint_as_float(v[hseg * 8 + 2 * i]), g1 = __uint_as_float(v[hseg * 8 + 2 * i + 1]);
-              float u0 = __uint_as_float(u[hseg * 8 + 2 * i]), u1 = __uint_as_float(u[hseg * 8 + 2 * i + 1]);
-              float h0 = g0 / (1.0f + __expf(-g0)) * u0;
-              float h1 = g1 / (1.0f + __expf(-g1)) * u1;
-              __nv_bfloat162 t = __floats2bfloat162_rn(h0, h1);
-              pw[i] = *reinterpret_cast<uint32_t *>(&t);
-            }
-            *reinterpret_cast<uint4 *>(H + (int64_t)row * p.N + col) = pk;
-          }
-        }
-      }
+      if (c + 16 < half_n) load(gb, ub, c + 16);
+      emit(ga, ua, c);
+      if (c + 16 >= half_n) break;
+      ptx::tmem_ld_wait();
+      if (c + 32 < half_n) load(ga, ua, c + 32);
+      emit(gb, ub, c + 16);
     }
   } else {  // EPI_LMHEAD
+    uint32_t v[16];
     const float L2E = 1.4426950408889634f;
     const int n0 = nt * p.tile_n;
     float m_run = -INFINITY, s_run = 0.f;
@@ -203,7 +233,10 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
 
   const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sA = base;
-  const uint32_t sB = base + p.n_stages * A_STAGE_BYTES;
+  const uint32_t sB = base + p.n_stages * p.a_stage_bytes;
+  const int slabs = p.slabs;
+  const int nbuf = slabs == 1 ? 2 : 1;            // accumulator buffers a unit can alternate between
+  const int unit_rows = TILE_M * CG * slabs;
   const uint32_t bar0 = ptx::smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
   auto empty_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };
@@ -211,8 +244,8 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
   auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * MAX_STAGES + 2 + b); };
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.n_stages; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), 1); }
-    for (int b = 0; b < 2; ++b) { ptx::mbar_init(tfull_bar(b), 1); ptx::mbar_init(tempty_bar(b), 4 * CG); }
+    for (int s = 0; s < p.n_stages; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), slabs); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(tfull_bar(b), slabs); ptx::mbar_init(tempty_bar(b), 4 * CG * slabs); }
     *abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
@@ -256,20 +289,21 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
       const uint64_t pol_w = ptx::policy_evict_first();   // weights are read once per step
       const uint64_t pol_a = ptx::policy_evict_last();    // activations are re-read by every column tile
       const uint32_t b_bytes = (CG == 2) ? (uint32_t)half_n * 128u : (uint32_t)p.tile_n * 128u;
-      const uint32_t tx = CG * (A_STAGE_BYTES + b_bytes);
+      const uint32_t tx = CG * (p.a_stage_bytes + b_bytes);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
       for (int u = group; u < num_units && ok; u += n_groups) {
         int mt, nt, kb0, kb1;
         decode(u, mt, nt, kb0, kb1);
-        const int m0 = mt * (TILE_M * CG) + (int)rank * TILE_M;
+        const int m0 = mt * unit_rows + (int)rank * TILE_M;
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
-          const uint32_t dstA = sA + stage * A_STAGE_BYTES, dstB = sB + stage * p.b_stage_bytes;
+          const uint32_t dstA = sA + stage * p.a_stage_bytes, dstB = sB + stage * p.b_stage_bytes;
           if (CG == 1) {
             ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
-            ptx::tma_load_2d_hint(dstA, tmA, full_bar(stage), kb * TILE_K, m0, pol_a);
+            for (int sl = 0; sl < slabs; ++sl)
+              ptx::tma_load_2d_hint(dstA + sl * A_STAGE_BYTES, tmA, full_bar(stage), kb * TILE_K, m0 + sl * TILE_M, pol_a);
             if (EPI == EPI_SWIGLU) {
               ptx::tma_load_2d_hint(dstB, tmB, full_bar(stage), kb * TILE_K, nt * half_n, pol_w);
               ptx::tma_load_2d_hint(dstB + half_n * 128, tmB2, full_bar(stage), kb * TILE_K, nt * half_n, pol_w);
@@ -279,7 +313,8 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
           } else {
             if (leader) ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
             const uint32_t lead_full = ptx::mapa(full_bar(stage), 0);
-            ptx::tma_load_2d_pair_hint(dstA, tmA, lead_full, kb * TILE_K, m0, pol_a);
+            for (int sl = 0; sl < slabs; ++sl)
+              ptx::tma_load_2d_pair_hint(dstA + sl * A_STAGE_BYTES, tmA, lead_full, kb * TILE_K, m0 + sl * TILE_M * CG, pol_a);
             if (EPI == EPI_SWIGLU)
               ptx::tma_load_2d_pair_hint(dstB, leader ? tmB : tmB2, lead_full, kb * TILE_K, nt * half_n, pol_w);
             else
@@ -290,9 +325,12 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
       }
       if (!ok) *abort_flag = 1;
     }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer (leader CTA only when paired)
-    if (lane == 0 && leader) {
+  } else if (warp == 1 || warp == 2) {
+    // ------------------------------------------------------------------ MMA issuers (leader CTA only when paired)
+    // warp 1 feeds slab 0, warp 2 slab 1: each slab has its own accumulator columns, so the two
+    // instruction streams need no ordering between them; both count on the stage's `empty` barrier.
+    const int sl = warp - 1;
+    if (lane == 0 && leader && sl < slabs) {
       const uint32_t idesc = ptx::idesc_bf16(TILE_M * CG, (uint32_t)p.tile_n);
       int stage = 0;
       uint32_t phase = 0;
@@ -301,15 +339,15 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
       for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
         int mt, nt, kb0, kb1;
         decode(u, mt, nt, kb0, kb1);
-        const int ab = lt & 1;
-        const uint32_t aphase = (lt >> 1) & 1;
+        const int ab = lt % nbuf;
+        const uint32_t aphase = (lt / nbuf) & 1;
         if (!ptx::mbar_wait(tempty_bar(ab), aphase ^ 1u)) { fail(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
         ptx::tc_fence_after_sync();
-        const uint32_t d_tmem = tmem_base + ab * ACC_COLS;
+        const uint32_t d_tmem = tmem_base + (ab + sl) * ACC_COLS;   // slab sl of a two-slab unit: column sl * ACC_COLS
         for (int kb = kb0; kb < kb1; ++kb) {
           if (!ptx::mbar_wait(full_bar(stage), phase)) { fail(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
           ptx::tc_fence_after_sync();
-          const uint64_t a_desc = ptx::smem_desc_sw128(sA + stage * A_STAGE_BYTES);
+          const uint64_t a_desc = ptx::smem_desc_sw128(sA + stage * p.a_stage_bytes + sl * A_STAGE_BYTES);
           const uint64_t b_desc = ptx::smem_desc_sw128(sB + stage * p.b_stage_bytes);
 #pragma unroll
           for (int k = 0; k < TILE_K / 16; ++k) {   // 16 bf16 = 32 bytes per MMA: descriptor address += 2
@@ -330,18 +368,19 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
     }
   } else {
     // ------------------------------------------------------------------ epilogue
-    const int q = warp & 3;
+    // warps 3-6 drain slab 0, warps 7-10 (two-slab units only) slab 1; warp w may touch TMEM lanes 32 (w % 4) ..
+    const int q = warp & 3, sl = (warp - 3) >> 2;
     int lt = 0;
     bool ok = true;
     for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
       int mt, nt, kb0, kb1;
       decode(u, mt, nt, kb0, kb1);
-      const int ab = lt & 1;
-      const uint32_t aphase = (lt >> 1) & 1;
+      const int ab = lt % nbuf;
+      const uint32_t aphase = (lt / nbuf) & 1;
       if (!ptx::mbar_wait(tfull_bar(ab), aphase)) { fail(p.status, DEV_TIMEOUT_EPILOGUE); ok = false; break; }
       ptx::tc_fence_after_sync();
-      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + ab * ACC_COLS;
-      const int row = mt * (TILE_M * CG) + (int)rank * TILE_M + q * 32 + lane;
+      const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (ab + sl) * ACC_COLS;
+      const int row = mt * unit_rows + sl * (TILE_M * CG) + (int)rank * TILE_M + q * 32 + lane;
       drain_tile<EPI>(p, taddr, row, nt, p.k_splits > 1);
       ptx::tc_fence_before_sync();
       __syncwarp();
@@ -372,7 +411,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
 }
 
 template <int EPI>
-__global__ void __launch_bounds__(192, 1)
+__global__ void __launch_bounds__(352, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmB2, const KParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -383,7 +422,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 }
 
 template <int EPI>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(192, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(352, 1)
 gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const __grid_constant__ CUtensorMap tmB2, const KParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -441,11 +480,18 @@ __global__ void merge_partials_kernel(const float *part_m, const float *part_s, 
 }  // namespace
 
 l2pd_status make_tma_2d_bf16(TmaDesc *out, const void *ptr, int64_t rows, int64_t cols, int box_rows) {
+  return make_tma_2d_bf16_strided(out, ptr, rows, cols, cols, box_rows);
+}
+
+l2pd_status make_tma_2d_bf16_strided(TmaDesc *out, const void *ptr, int64_t rows, int64_t cols, int64_t row_stride,
+                                     int box_rows) {
   EncodeTiledFn fn = get_encode_fn();
   if (!fn) return L2PD_ERR_CUDA;
-  if ((reinterpret_cast<uintptr_t>(ptr) & 15) || (cols % 8) || box_rows < 1 || box_rows > 256) return L2PD_ERR_SHAPE;
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15) || (cols % 8) || (row_stride % 8) || row_stride < cols || box_rows < 1 ||
+      box_rows > 256)
+    return L2PD_ERR_SHAPE;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint64_t strides[1] = {(cuuint64_t)row_stride * 2};
   cuuint32_t box[2] = {(cuuint32_t)TILE_K, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUresult r = fn(&out->map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box,
@@ -454,36 +500,45 @@ l2pd_status make_tma_2d_bf16(TmaDesc *out, const void *ptr, int64_t rows, int64_
   return r == CUDA_SUCCESS ? L2PD_OK : L2PD_ERR_CUDA;
 }
 
-// Modelled cycles of one GEMM for a tile width / K split: per 64-deep k-block a CTA needs
-// max(2 * tile_n MMA cycles, bytes it must take in / ~70 B per cycle), plus a fixed fill/drain part
-// per unit, times the number of waves over the SMs (or SM pairs).
-static double plan_cost(int M, int N, int K, int num_sms, int cg, int unit_n, int tile_n, int ks) {
+// Modelled cycles of one GEMM for a tile width / K split / slab count.  Per 64-deep k-block a CTA
+// needs the largest of: the tensor pipe's 2 * tile_n cycles per slab; the ~620 cycles one thread
+// takes to issue its four MMAs and the stage hand-over; the bytes it must take in at INGEST bytes
+// per cycle.  A unit adds a fixed fill part and, when its accumulators are not double-buffered
+// (two slabs), the drain of the accumulator; times the number of waves over the SMs (or SM pairs).
+static double plan_cost(int M, int N, int K, int num_sms, int cg, int slabs, int unit_n, int tile_n, int ks) {
+  const double INGEST = cg == 2 ? 58.0 : 68.0;   // measured: bytes per cycle an SM takes in from L2 through TMA
   const int groups = num_sms / cg;
-  const int m_tiles = ceil_div(M, TILE_M * cg);
+  const int m_tiles = ceil_div(M, TILE_M * cg * slabs);
   const int n_tiles = ceil_div(N, unit_n);
   const int units = m_tiles * n_tiles * ks;
   const int waves = ceil_div(units, groups);
   const int kb = ceil_div(ceil_div(K, TILE_K), ks);
-  const double bytes = A_STAGE_BYTES + 128.0 * tile_n / cg;
-  const double per_kb = fmax(2.0 * tile_n, bytes / 70.0);
-  return waves * (kb * per_kb + 1500.0 + 4.0 * tile_n + (ks > 1 ? 2.0 * tile_n : 0.0));
+  const double bytes = (double)slabs * A_STAGE_BYTES + 128.0 * tile_n / cg;
+  const double per_kb = fmax(fmax(2.0 * tile_n * slabs, 620.0), bytes / INGEST);
+  const double drain = 14.0 * tile_n + (ks > 1 ? 4.0 * tile_n : 0.0);   // cycles to empty one 128 x tile_n accumulator
+  const double exposed = slabs == 2 ? drain : 0.3 * drain;
+  return waves * (kb * per_kb + 2500.0 + exposed) + (slabs == 2 ? 0.0 : 0.7 * drain);
 }
 
 GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n) {
-  GemmPlan best{1, 256, 1};
+  GemmPlan best{1, 256, 1, 1};
   double best_cost = 1e300;
   const bool swiglu = epi == EPI_SWIGLU;
   const int step = swiglu ? 32 : 16;
   for (int cg = 1; cg <= 2; ++cg) {
     if (cg == 2 && (M <= TILE_M || epi == EPI_LMHEAD || num_sms < 2)) continue;
-    for (int tn = 256; tn >= 64; tn -= step) {
-      if (force_tile_n && tn != force_tile_n) continue;
-      const int unit_n = swiglu ? tn / 2 : tn;
-      const int max_ks = (epi == EPI_RESIDUAL) ? 4 : 1;
-      for (int ks = 1; ks <= max_ks; ++ks) {
-        if (ceil_div(K, TILE_K) < 8 * ks) break;
-        const double c = plan_cost(M, N, K, num_sms, cg, unit_n, tn, ks);
-        if (c < best_cost - 1e-9) { best_cost = c; best = GemmPlan{cg, tn, ks}; }
+    for (int slabs = 1; slabs <= 2; ++slabs) {
+      // a second slab: the weight tile is read once for twice the rows, and a second thread issues MMAs
+      if (slabs == 2 && (cg == 1 || epi == EPI_LMHEAD || M <= TILE_M * cg)) continue;
+      for (int tn = 256; tn >= 64; tn -= step) {
+        if (force_tile_n && tn != force_tile_n) continue;
+        const int unit_n = swiglu ? tn / 2 : tn;
+        const int max_ks = (epi == EPI_RESIDUAL) ? 4 : 1;
+        for (int ks = 1; ks <= max_ks; ++ks) {
+          if (ceil_div(K, TILE_K) < 8 * ks) break;
+          const double c = plan_cost(M, N, K, num_sms, cg, slabs, unit_n, tn, ks);
+          if (c < best_cost - 1e-9) { best_cost = c; best = GemmPlan{cg, tn, ks, slabs}; }
+        }
       }
     }
   }
@@ -507,12 +562,15 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
   KParams p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.tile_n = g.tile_n;
   p.b_stage_bytes = g.tile_n * 128 / cg;
-  const int stage_bytes = A_STAGE_BYTES + p.b_stage_bytes;
+  p.slabs = g.slabs == 2 ? 2 : 1;
+  if (p.slabs == 2 && g.epi == EPI_LMHEAD) return cudaErrorInvalidValue;
+  p.a_stage_bytes = p.slabs * A_STAGE_BYTES;
+  const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
   int stages = (SMEM_BUDGET - 2048) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) return cudaErrorInvalidValue;
   p.n_stages = stages;
-  p.m_tiles = ceil_div(g.M, TILE_M * cg);
+  p.m_tiles = ceil_div(g.M, TILE_M * cg * p.slabs);
   const int n_per_tile = (g.epi == EPI_SWIGLU) ? g.tile_n / 2 : g.tile_n;
   p.n_tiles = ceil_div(g.N, n_per_tile);
   p.k_splits = ks;
@@ -528,7 +586,7 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
 #define L2PD_LAUNCH(KERNEL, EPI)                                                                      \
   e = cudaFuncSetAttribute(KERNEL<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET - 1024); \
   if (e != cudaSuccess) return e;                                                                    \
-  e = launch_kernel(KERNEL<EPI>, dim3(grid), dim3(192), smem, st, g.a->map, g.b->map, b2, p);                \
+  e = launch_kernel(KERNEL<EPI>, dim3(grid), dim3(96 + 128 * p.slabs), smem, st, g.a->map, g.b->map, b2, p);                \
   if (e != cudaSuccess) return e;
   if (cg == 1) {
     switch (g.epi) {

@@ -36,6 +36,7 @@ def main():
     ap.add_argument("--ff", type=int, default=12288)
     ap.add_argument("--vocab", type=int, default=126464)
     ap.add_argument("--heads", type=int, default=32)
+    ap.add_argument("--impl", type=int, default=0, help="attn: 0 = tcgen05 kernel, 1 = mma.sync kernel")
     ap.add_argument("--ring", type=int, default=0, help="number of weight buffers to rotate through (0 = enough to exceed L2)")
     a = ap.parse_args()
     dev = "cuda:0"
@@ -87,12 +88,15 @@ def main():
         q, k, v = rnd(T, d, 1.0), rnd(T, d, 1.0), rnd(T, d, 1.0)
         out = torch.empty(T, d, dtype=torch.bfloat16, device=dev)
         run = lambda i: b._check(b.lib.l2pd_attention_bf16(b._stream(), q.data_ptr(), k.data_ptr(), v.data_ptr(),
-                                                           out.data_ptr(), T, T, H, dh, d, d, d))
+                                                           out.data_ptr(), T, T, H, dh, d, d, d, a.impl, 0))
         flops, byts = 4.0 * T * T * d, 2.0 * 4 * T * d
 
     for i in range(a.warmup):
         run(i)
     torch.cuda.synchronize()
+    # a device wait that ran out leaves its code in the library's status word: the checked call below reports it
+    probe = torch.zeros(16, 64, dtype=torch.bfloat16, device=dev)
+    b.gemm_bf16(probe, torch.zeros(64, 64, dtype=torch.bfloat16, device=dev))
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     tot = 0.0
     for i in range(a.iters):

@@ -1,0 +1,119 @@
+"""Full Learn2PD decodes at the LLaDA-8B widths (d 4096, 32 heads x 128, SwiGLU 12288, vocab
+126464) with two layers, so that the oracle can follow them: the launch shapes of the decode
+configurations — single sequence with an EoT bias, a batch of 16 with drop-out, and the batch of
+8 with the prefix key/value cache — through the C ABI.
+
+On every step of every sequence the decision logic (filter, threshold, fallback commit, EoTP,
+block advance) is replayed in fp64 on the decoder's own confidences and must match bit for bit;
+on sampled (sequence, step) pairs — the first step, the first step served from the cache, the
+step after [EoT] was committed, every sixth step — the oracle's forward pass is run on the
+decoder's token state and logits, confidences, ids and decisions are compared within the bf16
+tolerances.
+"""
+from __future__ import annotations
+
+import os
+
+import numpy as np
+import pytest
+
+from oracle import l2pd_oracle as orc
+from paper_2509_25188_b200 import workloads as wl
+from tests.helpers import lockstep, oracle_model
+
+pytestmark = pytest.mark.gpu
+
+SHAPE = wl.thin(wl.LLADA_8B, 2)
+
+
+@pytest.fixture(scope="module")
+def thin8b():
+    import torch
+    from paper_2509_25188_b200 import binding
+    w = wl.make_weights(SHAPE, seed=0, final_norm_gain=wl.spread_gain(SHAPE), threads=os.cpu_count() or 8)
+    dev = {"tok_emb": binding.to_device(w["tok_emb"]), "lm_head": binding.to_device(w["lm_head"]),
+           "final_norm": w["final_norm"],
+           "layers": [{k: binding.to_device(v) for k, v in layer.items()} for layer in w["layers"]]}
+    yield w, dev
+    del dev
+    torch.cuda.empty_cache()
+
+
+def _run(thin8b, *, B, P, G, kv_cache, eot_bias, seed, sample, max_steps=None):
+    from paper_2509_25188_b200 import binding
+    w, dev = thin8b
+    s = 32
+    bias = wl.make_eot_bias(SHAPE, eot_bias) if eot_bias is not None else None
+    m = oracle_model(SHAPE, w, lm_head_bias=bias)
+    filt = wl.make_filter(s, 0.96, seed=0)
+    prompts = wl.make_prompts(B, P, SHAPE, seed=seed)
+    cfg = orc.DecodeConfig(block_len=s, kv_cache=kv_cache)
+    dec = binding.Decoder(SHAPE, dev, filt, block_len=s, max_batch=B, max_seq=P + G, kv_cache=kv_cache,
+                          lm_head_bias=bias)
+    # spread logits (std ~ 7): |d conf| <= 0.5 max|d logit|, see test_gpu_decode
+    st = lockstep(dec, m, filt, cfg, prompts, G, logit_rtol=2e-2, conf_atol=0.05, p_margin=0.3,
+                  oracle_when=sample, max_steps=max_steps)
+    # the same decode through l2pd_decode: identical tokens, lengths and step counts
+    toks, out_len, steps, total = dec.decode(prompts, G)
+    dec.close()
+    return st, toks, out_len, steps, total
+
+
+def test_single_sequence_decode_with_eot_bias(thin8b):
+    """Prompt 256 + generation 256, block 32, EoT logit biased so that EoTP can fire before the end."""
+    seen = {"eot": False}
+
+    def sample(i, k, state):
+        # first step, every sixth step, and the first step after [EoT] has been committed
+        if state.eot_pos >= 0 and not seen["eot"]:
+            seen["eot"] = True
+            return True
+        return k == 0 or k % 6 == 5
+
+    st, toks, out_len, steps, total = _run(thin8b, B=1, P=256, G=256, kv_cache=False, eot_bias=14.0, seed=11,
+                                           sample=sample)
+    assert st["oracle_steps"] >= 2 and st["replay_checked"] >= 0.9 * st["steps"]
+    assert st["max_logit_rel"] < 2e-2
+    final = st["states"][0]
+    assert np.array_equal(toks[0], final.tokens[256:]) and out_len[0] == final.L_eff - 256
+    assert steps[0] == st["seq_steps"][0] == total
+    assert 1 <= steps[0] <= 256                        # never more steps than masks
+    if out_len[0] < 256:                               # EoTP fired: the tail is [EoT] and no later block ran
+        assert (toks[0][out_len[0] - 1:] == SHAPE.eot_id).all()
+        assert steps[0] < 256
+
+
+def test_batch_of_16_with_drop_out(thin8b):
+    """Batch 16, prompt 512 + generation 512: sequences finish at different steps and leave the batch."""
+    def sample(i, k, state):
+        return i == 3 and k in (0, 4)
+
+    st, toks, out_len, steps, total = _run(thin8b, B=16, P=512, G=512, kv_cache=False, eot_bias=15.0, seed=21,
+                                           sample=sample)
+    assert st["oracle_steps"] >= 1
+    assert st["replay_checked"] >= 0.9 * sum(st["seq_steps"])
+    for i in range(16):
+        final = st["states"][i]
+        assert np.array_equal(toks[i], final.tokens[512:]) and out_len[i] == final.L_eff - 512
+        assert steps[i] == st["seq_steps"][i]
+    assert total == st["steps"]
+    # drop-out: the batch shrinks before the last step unless every sequence took the same number of steps
+    if len(set(steps.tolist())) > 1:
+        taking_part = [int((np.asarray(t["done"]) >= 0).sum()) for t in st["trace"]]
+        assert taking_part[0] == 16 and min(taking_part) < 16
+
+
+def test_batch_of_8_prefix_cache(thin8b):
+    """Batch 8, prompt 1024 + generation 1024 with the prefix key/value cache; the oracle follows
+    sequence 0 with the same caching rule on the first (full) step and the first cached step."""
+    def sample(i, k, state):
+        return i == 0 and k in (0, 1)
+
+    st, toks, out_len, steps, total = _run(thin8b, B=8, P=1024, G=1024, kv_cache=True, eot_bias=15.0, seed=31,
+                                           sample=sample)
+    assert st["oracle_steps"] == 2
+    assert st["replay_checked"] >= 0.9 * sum(st["seq_steps"])
+    for i in range(8):
+        final = st["states"][i]
+        assert np.array_equal(toks[i], final.tokens[1024:]) and out_len[i] == final.L_eff - 1024
+        assert steps[i] == st["seq_steps"][i]

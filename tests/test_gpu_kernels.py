@@ -49,6 +49,10 @@ GEMM_SHAPES = [
     (640, 2048, 256, 2112),  # pair: several tiles per pair
     (129, 256, 128, 2256),   # pair: second CTA holds a single live row
     (4000, 4608, 320, 0),    # many row tiles: automatic plan
+    (512, 1056, 512, 202176),  # two 256-row slabs per unit (accumulators not double-buffered), one unit per pair
+    (300, 528, 1032, 202176),  # two slabs: the second one mostly empty, N and K tails
+    (1100, 2048, 256, 202128), # two slabs: several units per pair, ragged last row tile
+    (512, 12288, 320, 202256), # two slabs, full-width accumulators (all 512 tensor-memory columns)
 ]
 
 
@@ -67,6 +71,8 @@ RESIDUAL_SHAPES = GEMM_SHAPES[:5] + [
     (300, 528, 4104, 31064),    # single CTA, three K slices, K tail in the last slice
     (512, 512, 12288, 0),       # automatic plan for a narrow, deep projection
     (512, 4096, 1024, 2240),    # pair, width 240
+    (512, 4096, 4096, 232176),  # two slabs + three K slices
+    (400, 1024, 12288, 222176), # two slabs + two K slices, ragged rows
 ]
 
 
@@ -85,7 +91,9 @@ def test_gemm_bf16_residual(M, N, K, tile_n):
 
 @pytest.mark.parametrize("M,F,K,tile_n", [(128, 128, 64, 0), (200, 336, 192, 0), (512, 1408, 512, 224),
                                           (77, 136, 72, 64), (640, 2048, 256, 96), (512, 1408, 512, 2224),
-                                          (200, 336, 192, 2064), (1000, 2048, 256, 2256)])
+                                          (200, 336, 192, 2064), (1000, 2048, 256, 2256),
+                                          (512, 1408, 512, 202160), (300, 2048, 256, 202256),
+                                          (512, 24576, 256, 0)])
 def test_gemm_bf16_swiglu(M, F, K, tile_n):
     b = _b()
     A = _bf16(3, 0, (M, K), 1.0)
@@ -140,14 +148,18 @@ def test_lm_head_ties_pick_lowest_id():
     assert np.abs(conf.cpu().numpy() - rc).max() < 1e-6
 
 
-@pytest.mark.parametrize("Tq,Tk,H,dh", [(64, 64, 2, 128), (100, 100, 3, 128), (37, 200, 2, 64), (512, 512, 4, 128),
-                                        (5, 1, 1, 64), (130, 1030, 2, 128)])
-def test_attention_bidirectional(Tq, Tk, H, dh):
+# impl 0 = tensor-memory (tcgen05) kernel for head size 128, 1 = warp-level (mma.sync) kernel
+@pytest.mark.parametrize("Tq,Tk,H,dh,impl", [(64, 64, 2, 128, 0), (100, 100, 3, 128, 0), (37, 200, 2, 64, 0),
+                                             (512, 512, 4, 128, 0), (5, 1, 1, 64, 0), (130, 1030, 2, 128, 0),
+                                             (1, 1, 1, 128, 0), (129, 128, 1, 128, 0), (128, 129, 2, 128, 0),
+                                             (300, 257, 3, 128, 0), (256, 2048, 2, 128, 0),
+                                             (64, 64, 2, 128, 1), (130, 1030, 2, 128, 1), (512, 512, 4, 128, 1)])
+def test_attention_bidirectional(Tq, Tk, H, dh, impl):
     b = _b()
     q = _bf16(5, 0, (Tq, H * dh), 1.0)
     k = _bf16(5, 1, (Tk, H * dh), 1.0)
     v = _bf16(5, 2, (Tk, H * dh), 1.0)
-    got = b.attention_bf16(b.to_device(q), b.to_device(k), b.to_device(v), H, dh).float().cpu().numpy()
+    got = b.attention_bf16(b.to_device(q), b.to_device(k), b.to_device(v), H, dh, impl).float().cpu().numpy()
     want = orc.attention(orc.widen(q).reshape(Tq, H, dh), orc.widen(k).reshape(Tk, H, dh),
                          orc.widen(v).reshape(Tk, H, dh)).reshape(Tq, H * dh)
     # probabilities are rounded to bf16 before the second product: 2^-9 relative on each weight
