@@ -56,6 +56,9 @@ struct l2pd_ctx {
 
   // TMA descriptors (bf16 path)
   TmaDesc ta_n, ta_att, ta_h, ta_nf, ta_q, t_kstore, t_vstore;
+  // output maps of the four projections (staged epilogue stores); re-encoded when rows or tile width change
+  TmaDesc tc_qkv, tc_o, tc_h, tc_down;
+  int tc_rows = -1, tcw_qkv = 0, tcw_o = 0, tcw_h = 0, tcw_down = 0;   // tile width encoded (0 = none, -w = not usable for w)
   std::vector<TmaDesc> tb_qkv, tb_o, tb_gate, tb_up, tb_down;
   TmaDesc tb_lm;
   GemmPlan pl_qkv{}, pl_o{}, pl_gu{}, pl_down{};
@@ -176,9 +179,9 @@ l2pd_status run_gemm_simt(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const 
 }
 
 l2pd_status run_gemm_tc(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const TmaDesc *a, const TmaDesc *b,
-                        const TmaDesc *b2, void *out, int M, int N, int K, const GemmPlan &pl) {
+                        const TmaDesc *b2, const TmaDesc *cm, void *out, int M, int N, int K, const GemmPlan &pl) {
   GemmArgs g{};
-  g.epi = epi; g.a = a; g.b = b; g.b2 = b2; g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.out = out;
+  g.epi = epi; g.a = a; g.b = b; g.b2 = b2; g.c = cm; g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.out = out;
   g.cta_group = pl.cta_group; g.k_splits = pl.k_splits; g.slabs = pl.slabs;
   g.status = c->d_status;
   CKLK(kind, launch_gemm_tcgen05(s, g, c->num_sms));
@@ -212,6 +215,21 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
       r = encode_weight_maps(c, c->tb_up, c->w_up, F, d, box); if (r) return r;
       c->box_gu = box;
     }
+    // output maps: rows = this step's row count (the TMA unit clips the rows beyond it)
+    auto out_map = [&](TmaDesc &m, int &w_have, void *ptr, bool fp32, int64_t N, int w) -> l2pd_status {
+      if ((w_have == w || w_have == -w) && c->tc_rows == T_rows) return L2PD_OK;
+      if (N < w) { w_have = -w; return L2PD_OK; }   // a tile wider than the row: direct stores
+      l2pd_status r = make_tma_out_3d(&m, ptr, fp32, T_rows, N, w);
+      if (r) return set_err(c, r, "output tensor map encode failed (N %lld tile %d)", (long long)N, w);
+      w_have = w;
+      return L2PD_OK;
+    };
+    if (c->tc_rows != T_rows) { c->tcw_qkv = c->tcw_o = c->tcw_h = c->tcw_down = 0; }
+    l2pd_status r = out_map(c->tc_qkv, c->tcw_qkv, c->qkv, false, 3 * hd, c->pl_qkv.tile_n); if (r) return r;
+    r = out_map(c->tc_o, c->tcw_o, c->x, true, d, c->pl_o.tile_n); if (r) return r;
+    r = out_map(c->tc_h, c->tcw_h, c->h, false, F, c->pl_gu.tile_n / 2); if (r) return r;
+    r = out_map(c->tc_down, c->tcw_down, c->x, true, d, c->pl_down.tile_n); if (r) return r;
+    c->tc_rows = T_rows;
   }
 
   CKLK(L2PD_K_OTHER, launch_build_row_map(s, c->d_meta, n_slots, c->d_row_slot));
@@ -223,7 +241,7 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     T *kc = (T *)c->kc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
     T *vc = (T *)c->vc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
     l2pd_status r;
-    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_QKV, EPI_STORE, &c->ta_n, &c->tb_qkv[l], nullptr, qkv, T_rows, 3 * hd, d, c->pl_qkv);
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_QKV, EPI_STORE, &c->ta_n, &c->tb_qkv[l], nullptr, c->tcw_qkv > 0 ? &c->tc_qkv : nullptr, qkv, T_rows, 3 * hd, d, c->pl_qkv);
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_QKV, EPI_STORE, n, c->wqkv[l], nullptr, qkv, nullptr, T_rows, 3 * hd, d);
     if (r) return r;
     CKLK(L2PD_K_ROPE, launch_rope_scatter<T>(s, qkv, c->d_meta, c->d_row_slot, c->cs_table, q, kc, vc, c->kv_seq_stride, T_rows, H, dh));
@@ -237,14 +255,14 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     } else {
       CKLK(L2PD_K_ATTENTION, launch_simt_attention<T>(s, q, kc, vc, c->d_meta, c->d_row_slot, att, c->kv_seq_stride, T_rows, H, dh, max_kv));
     }
-    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_O, EPI_RESIDUAL, &c->ta_att, &c->tb_o[l], nullptr, c->x, T_rows, d, hd, c->pl_o);
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_O, EPI_RESIDUAL, &c->ta_att, &c->tb_o[l], nullptr, c->tcw_o > 0 ? &c->tc_o : nullptr, c->x, T_rows, d, hd, c->pl_o);
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_O, EPI_RESIDUAL, att, c->wo[l], nullptr, c->x, nullptr, T_rows, d, hd);
     if (r) return r;
     CKLK(L2PD_K_RMSNORM, launch_rmsnorm<T>(s, c->x, c->norm2[l], f.rms_eps, n, T_rows, d));
-    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_GATE_UP, EPI_SWIGLU, &c->ta_n, &c->tb_gate[l], &c->tb_up[l], hbuf, T_rows, F, d, c->pl_gu);
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_GATE_UP, EPI_SWIGLU, &c->ta_n, &c->tb_gate[l], &c->tb_up[l], c->tcw_h > 0 ? &c->tc_h : nullptr, hbuf, T_rows, F, d, c->pl_gu);
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_GATE_UP, EPI_SWIGLU, n, c->w_gate[l], c->w_up[l], hbuf, nullptr, T_rows, F, d);
     if (r) return r;
-    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_DOWN, EPI_RESIDUAL, &c->ta_h, &c->tb_down[l], nullptr, c->x, T_rows, d, F, c->pl_down);
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_DOWN, EPI_RESIDUAL, &c->ta_h, &c->tb_down[l], nullptr, c->tcw_down > 0 ? &c->tc_down : nullptr, c->x, T_rows, d, F, c->pl_down);
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_DOWN, EPI_RESIDUAL, hbuf, c->w_down[l], nullptr, c->x, nullptr, T_rows, d, F);
     if (r) return r;
     if (c->cap)
@@ -667,7 +685,13 @@ static l2pd_status gemm_common(void *stream, int epi, const void *A, const void 
   r = make_tma_2d_bf16(&tb, W, N, K, box);
   if (r) return r;
   if (epi == EPI_SWIGLU) { r = make_tma_2d_bf16(&tb2, W2, N, K, box); if (r) return r; }
+  // L2PD_DIRECT_STORES=1: epilogue with per-thread stores instead of the staged TMA stores (for comparison)
+  static const bool direct = [] { const char *e = getenv("L2PD_DIRECT_STORES"); return e && e[0] == '1'; }();
+  TmaDesc tcm;
+  const int out_w = epi == EPI_SWIGLU ? pl.tile_n / 2 : pl.tile_n;
+  const bool staged = !direct && N >= out_w && make_tma_out_3d(&tcm, out, epi == EPI_RESIDUAL, M, N, out_w) == L2PD_OK;
   GemmArgs g{};
+  g.c = staged ? &tcm : nullptr;
   g.epi = epi; g.a = &ta; g.b = &tb; g.b2 = epi == EPI_SWIGLU ? &tb2 : nullptr;
   g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.cta_group = pl.cta_group; g.k_splits = pl.k_splits;
   g.slabs = pl.slabs;

@@ -236,7 +236,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       if (j >= 2 && !ptx::mbar_wait(bar(B_PVDONE + st), ph ^ 1u)) { ok = false; break; }
       ptx::tc_fence_after_sync();
       ptx::tmem_st_x32(tP + lane_base + st * 64 + hf * 32, r);
-      if (rescale && j > 0) {
+      // tensor-memory loads and stores are warp-wide instructions: if any row of the warp moves its
+      // reference maximum, the whole warp rewrites its rows of O (rows that keep theirs scale by 1)
+      if (__any_sync(0xffffffffu, rescale && j > 0)) {
         // bring this thread's 64 columns of O to the new reference maximum
         if (!ptx::mbar_wait(bar(B_PVDONE + (st ^ 1)), ((j - 1) >> 1) & 1)) { ok = false; break; }
         ptx::tc_fence_after_sync();

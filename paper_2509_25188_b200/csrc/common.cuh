@@ -133,6 +133,9 @@ l2pd_status make_tma_2d_bf16(TmaDesc *out, const void *ptr, int64_t rows, int64_
 // The same for rows that are `row_stride` elements apart (a multiple of 8).
 l2pd_status make_tma_2d_bf16_strided(TmaDesc *out, const void *ptr, int64_t rows, int64_t cols, int64_t row_stride,
                                      int box_rows);
+// Output of a GEMM as a 3-D tensor [rows][N / tile_w][tile_w] (bf16, or fp32 for the residual stream) with a
+// box of 32 rows x 128 bytes, for the epilogue's staged stores; tile_w = the output columns one tile covers.
+l2pd_status make_tma_out_3d(TmaDesc *out, void *ptr, bool fp32, int64_t rows, int64_t N, int tile_w);
 int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile);
 // How one GEMM is laid over the SMs: CTAs per tile (1, or 2 = a cta_group::2 pair on a 256-row tile),
 // tile width, K slices (residual epilogue only: slices add into X with vector reductions), and row
@@ -145,6 +148,7 @@ GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n);
 struct GemmArgs {
   int epi;                 // EPI_STORE, EPI_RESIDUAL, EPI_SWIGLU, or EPI_LMHEAD
   const TmaDesc *a, *b, *b2;
+  const TmaDesc *c;        // output map from make_tma_out_3d (rows = M, tile_w matching tile_n), or null: direct stores
   int M, N, K, tile_n;
   int cta_group, k_splits; // 0 / 1 = single CTA, no split
   int slabs;               // 0 / 1 = one row slab per unit, 2 = two

@@ -49,6 +49,9 @@ struct KParams {
   int rows_padded;
   float *logits;
   int32_t *status;
+  int out_tma;          // 1: the epilogue may stage its output in shared memory and store it through tmC
+  int out_full_tiles;   // column tiles that lie wholly inside the row (the others use direct stores)
+  int gate;             // 1: every unit's epilogue is staged; the producer keeps off the staging area meanwhile
 };
 
 __device__ __forceinline__ void fail(int32_t *status, int code) {
@@ -213,6 +216,118 @@ __device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int
   }
 }
 
+// The same through shared memory and TMA: a thread owns one accumulator row, so direct stores touch
+// 32 different lines per instruction; instead each warp lays 128 bytes of 32 rows into a swizzled
+// staging tile (4 KB) and one thread hands it to the TMA unit, which writes whole lines (bf16
+// outputs) or adds them into X in L2 (fp32 residual).  The output tensor map is 3-D
+// [rows][column tile][column in tile], so a box that runs past the tile's width is clipped there,
+// and rows beyond M are clipped by the map's row count.
+// The warp's STAGE_BUFS staging tiles lie over the A operands of the ring's last two stages and are
+// used in turn.  That memory is idle during a CTA's last unit; for earlier units (two-slab units,
+// whose drain is not overlapped anyway) the producer refills those two stages only after the
+// epilogue warps have reported the staging area free.
+constexpr int STAGE_BUFS = 2;
+template <int EPI>
+__device__ __forceinline__ void drain_tile_staged(const KParams &p, const CUtensorMap *tmC, uint32_t taddr, int row0,
+                                                  int nt, uint32_t stage0, int lane) {
+  const int half_n = p.tile_n >> 1;
+  const uint32_t sw = (uint32_t)(lane & 7);
+  int n_flush = 0;                       // staging tiles handed over so far; the current one is n_flush % STAGE_BUFS
+  uint32_t stage = stage0;
+  auto chunk_addr = [&](int ch) { return stage + lane * 128 + (((uint32_t)ch ^ sw) << 4); };
+  auto st16 = [&](uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+  };
+  auto flush = [&](int c0) {   // hand the staged 32 x 128-byte tile to the TMA unit
+    ptx::fence_proxy_async();
+    __syncwarp();
+    if (lane == 0) {
+      if (EPI == EPI_RESIDUAL) ptx::tma_reduce_add_3d(tmC, stage, c0, nt, row0);
+      else ptx::tma_store_3d(tmC, stage, c0, nt, row0);
+      ptx::bulk_commit();
+    }
+    ++n_flush;
+  };
+  auto reuse = [&]() {         // pick the next staging tile; the flush that used it STAGE_BUFS turns ago has read it
+    stage = stage0 + (uint32_t)(n_flush % STAGE_BUFS) * 4096u;
+    if (n_flush >= STAGE_BUFS) {
+      if (lane == 0) ptx::bulk_wait_read_n<STAGE_BUFS - 1>();
+      __syncwarp();
+    }
+  };
+  auto pack2 = [](uint32_t a, uint32_t b) {
+    __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(a), __uint_as_float(b));
+    return *reinterpret_cast<uint32_t *>(&t);
+  };
+  if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+    const int n = p.tile_n;
+    uint32_t va[32], vb[32];
+    auto load = [&](uint32_t *v, int c) {
+      if (n - c >= 32) ptx::tmem_ld_x32(taddr + c, v);
+      else ptx::tmem_ld_x16(taddr + c, v);
+    };
+    auto emit = [&](const uint32_t *v, int c) {   // 32 columns starting at c (the upper 16 may lie beyond the tile)
+      if (EPI == EPI_RESIDUAL) {
+        reuse();
+#pragma unroll
+        for (int ch = 0; ch < 8; ++ch) st16(chunk_addr(ch), v[4 * ch], v[4 * ch + 1], v[4 * ch + 2], v[4 * ch + 3]);
+        flush(c);
+      } else {
+        const int hb = (c >> 5) & 1;              // which 64-byte half of the 128-byte staging row
+        if (hb == 0) reuse();
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch)
+          st16(chunk_addr(hb * 4 + ch), pack2(v[8 * ch], v[8 * ch + 1]), pack2(v[8 * ch + 2], v[8 * ch + 3]),
+               pack2(v[8 * ch + 4], v[8 * ch + 5]), pack2(v[8 * ch + 6], v[8 * ch + 7]));
+        if (hb == 1 || c + 32 >= n) flush(c & ~63);
+      }
+    };
+    load(va, 0);
+    for (int c = 0; c < n; c += 64) {
+      ptx::tmem_ld_wait();
+      if (c + 32 < n) load(vb, c + 32);
+      emit(va, c);
+      if (c + 32 >= n) break;
+      ptx::tmem_ld_wait();
+      if (c + 64 < n) load(va, c + 64);
+      emit(vb, c + 32);
+    }
+  } else {   // EPI_SWIGLU: 16 gate + 16 up columns give 16 outputs = 32 bytes of the staging row
+    uint32_t ga[16], ua[16], gb[16], ub[16];
+    auto load = [&](uint32_t *g, uint32_t *u, int c) {
+      ptx::tmem_ld_x16(taddr + c, g);
+      ptx::tmem_ld_x16(taddr + half_n + c, u);
+    };
+    auto emit = [&](const uint32_t *g, const uint32_t *u, int c) {
+      const int qb = (c >> 4) & 3;                // which 32-byte quarter of the staging row
+      if (qb == 0) reuse();
+#pragma unroll
+      for (int hseg = 0; hseg < 2; ++hseg) {
+        uint32_t pw[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float g0 = __uint_as_float(g[hseg * 8 + 2 * i]), g1 = __uint_as_float(g[hseg * 8 + 2 * i + 1]);
+          const float u0 = __uint_as_float(u[hseg * 8 + 2 * i]), u1 = __uint_as_float(u[hseg * 8 + 2 * i + 1]);
+          __nv_bfloat162 t = __floats2bfloat162_rn(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
+          pw[i] = *reinterpret_cast<uint32_t *>(&t);
+        }
+        st16(chunk_addr(qb * 2 + hseg), pw[0], pw[1], pw[2], pw[3]);
+      }
+      if (qb == 3 || c + 16 >= half_n) flush(c & ~63);
+    };
+    load(ga, ua, 0);
+    for (int c = 0; c < half_n; c += 32) {
+      ptx::tmem_ld_wait();
+      if (c + 16 < half_n) load(gb, ub, c + 16);
+      emit(ga, ua, c);
+      if (c + 16 >= half_n) break;
+      ptx::tmem_ld_wait();
+      if (c + 32 < half_n) load(ga, ua, c + 32);
+      emit(gb, ub, c + 16);
+    }
+  }
+}
+
 // CG = 1: one CTA per 128 x tile_n output tile.
 // CG = 2: a cluster of two CTAs per 256 x tile_n tile (cta_group::2).  CTA r loads A rows
 //         [128 r, 128 r + 128) and the r-th half of the B tile (for SwiGLU: CTA 0 the gate rows,
@@ -223,7 +338,7 @@ __device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int
 //         release the accumulator on the leader's `tmem empty` barrier.
 template <int EPI, int CG>
 __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensorMap *tmB, const CUtensorMap *tmB2,
-                                          const KParams &p, uint8_t *smem_raw, uint64_t *bars, uint32_t *tmem_slot,
+                                          const CUtensorMap *tmC, const KParams &p, uint8_t *smem_raw, uint64_t *bars, uint32_t *tmem_slot,
                                           int *abort_flag) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;
@@ -234,6 +349,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
   const uint32_t base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sA = base;
   const uint32_t sB = base + p.n_stages * p.a_stage_bytes;
+  const uint32_t sOut = sA + (uint32_t)(p.n_stages - 2) * p.a_stage_bytes;   // output staging: see drain_tile_staged
   const int slabs = p.slabs;
   const int nbuf = slabs == 1 ? 2 : 1;            // accumulator buffers a unit can alternate between
   const int unit_rows = TILE_M * CG * slabs;
@@ -242,10 +358,12 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
   auto empty_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };
   auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * MAX_STAGES + b); };
   auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * MAX_STAGES + 2 + b); };
+  const uint32_t sfree_bar = bar0 + 8u * (2 * MAX_STAGES + 4);
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.n_stages; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), slabs); }
     for (int b = 0; b < 2; ++b) { ptx::mbar_init(tfull_bar(b), slabs); ptx::mbar_init(tempty_bar(b), 4 * CG * slabs); }
+    ptx::mbar_init(sfree_bar, 4 * slabs);
     *abort_flag = 0;
     ptx::fence_barrier_init();
     ptx::fence_proxy_async();
@@ -254,6 +372,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
     ptx::prefetch_tensormap(tmA);
     ptx::prefetch_tensormap(tmB);
     if (EPI == EPI_SWIGLU) ptx::prefetch_tensormap(tmB2);
+    if (EPI != EPI_LMHEAD && p.out_tma) ptx::prefetch_tensormap(tmC);
   }
   if (warp == 1) {
     if (CG == 2) { ptx::tmem_alloc_pair(ptx::smem_u32(tmem_slot), TMEM_COLS); ptx::tmem_relinquish_pair(); }
@@ -290,15 +409,19 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
       const uint64_t pol_a = ptx::policy_evict_last();    // activations are re-read by every column tile
       const uint32_t b_bytes = (CG == 2) ? (uint32_t)half_n * 128u : (uint32_t)p.tile_n * 128u;
       const uint32_t tx = CG * (p.a_stage_bytes + b_bytes);
-      int stage = 0;
-      uint32_t phase = 0;
+      // every unit starts at stage 0 (so the staging area is what a unit fills last); one phase bit per stage
+      uint32_t phases = 0;
+      int lt = 0;
       bool ok = true;
-      for (int u = group; u < num_units && ok; u += n_groups) {
+      for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
         int mt, nt, kb0, kb1;
         decode(u, mt, nt, kb0, kb1);
         const int m0 = mt * unit_rows + (int)rank * TILE_M;
+        int stage = 0;
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!ptx::mbar_wait(empty_bar(stage), phase ^ 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
+          if (p.gate && lt > 0 && kb - kb0 == p.n_stages - 2 &&
+              !ptx::mbar_wait(sfree_bar, (uint32_t)(lt - 1) & 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
+          if (!ptx::mbar_wait(empty_bar(stage), ((phases >> stage) & 1u) ^ 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
           const uint32_t dstA = sA + stage * p.a_stage_bytes, dstB = sB + stage * p.b_stage_bytes;
           if (CG == 1) {
             ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
@@ -320,7 +443,8 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
             else
               ptx::tma_load_2d_pair_hint(dstB, tmB, lead_full, kb * TILE_K, nt * p.tile_n + (int)rank * half_n, pol_w);
           }
-          if (++stage == p.n_stages) { stage = 0; phase ^= 1u; }
+          phases ^= 1u << stage;
+          if (++stage == p.n_stages) stage = 0;
         }
       }
       if (!ok) *abort_flag = 1;
@@ -332,8 +456,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
     const int sl = warp - 1;
     if (lane == 0 && leader && sl < slabs) {
       const uint32_t idesc = ptx::idesc_bf16(TILE_M * CG, (uint32_t)p.tile_n);
-      int stage = 0;
-      uint32_t phase = 0;
+      uint32_t phases = 0;
       int lt = 0;
       bool ok = true;
       for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
@@ -344,8 +467,9 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
         if (!ptx::mbar_wait(tempty_bar(ab), aphase ^ 1u)) { fail(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
         ptx::tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + (ab + sl) * ACC_COLS;   // slab sl of a two-slab unit: column sl * ACC_COLS
+        int stage = 0;
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!ptx::mbar_wait(full_bar(stage), phase)) { fail(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
+          if (!ptx::mbar_wait(full_bar(stage), (phases >> stage) & 1u)) { fail(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
           ptx::tc_fence_after_sync();
           const uint64_t a_desc = ptx::smem_desc_sw128(sA + stage * p.a_stage_bytes + sl * A_STAGE_BYTES);
           const uint64_t b_desc = ptx::smem_desc_sw128(sB + stage * p.b_stage_bytes);
@@ -357,7 +481,8 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
           }
           if (CG == 2) ptx::mma_commit_pair(empty_bar(stage), 3);
           else ptx::mma_commit(empty_bar(stage));
-          if (++stage == p.n_stages) { stage = 0; phase ^= 1u; }
+          phases ^= 1u << stage;
+          if (++stage == p.n_stages) stage = 0;
         }
         if (ok) {
           if (CG == 2) ptx::mma_commit_pair(tfull_bar(ab), 3);
@@ -380,16 +505,27 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
       if (!ptx::mbar_wait(tfull_bar(ab), aphase)) { fail(p.status, DEV_TIMEOUT_EPILOGUE); ok = false; break; }
       ptx::tc_fence_after_sync();
       const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (ab + sl) * ACC_COLS;
-      const int row = mt * unit_rows + sl * (TILE_M * CG) + (int)rank * TILE_M + q * 32 + lane;
-      drain_tile<EPI>(p, taddr, row, nt, p.k_splits > 1);
+      const int row0 = mt * unit_rows + sl * (TILE_M * CG) + (int)rank * TILE_M + q * 32;
+      // the staging area is idle in a CTA's last unit (every load consumed, every MMA complete, in both
+      // CTAs of a pair), and in earlier units when the producer is kept off it (p.gate)
+      const bool last_unit = u + n_groups >= num_units;
+      if (EPI != EPI_LMHEAD && p.out_tma && nt < p.out_full_tiles && (last_unit || p.gate))
+        drain_tile_staged<EPI>(p, tmC, taddr, row0, nt, sOut + (uint32_t)(warp - 3) * (4096u * STAGE_BUFS), lane);
+      else
+        drain_tile<EPI>(p, taddr, row0 + lane, nt, p.k_splits > 1);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) {
         if (CG == 2) ptx::mbar_arrive_cluster(ptx::mapa(tempty_bar(ab), 0));
         else ptx::mbar_arrive(tempty_bar(ab));
+        if (EPI != EPI_LMHEAD && p.gate && !last_unit) {
+          ptx::bulk_wait_read();           // the TMA unit has read this warp's staging tiles
+          ptx::mbar_arrive(sfree_bar);
+        }
       }
     }
     if (!ok) *abort_flag = 1;
+    if (EPI != EPI_LMHEAD && p.out_tma && lane == 0) ptx::bulk_wait_all();   // staged stores are complete before the CTA leaves
   }
 
   // ---------------------------------------------------------------------- teardown
@@ -413,23 +549,23 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
 template <int EPI>
 __global__ void __launch_bounds__(352, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const __grid_constant__ CUtensorMap tmB2, const KParams p) {
+                    const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmC, const KParams p) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
+  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 5];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  gemm_body<EPI, 1>(&tmA, &tmB, &tmB2, p, smem_raw, bars, &tmem_slot, &abort_flag);
+  gemm_body<EPI, 1>(&tmA, &tmB, &tmB2, &tmC, p, smem_raw, bars, &tmem_slot, &abort_flag);
 }
 
 template <int EPI>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(352, 1)
 gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                         const __grid_constant__ CUtensorMap tmB2, const KParams p) {
+                         const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmC, const KParams p) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 4];
+  __shared__ __align__(8) uint64_t bars[2 * MAX_STAGES + 5];
   __shared__ uint32_t tmem_slot;
   __shared__ int abort_flag;
-  gemm_body<EPI, 2>(&tmA, &tmB, &tmB2, p, smem_raw, bars, &tmem_slot, &abort_flag);
+  gemm_body<EPI, 2>(&tmA, &tmB, &tmB2, &tmC, p, smem_raw, bars, &tmem_slot, &abort_flag);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -497,6 +633,23 @@ l2pd_status make_tma_2d_bf16_strided(TmaDesc *out, const void *ptr, int64_t rows
   CUresult r = fn(&out->map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(ptr), dims, strides, box,
                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? L2PD_OK : L2PD_ERR_CUDA;
+}
+
+l2pd_status make_tma_out_3d(TmaDesc *out, void *ptr, bool fp32, int64_t rows, int64_t N, int tile_w) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return L2PD_ERR_CUDA;
+  const int es = fp32 ? 4 : 2;
+  const int64_t full = N / tile_w;
+  if ((reinterpret_cast<uintptr_t>(ptr) & 15) || ((N * es) % 16) || ((tile_w * es) % 16) || full < 1 || rows < 1)
+    return L2PD_ERR_SHAPE;
+  cuuint64_t dims[3] = {(cuuint64_t)tile_w, (cuuint64_t)full, (cuuint64_t)rows};
+  cuuint64_t strides[2] = {(cuuint64_t)tile_w * es, (cuuint64_t)N * es};
+  cuuint32_t box[3] = {(cuuint32_t)(128 / es), 1, 32};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(&out->map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, ptr, dims,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? L2PD_OK : L2PD_ERR_CUDA;
 }
 
@@ -572,6 +725,10 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
   p.n_stages = stages;
   p.m_tiles = ceil_div(g.M, TILE_M * cg * p.slabs);
   const int n_per_tile = (g.epi == EPI_SWIGLU) ? g.tile_n / 2 : g.tile_n;
+  // staged output: needs the output map and a staging area (the A part of the ring's last two stages)
+  p.out_tma = (g.c != nullptr && g.epi != EPI_LMHEAD && stages >= 3) ? 1 : 0;
+  p.out_full_tiles = p.out_tma ? g.N / n_per_tile : 0;
+  p.gate = (p.out_tma && p.slabs == 2 && stages >= 4) ? 1 : 0;
   p.n_tiles = ceil_div(g.N, n_per_tile);
   p.k_splits = ks;
   p.out = g.out; p.bias = g.bias; p.part_m = g.part_m; p.part_s = g.part_s; p.part_i = g.part_i;
@@ -582,11 +739,12 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
   const int grid = cg * (units < groups ? units : groups);
   const size_t smem = (size_t)stages * stage_bytes + 1024;
   const CUtensorMap &b2 = g.b2 ? g.b2->map : g.b->map;
+  const CUtensorMap &cm = p.out_tma ? g.c->map : g.a->map;
   cudaError_t e;
 #define L2PD_LAUNCH(KERNEL, EPI)                                                                      \
   e = cudaFuncSetAttribute(KERNEL<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET - 1024); \
   if (e != cudaSuccess) return e;                                                                    \
-  e = launch_kernel(KERNEL<EPI>, dim3(grid), dim3(96 + 128 * p.slabs), smem, st, g.a->map, g.b->map, b2, p);                \
+  e = launch_kernel(KERNEL<EPI>, dim3(grid), dim3(96 + 128 * p.slabs), smem, st, g.a->map, g.b->map, b2, cm, p);                \
   if (e != cudaSuccess) return e;
   if (cg == 1) {
     switch (g.epi) {

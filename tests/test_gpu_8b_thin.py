@@ -50,8 +50,8 @@ def _run(thin8b, *, B, P, G, kv_cache, eot_bias, seed, sample, max_steps=None):
     cfg = orc.DecodeConfig(block_len=s, kv_cache=kv_cache)
     dec = binding.Decoder(SHAPE, dev, filt, block_len=s, max_batch=B, max_seq=P + G, kv_cache=kv_cache,
                           lm_head_bias=bias)
-    # spread logits (std ~ 7): |d conf| <= 0.5 max|d logit|, see test_gpu_decode
-    st = lockstep(dec, m, filt, cfg, prompts, G, logit_rtol=2e-2, conf_atol=0.05, p_margin=0.3,
+    # spread logits (row maxima ~32): |d conf| <= 0.5 max|d logit|, and a logit error of 6e-3 of the row maximum allows 0.1
+    st = lockstep(dec, m, filt, cfg, prompts, G, logit_rtol=2e-2, conf_atol=0.1, p_margin=0.3,
                   oracle_when=sample, max_steps=max_steps)
     # the same decode through l2pd_decode: identical tokens, lengths and step counts
     toks, out_len, steps, total = dec.decode(prompts, G)

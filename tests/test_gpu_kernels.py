@@ -167,6 +167,27 @@ def test_attention_bidirectional(Tq, Tk, H, dh, impl):
     assert np.sqrt(((got - want) ** 2).mean()) < 4e-3
 
 
+@pytest.mark.parametrize("impl", [0, 1])
+def test_attention_scores_that_grow_along_the_keys(impl):
+    """Later keys score far higher than earlier ones for some query rows and not for others, so the
+    running row maximum jumps by many powers of two between key tiles in part of each warp only:
+    exercises the rescaling of the partial output (for the tensor-memory kernel, the lazy one)."""
+    b = _b()
+    Tq, Tk, H, dh = 200, 640, 2, 128
+    rng = np.random.default_rng(7)
+    q = np.abs(rng.standard_normal((Tq, H * dh))).astype(np.float32)
+    q[::3] *= 0.01                                   # every third row: nearly flat scores
+    k = np.abs(rng.standard_normal((Tk, H * dh))).astype(np.float32)
+    k *= (0.05 + 2.0 * np.arange(Tk)[:, None] / Tk)  # key norm grows with the key index
+    v = rng.standard_normal((Tk, H * dh)).astype(np.float32)
+    qb, kb, vb = (wl.f32_to_bf16_bits(a) for a in (q, k, v))
+    got = b.attention_bf16(b.to_device(qb), b.to_device(kb), b.to_device(vb), H, dh, impl).float().cpu().numpy()
+    want = orc.attention(orc.widen(qb).reshape(Tq, H, dh), orc.widen(kb).reshape(Tk, H, dh),
+                         orc.widen(vb).reshape(Tk, H, dh)).reshape(Tq, H * dh)
+    assert np.abs(got - want).max() < 3e-2
+    assert np.sqrt(((got - want) ** 2).mean()) < 6e-3
+
+
 def test_shape_errors_are_reported_not_launched():
     b = _b()
     A = b.to_device(_bf16(6, 0, (16, 64), 1.0))
