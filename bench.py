@@ -292,6 +292,27 @@ def run_ours(args):
             breakdown[k] = {"ms_per_step": round(t_ms / 3, 4), "launches_per_step": n // 3}
         dec.profile_enable([])
 
+    # ---- untimed extra: one full decode (state set-up, every denoising step of every block, EoTP) on the same model
+    decode_info = None
+    if rank == 0:
+        eot_bias = 14.0
+        dec2 = binding.Decoder(SHAPE, w, filt, block_len=s, tau=DEC.tau, max_batch=B, max_seq=P + G, device=local,
+                               lm_head_bias=wl.make_eot_bias(SHAPE, eot_bias))
+        d_out = torch.empty(B, G, dtype=torch.int32, device=dev)
+        dec2.decode_device(d_prompts, G, d_out)
+        torch.cuda.synchronize()
+        ev0.record()
+        out_len, seq_steps, total_steps = dec2.decode_device(d_prompts, G, d_out)
+        ev1.record()
+        torch.cuda.synchronize()
+        ms_dec = ev0.elapsed_time(ev1)
+        decode_info = {"workload": "C2: full Learn2PD decode, prompt %d + generation %d, block %d, filter + EoTP, "
+                                   "EoT logit biased by the constant %.1f" % (P, G, s, eot_bias),
+                       "steps_per_sequence": float(np.mean(seq_steps)), "steps_one_token_per_step": G,
+                       "out_len": [int(v) for v in out_len], "ms": ms_dec, "ms_per_step": ms_dec / max(total_steps, 1),
+                       "generated_tokens_per_s": float(np.sum(out_len)) / (ms_dec * 1e-3)}
+        dec2.close()
+
     if rank == 0:
         T, R = B * (P + G), B * s
         work = step_work(SHAPE, T, P + G, R)
@@ -322,6 +343,7 @@ def run_ours(args):
                               "t_flops_ms": 1e3 * t_flops, "t_bytes_ms": 1e3 * t_bytes, "t_roof_ms": t_roof_ms,
                               "frac": t_roof_ms / ms_step, "peaks": pk, "peak_source": pk_src},
             "breakdown": breakdown,
+            "decode": decode_info,
         }
         if world == 1 and not args.no_cpu_baseline:
             import threadpoolctl

@@ -42,6 +42,7 @@ struct KParams {
   int M, N, K, tile_n, n_stages, b_stage_bytes;
   int slabs, a_stage_bytes;         // row slabs (of 128 * CG rows) one unit covers: 1, or 2 = accumulators not double-buffered
   int m_tiles, n_tiles, k_splits;   // m_tiles counts row tiles of 128 * CG * slabs rows
+  int group_m;                      // row tiles per raster group (see the unit order in gemm_body)
   void *out;
   const float *bias;
   float *part_m, *part_s;
@@ -383,21 +384,30 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
   if (CG == 2) ptx::cluster_sync();     // the peer's barriers exist before anything arrives on them
   ptx::tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  // set-up above overlaps the previous kernel's tail; from here on its results are needed
+  // The set-up above overlaps the previous kernel's tail.  Of what follows, only the activation loads
+  // (producer) and the output stores (epilogue warps) touch memory that other kernels of the stream
+  // write or read: those threads call grid_dep_wait() themselves, after the producer has already
+  // requested the first weight tiles, which no kernel writes.
   grid_dep_launch();
-  grid_dep_wait();
 
   const int num_units = p.m_tiles * p.n_tiles * p.k_splits;
   const int num_kb = (p.K + TILE_K - 1) / TILE_K;
   const int kb_per = (num_kb + p.k_splits - 1) / p.k_splits;
   const int half_n = p.tile_n >> 1;
-  // unit -> (row tile, column tile, K slice); row tiles of one column tile are adjacent so that the
-  // CTAs running at the same time share the weight tile in L2
+  // unit -> (row tile, column tile, K slice).  Within a K slice the units run group by group of
+  // group_m row tiles; inside a group the row tiles of one column tile are adjacent, then the next
+  // column tile follows.  The CTAs running at the same time thus share a few weight tiles, and a
+  // group's activation rows (sized to a fraction of L2) stay resident while its column tiles stream by.
   auto decode = [&](int u, int &mt, int &nt, int &kb0, int &kb1) {
-    mt = u % p.m_tiles;
-    const int r = u / p.m_tiles;
-    nt = r % p.n_tiles;
-    const int ks = r / p.n_tiles;
+    const int per_slice = p.m_tiles * p.n_tiles;
+    const int ks = u / per_slice;
+    const int r = u - ks * per_slice;
+    const int per_group = p.group_m * p.n_tiles;
+    const int g = r / per_group;
+    const int w = r - g * per_group;
+    const int gm = min(p.group_m, p.m_tiles - g * p.group_m);   // the last group may be smaller
+    nt = w / gm;
+    mt = g * p.group_m + (w - nt * gm);
     kb0 = ks * kb_per;
     kb1 = min(num_kb, kb0 + kb_per);
   };
@@ -409,6 +419,46 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
       const uint64_t pol_a = ptx::policy_evict_last();    // activations are re-read by every column tile
       const uint32_t b_bytes = (CG == 2) ? (uint32_t)half_n * 128u : (uint32_t)p.tile_n * 128u;
       const uint32_t tx = CG * (p.a_stage_bytes + b_bytes);
+      auto issue_b = [&](int stage, int kb, int nt) {   // weight tile of k-block kb (and the stage's byte count)
+        const uint32_t dstB = sB + stage * p.b_stage_bytes;
+        if (CG == 1) {
+          ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
+          if (EPI == EPI_SWIGLU) {
+            ptx::tma_load_2d_hint(dstB, tmB, full_bar(stage), kb * TILE_K, nt * half_n, pol_w);
+            ptx::tma_load_2d_hint(dstB + half_n * 128, tmB2, full_bar(stage), kb * TILE_K, nt * half_n, pol_w);
+          } else {
+            ptx::tma_load_2d_hint(dstB, tmB, full_bar(stage), kb * TILE_K, nt * p.tile_n, pol_w);
+          }
+        } else {
+          if (leader) ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
+          const uint32_t lead_full = ptx::mapa(full_bar(stage), 0);
+          if (EPI == EPI_SWIGLU)
+            ptx::tma_load_2d_pair_hint(dstB, leader ? tmB : tmB2, lead_full, kb * TILE_K, nt * half_n, pol_w);
+          else
+            ptx::tma_load_2d_pair_hint(dstB, tmB, lead_full, kb * TILE_K, nt * p.tile_n + (int)rank * half_n, pol_w);
+        }
+      };
+      auto issue_a = [&](int stage, int kb, int m0) {   // activation rows of k-block kb, one box per slab
+        const uint32_t dstA = sA + stage * p.a_stage_bytes;
+        if (CG == 1) {
+          for (int sl = 0; sl < slabs; ++sl)
+            ptx::tma_load_2d_hint(dstA + sl * A_STAGE_BYTES, tmA, full_bar(stage), kb * TILE_K, m0 + sl * TILE_M, pol_a);
+        } else {
+          const uint32_t lead_full = ptx::mapa(full_bar(stage), 0);
+          for (int sl = 0; sl < slabs; ++sl)
+            ptx::tma_load_2d_pair_hint(dstA + sl * A_STAGE_BYTES, tmA, lead_full, kb * TILE_K, m0 + sl * TILE_M * CG, pol_a);
+        }
+      };
+      // the weight tiles of the first unit's first k-blocks are requested while the previous kernel may
+      // still be running; the activations only once it has completed
+      int pre = 0;
+      if (group < num_units) {
+        int mt, nt, kb0, kb1;
+        decode(group, mt, nt, kb0, kb1);
+        pre = min(kb1 - kb0, p.n_stages);
+        for (int i = 0; i < pre; ++i) issue_b(i, kb0 + i, nt);
+      }
+      grid_dep_wait();
       // every unit starts at stage 0 (so the staging area is what a unit fills last); one phase bit per stage
       uint32_t phases = 0;
       int lt = 0;
@@ -419,29 +469,14 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
         const int m0 = mt * unit_rows + (int)rank * TILE_M;
         int stage = 0;
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (p.gate && lt > 0 && kb - kb0 == p.n_stages - 2 &&
-              !ptx::mbar_wait(sfree_bar, (uint32_t)(lt - 1) & 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
-          if (!ptx::mbar_wait(empty_bar(stage), ((phases >> stage) & 1u) ^ 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
-          const uint32_t dstA = sA + stage * p.a_stage_bytes, dstB = sB + stage * p.b_stage_bytes;
-          if (CG == 1) {
-            ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
-            for (int sl = 0; sl < slabs; ++sl)
-              ptx::tma_load_2d_hint(dstA + sl * A_STAGE_BYTES, tmA, full_bar(stage), kb * TILE_K, m0 + sl * TILE_M, pol_a);
-            if (EPI == EPI_SWIGLU) {
-              ptx::tma_load_2d_hint(dstB, tmB, full_bar(stage), kb * TILE_K, nt * half_n, pol_w);
-              ptx::tma_load_2d_hint(dstB + half_n * 128, tmB2, full_bar(stage), kb * TILE_K, nt * half_n, pol_w);
-            } else {
-              ptx::tma_load_2d_hint(dstB, tmB, full_bar(stage), kb * TILE_K, nt * p.tile_n, pol_w);
-            }
+          if (lt == 0 && kb - kb0 < pre) {
+            issue_a(stage, kb, m0);
           } else {
-            if (leader) ptx::mbar_arrive_expect_tx(full_bar(stage), tx);
-            const uint32_t lead_full = ptx::mapa(full_bar(stage), 0);
-            for (int sl = 0; sl < slabs; ++sl)
-              ptx::tma_load_2d_pair_hint(dstA + sl * A_STAGE_BYTES, tmA, lead_full, kb * TILE_K, m0 + sl * TILE_M * CG, pol_a);
-            if (EPI == EPI_SWIGLU)
-              ptx::tma_load_2d_pair_hint(dstB, leader ? tmB : tmB2, lead_full, kb * TILE_K, nt * half_n, pol_w);
-            else
-              ptx::tma_load_2d_pair_hint(dstB, tmB, lead_full, kb * TILE_K, nt * p.tile_n + (int)rank * half_n, pol_w);
+            if (p.gate && lt > 0 && kb - kb0 == p.n_stages - 2 &&
+                !ptx::mbar_wait(sfree_bar, (uint32_t)(lt - 1) & 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
+            if (!ptx::mbar_wait(empty_bar(stage), ((phases >> stage) & 1u) ^ 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
+            issue_b(stage, kb, nt);
+            issue_a(stage, kb, m0);
           }
           phases ^= 1u << stage;
           if (++stage == p.n_stages) stage = 0;
@@ -497,6 +532,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
     const int q = warp & 3, sl = (warp - 3) >> 2;
     int lt = 0;
     bool ok = true;
+    grid_dep_wait();   // the outputs may still be in use by earlier kernels until they have completed
     for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
       int mt, nt, kb0, kb1;
       decode(u, mt, nt, kb0, kb1);
@@ -731,6 +767,11 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
   p.gate = (p.out_tma && p.slabs == 2 && stages >= 4) ? 1 : 0;
   p.n_tiles = ceil_div(g.N, n_per_tile);
   p.k_splits = ks;
+  {   // a raster group's activation rows: about 32 MB, a quarter of L2
+    const double tile_bytes = (double)TILE_M * cg * p.slabs * ((double)g.K / ks) * 2.0;
+    int gm = (int)(32.0e6 / tile_bytes);
+    p.group_m = gm < 1 ? 1 : (gm > p.m_tiles ? p.m_tiles : gm);
+  }
   p.out = g.out; p.bias = g.bias; p.part_m = g.part_m; p.part_s = g.part_s; p.part_i = g.part_i;
   p.rows_padded = g.rows_padded; p.logits = g.logits; p.status = g.status;
   const int units = p.m_tiles * p.n_tiles * ks;
