@@ -12,9 +12,12 @@
 //   EPI_LMHEAD    per-row running (max, sum exp, argmax) over the vocabulary tile, written as one
 //                 record per (tile, row): the logits are never stored (Eq. 3-4 need only these).
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = TMEM owner and MMA issuer, warp 2 = second MMA
-// issuer (two-slab units only), warps 3-6 (and 7-10 for the second slab) = epilogue; warp w reads
-// TMEM lanes 32*(w%4) .. +31.
+// Warp roles: warp 0 = TMA producer of the weight tiles, warp 1 = TMEM owner and MMA issuer,
+// warp 2 = second MMA issuer (two-slab units only), warps 3-6 (and 7-10 for the second slab) =
+// epilogue (warp w reads TMEM lanes 32*(w%4) .. +31), last warp = TMA producer of the activation
+// tiles.  The loads have two issuing threads because one thread needs ~170 cycles per TMA
+// instruction, and a k-block of a two-slab unit takes three of them plus an L2 prefetch; the weight
+// producer depends on no earlier kernel and starts while the previous kernel is still running.
 //
 // One thread can issue a tcgen05.mma (K = 16) only every ~132 cycles, whatever its N, while the
 // tensor pipe needs N/2 cycles for it: a single issuer keeps the pipe busy only for N = 256.
@@ -59,6 +62,9 @@ __device__ __forceinline__ void fail(int32_t *status, int code) {
   if (status) atomicCAS(status, 0, code);
 }
 
+// silu(g) * u with the fast exponential and division (a few ulp, far below the bf16 rounding of the result)
+__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
+
 // Emitters: what the epilogue does with 16 consecutive accumulator columns of one row.
 // `valid` = columns left in the row from the first of the 16 (the row length is a multiple of 8).
 __device__ __forceinline__ void emit_store16(bf16 *dst, const uint32_t *v, int valid) {   // 16 fp32 -> 16 bf16, 32 bytes
@@ -102,7 +108,7 @@ __device__ __forceinline__ void emit_swiglu16(bf16 *dst, const uint32_t *g, cons
     for (int i = 0; i < 4; ++i) {
       const float g0 = __uint_as_float(g[hseg * 8 + 2 * i]), g1 = __uint_as_float(g[hseg * 8 + 2 * i + 1]);
       const float u0 = __uint_as_float(u[hseg * 8 + 2 * i]), u1 = __uint_as_float(u[hseg * 8 + 2 * i + 1]);
-      __nv_bfloat162 t = __floats2bfloat162_rn(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
+      __nv_bfloat162 t = __floats2bfloat162_rn(silu_mul(g0, u0), silu_mul(g1, u1));
       pw[i] = *reinterpret_cast<uint32_t *>(&t);
     }
     *reinterpret_cast<uint4 *>(dst + hseg * 8) = pk;
@@ -309,7 +315,7 @@ __device__ __forceinline__ void drain_tile_staged(const KParams &p, const CUtens
         for (int i = 0; i < 4; ++i) {
           const float g0 = __uint_as_float(g[hseg * 8 + 2 * i]), g1 = __uint_as_float(g[hseg * 8 + 2 * i + 1]);
           const float u0 = __uint_as_float(u[hseg * 8 + 2 * i]), u1 = __uint_as_float(u[hseg * 8 + 2 * i + 1]);
-          __nv_bfloat162 t = __floats2bfloat162_rn(g0 / (1.0f + __expf(-g0)) * u0, g1 / (1.0f + __expf(-g1)) * u1);
+          __nv_bfloat162 t = __floats2bfloat162_rn(silu_mul(g0, u0), silu_mul(g1, u1));
           pw[i] = *reinterpret_cast<uint32_t *>(&t);
         }
         st16(chunk_addr(qb * 2 + hseg), pw[0], pw[1], pw[2], pw[3]);
@@ -416,7 +422,6 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
       const uint64_t pol_w = ptx::policy_evict_first();   // weights are read once per step
-      const uint64_t pol_a = ptx::policy_evict_last();    // activations are re-read by every column tile
       const uint32_t b_bytes = (CG == 2) ? (uint32_t)half_n * 128u : (uint32_t)p.tile_n * 128u;
       const uint32_t tx = CG * (p.a_stage_bytes + b_bytes);
       auto issue_b = [&](int stage, int kb, int nt) {   // weight tile of k-block kb (and the stage's byte count)
@@ -438,46 +443,42 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
             ptx::tma_load_2d_pair_hint(dstB, tmB, lead_full, kb * TILE_K, nt * p.tile_n + (int)rank * half_n, pol_w);
         }
       };
-      auto issue_a = [&](int stage, int kb, int m0) {   // activation rows of k-block kb, one box per slab
-        const uint32_t dstA = sA + stage * p.a_stage_bytes;
+      // Weights come from HBM exactly once and the ring holds only a few k-blocks, fewer than HBM's latency
+      // under load is worth: the tile PF_AHEAD k-blocks further on is asked into L2 with every load.
+      constexpr int PF_AHEAD = 8;
+      auto prefetch_b = [&](int kb, int nt) {
         if (CG == 1) {
-          for (int sl = 0; sl < slabs; ++sl)
-            ptx::tma_load_2d_hint(dstA + sl * A_STAGE_BYTES, tmA, full_bar(stage), kb * TILE_K, m0 + sl * TILE_M, pol_a);
+          if (EPI == EPI_SWIGLU) {
+            ptx::tma_prefetch_l2_2d(tmB, kb * TILE_K, nt * half_n);
+            ptx::tma_prefetch_l2_2d(tmB2, kb * TILE_K, nt * half_n);
+          } else {
+            ptx::tma_prefetch_l2_2d(tmB, kb * TILE_K, nt * p.tile_n);
+          }
+        } else if (EPI == EPI_SWIGLU) {
+          ptx::tma_prefetch_l2_2d(leader ? tmB : tmB2, kb * TILE_K, nt * half_n);
         } else {
-          const uint32_t lead_full = ptx::mapa(full_bar(stage), 0);
-          for (int sl = 0; sl < slabs; ++sl)
-            ptx::tma_load_2d_pair_hint(dstA + sl * A_STAGE_BYTES, tmA, lead_full, kb * TILE_K, m0 + sl * TILE_M * CG, pol_a);
+          ptx::tma_prefetch_l2_2d(tmB, kb * TILE_K, nt * p.tile_n + (int)rank * half_n);
         }
       };
-      // the weight tiles of the first unit's first k-blocks are requested while the previous kernel may
-      // still be running; the activations only once it has completed
-      int pre = 0;
-      if (group < num_units) {
-        int mt, nt, kb0, kb1;
-        decode(group, mt, nt, kb0, kb1);
-        pre = min(kb1 - kb0, p.n_stages);
-        for (int i = 0; i < pre; ++i) issue_b(i, kb0 + i, nt);
-      }
-      grid_dep_wait();
-      // every unit starts at stage 0 (so the staging area is what a unit fills last); one phase bit per stage
+      // one producer thread for the weights (this warp), one for the activations (last warp): both walk the
+      // same units, k-blocks and stages; every unit starts at stage 0 (so the staging area is what a unit
+      // fills last), with one phase bit per stage.  No kernel writes weights, so this thread does not wait
+      // for the previous kernel of the stream.
       uint32_t phases = 0;
       int lt = 0;
       bool ok = true;
       for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
         int mt, nt, kb0, kb1;
         decode(u, mt, nt, kb0, kb1);
-        const int m0 = mt * unit_rows + (int)rank * TILE_M;
         int stage = 0;
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (lt == 0 && kb - kb0 < pre) {
-            issue_a(stage, kb, m0);
-          } else {
-            if (p.gate && lt > 0 && kb - kb0 == p.n_stages - 2 &&
-                !ptx::mbar_wait(sfree_bar, (uint32_t)(lt - 1) & 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
-            if (!ptx::mbar_wait(empty_bar(stage), ((phases >> stage) & 1u) ^ 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
-            issue_b(stage, kb, nt);
-            issue_a(stage, kb, m0);
-          }
+          if (kb + p.n_stages + PF_AHEAD < kb1) prefetch_b(kb + p.n_stages + PF_AHEAD, nt);
+          if (p.gate && lt > 0 && kb - kb0 == p.n_stages - 2 &&
+              !ptx::mbar_wait(sfree_bar, (uint32_t)(lt - 1) & 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
+          if (!ptx::mbar_wait(empty_bar(stage), ((phases >> stage) & 1u) ^ 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
+          issue_b(stage, kb, nt);
+          if (kb - kb0 == p.n_stages - 1)   // the ring is primed: ask for the tiles between it and the running prefetch
+            for (int i = p.n_stages; i < min(kb1 - kb0, p.n_stages + PF_AHEAD); ++i) prefetch_b(kb0 + i, nt);
           phases ^= 1u << stage;
           if (++stage == p.n_stages) stage = 0;
         }
@@ -522,6 +523,41 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
         if (ok) {
           if (CG == 2) ptx::mma_commit_pair(tfull_bar(ab), 3);
           else ptx::mma_commit(tfull_bar(ab));
+        }
+      }
+      if (!ok) *abort_flag = 1;
+    }
+  } else if (warp == 3 + 4 * slabs) {
+    // ------------------------------------------------------------------ TMA producer of the activation tiles
+    if (lane == 0) {
+      const uint64_t pol_a = ptx::policy_evict_last();    // activations are re-read by every column tile
+      auto issue_a = [&](int stage, int kb, int m0) {   // activation rows of k-block kb, one box per slab
+        const uint32_t dstA = sA + stage * p.a_stage_bytes;
+        if (CG == 1) {
+          for (int sl = 0; sl < slabs; ++sl)
+            ptx::tma_load_2d_hint(dstA + sl * A_STAGE_BYTES, tmA, full_bar(stage), kb * TILE_K, m0 + sl * TILE_M, pol_a);
+        } else {
+          const uint32_t lead_full = ptx::mapa(full_bar(stage), 0);
+          for (int sl = 0; sl < slabs; ++sl)
+            ptx::tma_load_2d_pair_hint(dstA + sl * A_STAGE_BYTES, tmA, lead_full, kb * TILE_K, m0 + sl * TILE_M * CG, pol_a);
+        }
+      };
+      grid_dep_wait();   // the activations are the previous kernel's output
+      uint32_t phases = 0;
+      int lt = 0;
+      bool ok = true;
+      for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
+        int mt, nt, kb0, kb1;
+        decode(u, mt, nt, kb0, kb1);
+        const int m0 = mt * unit_rows + (int)rank * TILE_M;
+        int stage = 0;
+        for (int kb = kb0; kb < kb1; ++kb) {
+          if (p.gate && lt > 0 && kb - kb0 == p.n_stages - 2 &&
+              !ptx::mbar_wait(sfree_bar, (uint32_t)(lt - 1) & 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
+          if (!ptx::mbar_wait(empty_bar(stage), ((phases >> stage) & 1u) ^ 1u)) { fail(p.status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
+          issue_a(stage, kb, m0);
+          phases ^= 1u << stage;
+          if (++stage == p.n_stages) stage = 0;
         }
       }
       if (!ok) *abort_flag = 1;
@@ -583,7 +619,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
 }
 
 template <int EPI>
-__global__ void __launch_bounds__(352, 1)
+__global__ void __launch_bounds__(384, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmC, const KParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -594,7 +630,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 }
 
 template <int EPI>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(352, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(384, 1)
 gemm_tcgen05_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                          const __grid_constant__ CUtensorMap tmB2, const __grid_constant__ CUtensorMap tmC, const KParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -694,7 +730,7 @@ l2pd_status make_tma_out_3d(TmaDesc *out, void *ptr, bool fp32, int64_t rows, in
 // takes to issue its four MMAs and the stage hand-over; the bytes it must take in at INGEST bytes
 // per cycle.  A unit adds a fixed fill part and, when its accumulators are not double-buffered
 // (two slabs), the drain of the accumulator; times the number of waves over the SMs (or SM pairs).
-static double plan_cost(int M, int N, int K, int num_sms, int cg, int slabs, int unit_n, int tile_n, int ks) {
+static double plan_cost(int M, int N, int K, int num_sms, int cg, int slabs, int unit_n, int tile_n, int ks, bool is_residual) {
   const double INGEST = cg == 2 ? 58.0 : 68.0;   // measured: bytes per cycle an SM takes in from L2 through TMA
   const int groups = num_sms / cg;
   const int m_tiles = ceil_div(M, TILE_M * cg * slabs);
@@ -703,10 +739,12 @@ static double plan_cost(int M, int N, int K, int num_sms, int cg, int slabs, int
   const int waves = ceil_div(units, groups);
   const int kb = ceil_div(ceil_div(K, TILE_K), ks);
   const double bytes = (double)slabs * A_STAGE_BYTES + 128.0 * tile_n / cg;
-  const double per_kb = fmax(fmax(2.0 * tile_n * slabs, 620.0), bytes / INGEST);
-  const double drain = 14.0 * tile_n + (ks > 1 ? 4.0 * tile_n : 0.0);   // cycles to empty one 128 x tile_n accumulator
+  const double per_kb = fmax(fmax(2.0 * tile_n * slabs, 620.0), bytes / INGEST) * 1.06;
+  // emptying the accumulators: bf16 stores leave an SM at ~34 B per cycle; fp32 additions into X are bound
+  // by L2's atomic units, ~2500 B per cycle for the whole chip, i.e. ~17 B per cycle and SM when all drain at once
+  const double drain = (double)TILE_M * slabs * unit_n * (is_residual ? 4.0 / 17.0 : 2.0 / 34.0) + 1500.0;
   const double exposed = slabs == 2 ? drain : 0.3 * drain;
-  return waves * (kb * per_kb + 2500.0 + exposed) + (slabs == 2 ? 0.0 : 0.7 * drain);
+  return waves * (kb * per_kb + 6000.0 + exposed) + (slabs == 2 ? 0.0 : 0.7 * drain);
 }
 
 GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n) {
@@ -725,7 +763,7 @@ GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n) 
         const int max_ks = (epi == EPI_RESIDUAL) ? 4 : 1;
         for (int ks = 1; ks <= max_ks; ++ks) {
           if (ceil_div(K, TILE_K) < 8 * ks) break;
-          const double c = plan_cost(M, N, K, num_sms, cg, slabs, unit_n, tn, ks);
+          const double c = plan_cost(M, N, K, num_sms, cg, slabs, unit_n, tn, ks, epi == EPI_RESIDUAL);
           if (c < best_cost - 1e-9) { best_cost = c; best = GemmPlan{cg, tn, ks, slabs}; }
         }
       }
@@ -785,7 +823,7 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
 #define L2PD_LAUNCH(KERNEL, EPI)                                                                      \
   e = cudaFuncSetAttribute(KERNEL<EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET - 1024); \
   if (e != cudaSuccess) return e;                                                                    \
-  e = launch_kernel(KERNEL<EPI>, dim3(grid), dim3(96 + 128 * p.slabs), smem, st, g.a->map, g.b->map, b2, cm, p);                \
+  e = launch_kernel(KERNEL<EPI>, dim3(grid), dim3(128 + 128 * p.slabs), smem, st, g.a->map, g.b->map, b2, cm, p);                \
   if (e != cudaSuccess) return e;
   if (cg == 1) {
     switch (g.epi) {
