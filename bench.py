@@ -33,6 +33,9 @@ WORKLOAD = "C1"
 SHAPE = wl.LLADA_8B
 DEC = wl.DECODES[WORKLOAD]
 METRIC, UNIT = "generated_tokens_per_s", "tokens/s"
+# DRAM bytes (read + write) of one gate/up launch at T = 512: dram__bytes_read.sum + dram__bytes_write.sum of
+# the ncu capture summarised in profiles/gemm_pair_T512_layer_shapes.md (208.2 MB + 3.6 MB)
+GATE_UP_DRAM_BYTES_PER_LAUNCH = 211.8e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -338,7 +341,8 @@ def run_ours(args):
                          "frac": (achieved / pk["bf16_tflops_sustained"]) if achieved else None,
                          "peak_source": pk_src + " (sustained bf16, kernel timed inside a long step)",
                          "flops_per_launch": gu_flops, "avg_launch_ms": gu_ms / gu_n if gu_n else None,
-                         "traffic": None},
+                         "traffic": GATE_UP_DRAM_BYTES_PER_LAUNCH,
+                         "algorithmic_bytes": 2.0 * (2 * SHAPE.d_ff * SHAPE.d_model + T * SHAPE.d_model + T * SHAPE.d_ff)},
             "step_roofline": {"flops": work["flops"], "weight_bytes": work["weight_bytes"], "act_bytes": work["act_bytes"],
                               "t_flops_ms": 1e3 * t_flops, "t_bytes_ms": 1e3 * t_bytes, "t_roof_ms": t_roof_ms,
                               "frac": t_roof_ms / ms_step, "peaks": pk, "peak_source": pk_src},

@@ -8,7 +8,7 @@
 //   * EoTP (Section 3.3): the earliest committed [EoT] cuts the sequence; later positions leave
 //     the mask set and read as [EoT];
 //   * block advance / stop (Algorithm 3: no block after one that holds [EoT]).
-// One thread block per sequence taking part in the step.
+// One thread block per sequence taking part in the step (a warp per block row where possible).
 #include "common.cuh"
 
 namespace l2pd {
@@ -17,7 +17,7 @@ namespace {
 
 constexpr int MAX_S = 64;
 
-__global__ void __launch_bounds__(256) decide_kernel(DecideArgs a) {
+__global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
   __shared__ float s_conf[MAX_S];
   __shared__ int s_pred[MAX_S];
   __shared__ float s_c[MAX_S];
@@ -174,7 +174,10 @@ __global__ void __launch_bounds__(256) decide_kernel(DecideArgs a) {
 }  // namespace
 
 cudaError_t launch_decide(cudaStream_t st, const DecideArgs &a, int n_slots) {
-  return launch_kernel(decide_kernel, dim3(n_slots), dim3(256), 0, st, a);
+  // one warp per block row for the merge of the tile records (the latency-bound part): up to 32 warps
+  int threads = 32 * a.s;
+  threads = threads < 256 ? 256 : (threads > 1024 ? 1024 : threads);
+  return launch_kernel(decide_kernel, dim3(n_slots), dim3(threads), 0, st, a);
 }
 
 }  // namespace l2pd

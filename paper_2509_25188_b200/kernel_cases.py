@@ -9,6 +9,9 @@ Cases (LLaDA-8B layer shapes unless overridden with --d/--ff/--vocab/--heads):
   down     X[T,d]  += H[T,F] Wd^T                   residual epilogue
   lm_head  pred/conf over V for R = --rows rows     fused confidence head
   attn     bidirectional attention, --rows queries and keys, 32 heads x 128
+  step     whole denoising steps of a --layers deep model of these widths (batch 1, --rows / 2 prompt
+           tokens + --rows / 2 masks, block 32): the small, self-ending case for profiling the
+           memory-bound kernels (RMSNorm, RoPE/scatter, embedding, final norm, decision)
 
 Each iteration uses a different weight buffer out of a ring larger than L2 (126 MB), so that the
 weights come from HBM as they do inside a step.  Prints one JSON line with the mean device time
@@ -27,7 +30,7 @@ from . import binding as b
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["qkv", "o", "gate_up", "down", "lm_head", "attn"])
+    ap.add_argument("case", choices=["qkv", "o", "gate_up", "down", "lm_head", "attn", "step"])
     ap.add_argument("--rows", type=int, default=512)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
@@ -36,6 +39,7 @@ def main():
     ap.add_argument("--ff", type=int, default=12288)
     ap.add_argument("--vocab", type=int, default=126464)
     ap.add_argument("--heads", type=int, default=32)
+    ap.add_argument("--layers", type=int, default=2, help="step: number of layers")
     ap.add_argument("--impl", type=int, default=0, help="attn: 0 = tcgen05 kernel, 1 = mma.sync kernel")
     ap.add_argument("--ring", type=int, default=0, help="number of weight buffers to rotate through (0 = enough to exceed L2)")
     a = ap.parse_args()
@@ -51,7 +55,24 @@ def main():
         n = a.ring if a.ring > 0 else max(2, int(min_bytes // (r * c * 2)) + 1)
         return [rnd(r, c) for _ in range(n)]
 
-    if a.case == "qkv":
+    if a.case == "step":
+        from . import workloads as wl
+        shape = wl.ModelShape(n_layers=a.layers, d_model=d, n_heads=H, head_dim=dh, d_ff=F, vocab=V, rms_eps=1e-5,
+                              rope_theta=500000.0, mask_id=V - 1, eot_id=V - 2, dtype="bf16")
+        ones = torch.ones(d, device=dev)
+        w = {"tok_emb": rnd(V, d), "lm_head": rnd(V, d),
+             "final_norm": torch.full((d,), wl.spread_gain(shape), device=dev),
+             "layers": [{"wqkv": rnd(3 * d, d), "wo": rnd(d, d), "w_gate": rnd(F, d), "w_up": rnd(F, d),
+                         "w_down": rnd(d, F), "norm1": ones, "norm2": ones} for _ in range(a.layers)]}
+        dec = b.Decoder(shape, w, wl.make_filter(32, 0.96, seed=0), block_len=32, max_batch=1, max_seq=T)
+        prompts = torch.from_numpy(wl.make_prompts(1, T // 2, shape, seed=1)).to(dev)
+
+        def run(i):
+            dec.state_reset_device(prompts, T - T // 2)
+            dec.denoise_step(outputs=False)
+        per_layer = 2.0 * T * (4 * d * d + 3 * d * F) + 4.0 * T * T * d
+        flops, byts = a.layers * per_layer + 2.0 * 32 * d * V, 2.0 * (a.layers * (4 * d * d + 3 * d * F) + V * d)
+    elif a.case == "qkv":
         A, W = rnd(T, d, 1.0), ring(3 * d, d)
         Cc = torch.empty(T, 3 * d, dtype=torch.bfloat16, device=dev)
         run = lambda i: b._check(b.lib.l2pd_gemm_bf16(b._stream(), A.data_ptr(), W[i % len(W)].data_ptr(),
