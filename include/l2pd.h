@@ -223,10 +223,14 @@ void l2pd_destroy(l2pd_ctx *ctx);                   /* NULL is allowed */
  */
 
 /* C[M,N] (bf16) = A[M,K] (bf16, row-major) x W[N,K]^T (bf16, row-major); tcgen05 path.
- * K and N multiples of 8.  tile_n = width + 1000 * cta_group + 10000 * k_splits, every part optional
- * (0 = chosen automatically): width a multiple of 16 (SwiGLU: 32) in [32, 256]; cta_group 1, or 2 for
- * a pair of SMs on one 256-row tile; k_splits (residual epilogue only) slices K, the slices adding
- * into X with floating-point reductions whose order is not fixed. */
+ * K and N multiples of 8.  tile_n = width + 1000 * cta_group + 10000 * k_splits + 100000 * slabs,
+ * every part optional (0 = chosen automatically): width a multiple of 16 in [32, 256]; cta_group 1,
+ * or 2 for a pair of SMs on one 256-row tile; k_splits (residual epilogue only) slices K, the
+ * slices adding into X with floating-point reductions whose order is not fixed; slabs 2 (pairs
+ * only) lets one unit cover two 256-row slabs against one load of the weight tile.
+ * A and the output follow stream order.  The weights W are requested before the kernel launched
+ * just ahead of this one in the stream has completed (programmatic dependent launch): that kernel
+ * must not be the one that writes them. */
 l2pd_status l2pd_gemm_bf16(void *stream, const void *A, const void *W, void *C,
                            int32_t M, int32_t N, int32_t K, int32_t tile_n, int32_t check);
 /* X[M,N] (fp32) += A[M,K] x W[N,K]^T : projection with the residual add in the epilogue. */

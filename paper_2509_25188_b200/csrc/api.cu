@@ -666,7 +666,7 @@ static l2pd_status gemm_common(void *stream, int epi, const void *A, const void 
   // tile_n = width + 1000 * cta_group + 10000 * k_splits + 100000 * slabs; any part 0 = chosen automatically
   const int want_sl = tile_n / 100000, want_ks = (tile_n % 100000) / 10000, want_cg = (tile_n % 10000) / 1000,
             want_tn = tile_n % 1000;
-  const int unit = epi == EPI_SWIGLU ? 32 : 16;
+  const int unit = 16;
   if (want_tn && (want_tn < 32 || want_tn > 256 || (want_tn % unit))) return L2PD_ERR_SHAPE;
   if (want_cg > 2 || want_ks > 8 || (want_ks > 1 && epi != EPI_RESIDUAL) || want_sl > 2) return L2PD_ERR_SHAPE;
   GemmPlan pl = plan_gemm(epi, M, N, K, sms, want_tn);

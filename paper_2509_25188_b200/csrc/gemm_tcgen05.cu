@@ -162,7 +162,7 @@ __device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int
       ptx::tmem_ld_x16(taddr + half_n + c, u);
     };
     auto emit = [&](const uint32_t *g, const uint32_t *u, int c) {
-      if (row_ok && n0 + c < p.N) emit_swiglu16(H + (int64_t)row * p.N + n0 + c, g, u, p.N - n0 - c);
+      if (row_ok && n0 + c < p.N) emit_swiglu16(H + (int64_t)row * p.N + n0 + c, g, u, min(p.N - n0 - c, half_n - c));
     };
     load(ga, ua, 0);
     for (int c = 0; c < half_n; c += 32) {
@@ -752,7 +752,7 @@ GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n) 
   GemmPlan best{1, 256, 1, 1};
   double best_cost = 1e300;
   const bool swiglu = epi == EPI_SWIGLU;
-  const int step = swiglu ? 32 : 16;
+  const int step = 16;   // SwiGLU: the gate and up halves are then multiples of 8 (one swizzle group of rows)
   for (int cg = 1; cg <= 2; ++cg) {
     if (cg == 2 && (M <= TILE_M || epi == EPI_LMHEAD || num_sms < 2)) continue;
     for (int slabs = 1; slabs <= 2; ++slabs) {

@@ -93,6 +93,7 @@ def test_gemm_bf16_residual(M, N, K, tile_n):
                                           (77, 136, 72, 64), (640, 2048, 256, 96), (512, 1408, 512, 2224),
                                           (200, 336, 192, 2064), (1000, 2048, 256, 2256),
                                           (512, 1408, 512, 202160), (300, 2048, 256, 202256),
+                                          (512, 1408, 512, 202176), (200, 336, 192, 1176), (130, 1408, 128, 2144),
                                           (512, 24576, 256, 0)])
 def test_gemm_bf16_swiglu(M, F, K, tile_n):
     b = _b()
