@@ -20,6 +20,13 @@ struct l2pd_ctx {
   int device = 0, num_sms = 148;
   bool force_simt = false;   // L2PD_FORCE_SIMT=1: bf16 GEMMs and attention on the CUDA-core cross-check kernels
   bool attn_tc = false;      // head size 128: attention on tcgen05 (L2PD_ATTN_WARP=1 keeps the mma.sync kernel)
+  // RoPE in the QKV epilogue (tcgen05 attention, no prefix cache; L2PD_NO_ROPE_FUSION=1 turns it off): the context
+  // owns copies of the QKV weights with the q / k rows of each head reordered so that rotary pairs are adjacent;
+  // q and k then live in that order, which leaves every q . k unchanged; attention reads q, k, v from the packed qkv rows
+  bool fuse_rope = false;
+  std::vector<void *> wqkv_perm;
+  int32_t *d_row_pos = nullptr;
+  TmaDesc tq_packed, tk_packed, tv_packed;
 
   // weights (borrowed device pointers)
   const void *tok_emb = nullptr, *lm_head = nullptr;
@@ -53,6 +60,7 @@ struct l2pd_ctx {
   StepSummary *d_summary = nullptr, *h_summary = nullptr;
   int32_t *d_status = nullptr, *h_status = nullptr;
   float2 *cs_table = nullptr;
+  float2 *cs_table_t = nullptr;      // the same table as [pair][position] (fused rotation in the QKV epilogue)
 
   // TMA descriptors (bf16 path)
   TmaDesc ta_n, ta_att, ta_h, ta_nf, ta_q, t_kstore, t_vstore;
@@ -184,6 +192,10 @@ l2pd_status run_gemm_tc(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const Tm
   g.epi = epi; g.a = a; g.b = b; g.b2 = b2; g.c = cm; g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.out = out;
   g.cta_group = pl.cta_group; g.k_splits = pl.k_splits; g.slabs = pl.slabs;
   g.status = c->d_status;
+  if (epi == EPI_QKV_ROPE) {
+    g.rope_cols = 2 * c->cfg.n_heads * c->cfg.head_dim; g.rope_dh = c->cfg.head_dim;
+    g.cs_table = c->cs_table_t; g.cs_stride = c->cfg.max_seq; g.row_pos = c->d_row_pos;
+  }
   CKLK(kind, launch_gemm_tcgen05(s, g, c->num_sms));
   return L2PD_OK;
 }
@@ -232,7 +244,7 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     c->tc_rows = T_rows;
   }
 
-  CKLK(L2PD_K_OTHER, launch_build_row_map(s, c->d_meta, n_slots, c->d_row_slot));
+  CKLK(L2PD_K_OTHER, launch_build_row_map(s, c->d_meta, n_slots, c->d_row_slot, c->d_row_pos));
   CKLK(L2PD_K_EMBED, launch_embed_rmsnorm<T>(s, c->d_tokens, c->P + c->G, c->d_meta, c->d_row_slot, (const T *)c->tok_emb,
                               c->norm1[0], f.rms_eps, c->x, n, T_rows, d));
   if (c->cap) CK(cudaMemcpyAsync(c->cap, c->x, (size_t)T_rows * d * 4, cudaMemcpyDeviceToDevice, s));
@@ -241,14 +253,18 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     T *kc = (T *)c->kc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
     T *vc = (T *)c->vc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
     l2pd_status r;
-    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_QKV, EPI_STORE, &c->ta_n, &c->tb_qkv[l], nullptr, c->tcw_qkv > 0 ? &c->tc_qkv : nullptr, qkv, T_rows, 3 * hd, d, c->pl_qkv);
+    if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_QKV, c->fuse_rope ? EPI_QKV_ROPE : EPI_STORE, &c->ta_n, &c->tb_qkv[l], nullptr, c->tcw_qkv > 0 ? &c->tc_qkv : nullptr, qkv, T_rows, 3 * hd, d, c->pl_qkv);
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_QKV, EPI_STORE, n, c->wqkv[l], nullptr, qkv, nullptr, T_rows, 3 * hd, d);
     if (r) return r;
-    CKLK(L2PD_K_ROPE, launch_rope_scatter<T>(s, qkv, c->d_meta, c->d_row_slot, c->cs_table, q, kc, vc, c->kv_seq_stride, T_rows, H, dh));
-    if (tc && c->attn_tc) {
+    if (!(tc && c->fuse_rope))
+      CKLK(L2PD_K_ROPE, launch_rope_scatter<T>(s, qkv, c->d_meta, c->d_row_slot, c->cs_table, q, kc, vc, c->kv_seq_stride, T_rows, H, dh));
+    if (tc && c->fuse_rope) {
+      CKLK(L2PD_K_ATTENTION, launch_attention_tc(s, c->tq_packed, c->tk_packed, c->tv_packed, c->d_meta, (bf16 *)att, hd, 0, 0, 1,
+                                n_slots, max_q_rows, H, c->d_status));
+    } else if (tc && c->attn_tc) {
       const int kv_row_base = f.kv_cache_mode ? l * f.max_batch * f.max_seq : 0;
       CKLK(L2PD_K_ATTENTION, launch_attention_tc(s, c->ta_q, c->t_kstore, c->t_vstore, c->d_meta, (bf16 *)att, hd, f.max_seq,
-                                kv_row_base, n_slots, max_q_rows, H, c->d_status));
+                                kv_row_base, 0, n_slots, max_q_rows, H, c->d_status));
     } else if (tc) {
       CKLK(L2PD_K_ATTENTION, launch_attention_bf16(s, (const bf16 *)q, (const bf16 *)kc, (const bf16 *)vc, c->d_meta, (bf16 *)att, hd, hd,
                                 c->kv_seq_stride, hd, n_slots, max_q_rows, H, dh));
@@ -331,6 +347,8 @@ void free_all(l2pd_ctx *c) {
   cudaFree(c->d_tokens); cudaFree(c->d_masked); cudaFree(c->d_state_ints);
   cudaFree(c->x); cudaFree(c->n); cudaFree(c->qkv); cudaFree(c->q); cudaFree(c->att); cudaFree(c->h); cudaFree(c->nf);
   cudaFree(c->kc); cudaFree(c->vc); cudaFree(c->part); cudaFree(c->logits_f32);
+  for (void *w : c->wqkv_perm) cudaFree(w);
+  cudaFree(c->d_row_pos); cudaFree(c->cs_table_t);
   cudaFree(c->d_meta); cudaFree(c->d_row_slot); cudaFree(c->d_summary); cudaFree(c->d_status); cudaFree(c->cs_table);
   if (c->h_meta) cudaFreeHost(c->h_meta);
   if (c->h_summary) cudaFreeHost(c->h_summary);
@@ -433,6 +451,7 @@ l2pd_status l2pd_init(const l2pd_config *cfg, const l2pd_weights *w, int device,
   A(dev_alloc(c, &c->logits_f32, c->max_lm_rows * (int64_t)V));
   A(dev_alloc(c, &c->d_meta, (int64_t)f.max_batch));
   A(dev_alloc(c, &c->d_row_slot, mr));
+  A(dev_alloc(c, &c->d_row_pos, mr));
   A(dev_alloc(c, &c->d_summary, (int64_t)f.max_batch));
   A(dev_alloc(c, &c->d_status, (int64_t)1));
   A(dev_alloc(c, &c->cs_table, (int64_t)f.max_seq * (f.head_dim / 2)));
@@ -445,7 +464,7 @@ l2pd_status l2pd_init(const l2pd_config *cfg, const l2pd_weights *w, int device,
   // the activation buffers back TMA boxes that reach past the live rows: start them defined
   if (cudaMemset(c->n, 0, mr * d * es) != cudaSuccess || cudaMemset(c->att, 0, mr * hd * es) != cudaSuccess ||
       cudaMemset(c->h, 0, mr * F * es) != cudaSuccess || cudaMemset(c->nf, 0, c->max_lm_rows * d * es) != cudaSuccess ||
-      cudaMemset(c->q, 0, mr * hd * es) != cudaSuccess)
+      cudaMemset(c->q, 0, mr * hd * es) != cudaSuccess || cudaMemset(c->qkv, 0, mr * 3 * hd * es) != cudaSuccess)
     return fail(L2PD_ERR_CUDA);
   // key tiles reach past a sequence's last key: what lies there is masked out of the scores, but
   // the value rows are multiplied by a probability of zero, so they must never hold NaN or Inf
@@ -467,6 +486,12 @@ l2pd_status l2pd_init(const l2pd_config *cfg, const l2pd_weights *w, int device,
       }
     if (cudaMemcpy(c->cs_table, tab.data(), tab.size() * sizeof(float2), cudaMemcpyHostToDevice) != cudaSuccess)
       return fail(L2PD_ERR_CUDA);
+    std::vector<float2> tab_t(tab.size());
+    for (int pos = 0; pos < f.max_seq; ++pos)
+      for (int i = 0; i < half; ++i) tab_t[(size_t)i * f.max_seq + pos] = tab[(size_t)pos * half + i];
+    if (cudaMalloc((void **)&c->cs_table_t, tab_t.size() * sizeof(float2)) != cudaSuccess) return fail(L2PD_ERR_OOM);
+    if (cudaMemcpy(c->cs_table_t, tab_t.data(), tab_t.size() * sizeof(float2), cudaMemcpyHostToDevice) != cudaSuccess)
+      return fail(L2PD_ERR_CUDA);
   }
   if (f.dtype == L2PD_BF16) {
     l2pd_status s1 = make_tma_2d_bf16(&c->ta_n, c->n, mr, d, 128);
@@ -481,6 +506,25 @@ l2pd_status l2pd_init(const l2pd_config *cfg, const l2pd_weights *w, int device,
       if (make_tma_2d_bf16(&c->ta_q, c->q, mr, hd, 128) || make_tma_2d_bf16(&c->t_kstore, c->kc, store_rows, hd, 128) ||
           make_tma_2d_bf16(&c->t_vstore, c->vc, store_rows, hd, 128))
         return fail(L2PD_ERR_CUDA);
+    }
+    const char *nf = getenv("L2PD_NO_ROPE_FUSION");
+    c->fuse_rope = c->attn_tc && !c->force_simt && f.kv_cache_mode == 0 && (f.head_dim & (f.head_dim - 1)) == 0 &&
+                   !(nf && nf[0] == '1');
+    if (c->fuse_rope) {
+      bf16 *qkvb = (bf16 *)c->qkv;
+      if (make_tma_2d_bf16_strided(&c->tq_packed, qkvb, mr, hd, 3 * hd, 128) ||
+          make_tma_2d_bf16_strided(&c->tk_packed, qkvb + hd, mr, hd, 3 * hd, 128) ||
+          make_tma_2d_bf16_strided(&c->tv_packed, qkvb + 2 * hd, mr, hd, 3 * hd, 128))
+        return fail(L2PD_ERR_CUDA);
+      for (int l = 0; l < f.n_layers; ++l) {
+        void *w = nullptr;
+        if (cudaMalloc(&w, (size_t)3 * hd * d * 2) != cudaSuccess) return fail(L2PD_ERR_OOM);
+        c->wqkv_perm.push_back(w);
+        if (launch_permute_qkv_rows(0, (const bf16 *)c->wqkv[l], (bf16 *)w, f.n_heads, f.head_dim, d) != cudaSuccess)
+          return fail(L2PD_ERR_CUDA);
+        c->wqkv[l] = w;   // the tensor maps of the QKV projection are encoded over the reordered copy
+      }
+      if (cudaDeviceSynchronize() != cudaSuccess) return fail(L2PD_ERR_CUDA);
     }
   }
   if (cudaEventCreate(&c->ev0) != cudaSuccess || cudaEventCreate(&c->ev1) != cudaSuccess) return fail(L2PD_ERR_CUDA);
@@ -764,7 +808,7 @@ l2pd_status l2pd_attention_bf16(void *stream, const void *q, const void *k, cons
     if (r) return r;
     r = make_tma_2d_bf16_strided(&tv, v, Tk, (int64_t)H * dh, kv_stride, 128);
     if (r) return r;
-    if (launch_attention_tc((cudaStream_t)stream, tq, tk, tv, nullptr, (bf16 *)out, out_stride, 0, 0, Tk, Tq, H, status) !=
+    if (launch_attention_tc((cudaStream_t)stream, tq, tk, tv, nullptr, (bf16 *)out, out_stride, 0, 0, 0, Tk, Tq, H, status) !=
         cudaSuccess)
       return L2PD_ERR_CUDA;
     return finish_standalone((cudaStream_t)stream, status, check);

@@ -45,6 +45,7 @@ struct AttnTcParams {
   float scale_log2;
   int kv_rows_per_seq;   // rows between two sequences in the key/value tensor maps
   int kv_row_base;       // first row of this layer's store in the key/value tensor maps
+  int kv_packed;         // keys / values are the packed activation rows: row = row0 of the sequence + key
   int32_t *status;
 };
 
@@ -112,7 +113,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
       ptx::mbar_arrive_expect_tx(bar(B_QFULL), TILE_BYTES);
       ptx::tma_load_2d_hint(sQ, &tmQ, bar(B_QFULL), h * DH, m.row0 + q0, pol);
       ptx::tma_load_2d_hint(sQ + HALF_BYTES, &tmQ, bar(B_QFULL), h * DH + 64, m.row0 + q0, pol);
-      const int krow = p.kv_row_base + m.seq * p.kv_rows_per_seq;
+      const int krow = p.kv_row_base + (p.kv_packed ? m.row0 : m.seq * p.kv_rows_per_seq);
       for (int j = 0; j < n_tiles && ok; ++j) {
         const int st = j & 1;
         const uint32_t ph = (j >> 1) & 1;
@@ -311,11 +312,11 @@ bool attention_tc_supported(int dh, int64_t q_stride, int64_t kv_row_stride, int
 
 cudaError_t launch_attention_tc(cudaStream_t st, const TmaDesc &tq, const TmaDesc &tk, const TmaDesc &tv,
                                 const SeqMeta *meta, bf16 *out, int64_t out_stride, int kv_rows_per_seq,
-                                int kv_row_base, int n_slots, int max_q_rows, int H, int32_t *status) {
+                                int kv_row_base, int kv_packed, int n_slots, int max_q_rows, int H, int32_t *status) {
   AttnTcParams p;
   p.out = out; p.meta = meta; p.use_single = 0; p.out_stride = out_stride;
   p.scale_log2 = 1.4426950408889634f / sqrtf((float)DH);
-  p.kv_rows_per_seq = kv_rows_per_seq; p.kv_row_base = kv_row_base; p.status = status;
+  p.kv_rows_per_seq = kv_rows_per_seq; p.kv_row_base = kv_row_base; p.kv_packed = kv_packed; p.status = status;
   if (meta == nullptr) {
     // stand-alone call: one sequence, max_q_rows queries, n_slots carries the key count
     p.use_single = 1;

@@ -90,14 +90,17 @@ template <typename T>
 cudaError_t launch_final_norm_gather(cudaStream_t st, const float *x, const SeqMeta *meta,
                                      const float *gain, float eps, T *nf, int n_slots, int s,
                                      int rows_padded, int d);
-cudaError_t launch_build_row_map(cudaStream_t st, const SeqMeta *meta, int n_slots, int32_t *row_slot);
+cudaError_t launch_build_row_map(cudaStream_t st, const SeqMeta *meta, int n_slots, int32_t *row_slot, int32_t *row_pos);
+// Library-owned copy of a QKV weight [3*H*dh, d] whose q and k rows are reordered inside each head so that the
+// rotary pair (i, i + dh/2) sits in adjacent rows (2i, 2i + 1); the v rows are copied as they are.
+cudaError_t launch_permute_qkv_rows(cudaStream_t st, const bf16 *src, bf16 *dst, int H, int dh, int d);
 cudaError_t launch_state_reset(cudaStream_t st, const int32_t *prompts, int B, int P, int G, int vocab,
                                int mask_id, int32_t *tokens, uint8_t *masked, SeqState s, int32_t *bad);
 cudaError_t launch_gather_response(cudaStream_t st, const int32_t *tokens, int B, int P, int G,
                                    int32_t *out);
 
 // simt.cu : CUDA-core GEMM and attention (fp32 configurations; also a bf16 cross-check path)
-enum { EPI_STORE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_STORE_F32 = 3, EPI_LMHEAD = 4 };
+enum { EPI_STORE = 0, EPI_RESIDUAL = 1, EPI_SWIGLU = 2, EPI_STORE_F32 = 3, EPI_LMHEAD = 4, EPI_QKV_ROPE = 5 };
 template <typename T>
 cudaError_t launch_simt_gemm(cudaStream_t st, int epi, const T *A, const T *W, const T *W2, void *C,
                              const float *bias, int M, int N, int K);
@@ -156,6 +159,9 @@ struct GemmArgs {
   // LM head
   const float *bias; float *part_m, *part_s; int32_t *part_i; int rows_padded; float *logits;
   int32_t *status;         // device status word
+  // EPI_QKV_ROPE: columns [0, rope_cols) are rotated in adjacent pairs (2i, 2i + 1) by the angle of pair
+  // ((column % dh) / 2) at the row's position; cs_table [dh/2][cs_stride] (cos, sin) indexed [pair][position], row_pos [M]
+  int rope_cols, rope_dh, cs_stride; const float2 *cs_table; const int32_t *row_pos;
 };
 cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms);
 cudaError_t launch_merge_partials(cudaStream_t st, const float *part_m, const float *part_s,
@@ -171,9 +177,10 @@ cudaError_t launch_attention_bf16(cudaStream_t st, const bf16 *q, const bf16 *kc
 
 // attention_tc.cu : head size 128 on tcgen05.  tq covers the packed query rows [rows, H*128], tk / tv the
 // key / value store as one matrix of rows (layer, sequence, position) x H*128; all with a box of 128 rows.
+// kv_packed != 0: keys and values lie in the packed activation rows instead (row = the sequence's row0 + key).
 bool attention_tc_supported(int dh, int64_t q_stride, int64_t kv_row_stride, int64_t out_stride);
 cudaError_t launch_attention_tc(cudaStream_t st, const TmaDesc &tq, const TmaDesc &tk, const TmaDesc &tv,
                                 const SeqMeta *meta, bf16 *out, int64_t out_stride, int kv_rows_per_seq,
-                                int kv_row_base, int n_slots, int max_q_rows, int H, int32_t *status);
+                                int kv_row_base, int kv_packed, int n_slots, int max_q_rows, int H, int32_t *status);
 
 }  // namespace l2pd

@@ -235,11 +235,28 @@ __global__ void final_norm_gather_kernel(const float *x, const SeqMeta *meta, co
   for (int i = threadIdx.x; i < d; i += blockDim.x) out[i] = from_f32<T>(xr[i] * gain[i] * inv);
 }
 
-__global__ void build_row_map_kernel(const SeqMeta *meta, int32_t *row_slot) {
+__global__ void build_row_map_kernel(const SeqMeta *meta, int32_t *row_slot, int32_t *row_pos) {
   grid_dep_launch();
   grid_dep_wait();
   SeqMeta m = meta[blockIdx.x];
-  for (int i = threadIdx.x; i < m.n_rows; i += blockDim.x) row_slot[m.row0 + i] = blockIdx.x;
+  for (int i = threadIdx.x; i < m.n_rows; i += blockDim.x) {
+    row_slot[m.row0 + i] = blockIdx.x;
+    row_pos[m.row0 + i] = m.pos0 + i;
+  }
+}
+
+// dst row (h, r) of the q and k parts = src row (h, r / 2 + (r odd ? dh / 2 : 0)); v rows unchanged
+__global__ void permute_qkv_rows_kernel(const bf16 *src, bf16 *dst, int H, int dh, int d) {
+  const int row = blockIdx.x;                 // destination row in [0, 3 * H * dh)
+  const int hd = H * dh;
+  int srow = row;
+  if (row < 2 * hd) {
+    const int part = row / hd, in = row - part * hd, h = in / dh, r = in - h * dh;
+    srow = part * hd + h * dh + (r >> 1) + ((r & 1) ? (dh >> 1) : 0);
+  }
+  const uint4 *s = reinterpret_cast<const uint4 *>(src + (int64_t)srow * d);
+  uint4 *t = reinterpret_cast<uint4 *>(dst + (int64_t)row * d);
+  for (int i = threadIdx.x; i < d / 8; i += blockDim.x) t[i] = s[i];
 }
 
 // Algorithm 2: X <- concat(prompt, [MASK]^G); all generation positions masked.
@@ -300,8 +317,12 @@ cudaError_t launch_final_norm_gather(cudaStream_t st, const float *x, const SeqM
                                      int rows_padded, int d) {
   return launch_kernel(final_norm_gather_kernel<T>, dim3(rows_padded), dim3(256), 0, st, x, meta, gain, eps, nf, n_slots, s, d);
 }
-cudaError_t launch_build_row_map(cudaStream_t st, const SeqMeta *meta, int n_slots, int32_t *row_slot) {
-  return launch_kernel(build_row_map_kernel, dim3(n_slots), dim3(256), 0, st, meta, row_slot);
+cudaError_t launch_build_row_map(cudaStream_t st, const SeqMeta *meta, int n_slots, int32_t *row_slot, int32_t *row_pos) {
+  return launch_kernel(build_row_map_kernel, dim3(n_slots), dim3(256), 0, st, meta, row_slot, row_pos);
+}
+cudaError_t launch_permute_qkv_rows(cudaStream_t st, const bf16 *src, bf16 *dst, int H, int dh, int d) {
+  permute_qkv_rows_kernel<<<3 * H * dh, 256, 0, st>>>(src, dst, H, dh, d);
+  return cudaGetLastError();
 }
 cudaError_t launch_state_reset(cudaStream_t st, const int32_t *prompts, int B, int P, int G, int vocab,
                                int mask_id, int32_t *tokens, uint8_t *masked, SeqState s, int32_t *bad) {

@@ -5,7 +5,9 @@
 // next tile's main loop.
 //
 // Epilogues
-//   EPI_STORE     C (bf16)  = acc                                   QKV projection
+//   EPI_STORE     C (bf16)  = acc                                   plain projection
+//   EPI_QKV_ROPE  C (bf16)  = acc, the q and k columns rotated by the row's position (RoPE): QKV
+//                 projection whose weight rows were reordered so that a rotary pair is two adjacent columns
 //   EPI_RESIDUAL  X (fp32) += acc                                   output / down projection
 //   EPI_SWIGLU    H (bf16)  = silu(acc_gate) * acc_up               gate/up projection; the B tile
 //                 holds tile_n/2 rows of W_gate followed by tile_n/2 rows of W_up
@@ -56,6 +58,9 @@ struct KParams {
   int out_tma;          // 1: the epilogue may stage its output in shared memory and store it through tmC
   int out_full_tiles;   // column tiles that lie wholly inside the row (the others use direct stores)
   int gate;             // 1: every unit's epilogue is staged; the producer keeps off the staging area meanwhile
+  int rope_cols, rope_dh, cs_stride;   // EPI_QKV_ROPE, see GemmArgs
+  const float2 *cs_table;
+  const int32_t *row_pos;
 };
 
 __device__ __forceinline__ void fail(int32_t *status, int code) {
@@ -115,6 +120,28 @@ __device__ __forceinline__ void emit_swiglu16(bf16 *dst, const uint32_t *g, cons
   }
 }
 
+// Rotary embedding on 32 (or 16) consecutive accumulator columns of one row, starting at the even column col0:
+// the pair (x1, x2) = columns (2t, 2t + 1) becomes (x1 cos - x2 sin, x2 cos + x1 sin), the angle being that of
+// pair index ((column % dh) / 2) at position pos.  Columns from rope_cols on (the v part) are left alone.
+__device__ __forceinline__ void rope_pairs(const KParams &p, uint32_t *v, int col0, int ncols, int pos) {
+  if (col0 >= p.rope_cols) return;               // a chunk of v columns (warp-uniform)
+  // the table is laid out [pair][position]: the 32 rows of a warp are consecutive positions, so a load is one line.
+  // All 16 angles are fetched before any is used.
+  const float2 *cs = p.cs_table + pos;
+  const int mask = p.rope_dh - 1;
+  float2 a[16];
+#pragma unroll
+  for (int t = 0; t < 16; ++t) a[t] = __ldg(cs + (int64_t)(((col0 + 2 * t) & mask) >> 1) * p.cs_stride);
+#pragma unroll
+  for (int t = 0; t < 16; ++t) {
+    if (2 * t < ncols && col0 + 2 * t < p.rope_cols) {
+      const float x1 = __uint_as_float(v[2 * t]), x2 = __uint_as_float(v[2 * t + 1]);
+      v[2 * t] = __float_as_uint(x1 * a[t].x - x2 * a[t].y);
+      v[2 * t + 1] = __float_as_uint(x2 * a[t].x + x1 * a[t].y);
+    }
+  }
+}
+
 // Drains one 128-row x tile_n accumulator from tensor memory (this warp's 32 lanes) and applies the
 // epilogue with per-thread stores (a thread owns one row).  The loads run one step ahead of the
 // arithmetic and stores: while chunk c is converted and written, chunk c + 1 is in flight
@@ -124,7 +151,8 @@ template <int EPI>
 __device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int row, int nt, bool atomic) {
   const bool row_ok = row < p.M;
   const int half_n = p.tile_n >> 1;
-  if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+  if (EPI == EPI_STORE || EPI == EPI_RESIDUAL || EPI == EPI_QKV_ROPE) {
+    const int pos = (EPI == EPI_QKV_ROPE && row_ok) ? p.row_pos[row] : 0;
     // 32 columns per step (tile_n is a multiple of 16: the last step may hold 16)
     const int n0 = nt * p.tile_n, n = p.tile_n;
     uint32_t va[32], vb[32];
@@ -132,13 +160,14 @@ __device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int
       if (n - c >= 32) ptx::tmem_ld_x32(taddr + c, v);
       else ptx::tmem_ld_x16(taddr + c, v);
     };
-    auto emit = [&](const uint32_t *v, int c) {
+    auto emit = [&](uint32_t *v, int c) {
       if (!row_ok) return;
+      if (EPI == EPI_QKV_ROPE) rope_pairs(p, v, n0 + c, min(32, n - c), pos);
 #pragma unroll
       for (int h16 = 0; h16 < 2; ++h16) {
         const int col = n0 + c + 16 * h16;
         if (c + 16 * h16 < n && col < p.N) {
-          if (EPI == EPI_STORE) emit_store16(reinterpret_cast<bf16 *>(p.out) + (int64_t)row * p.N + col, v + 16 * h16, p.N - col);
+          if (EPI != EPI_RESIDUAL) emit_store16(reinterpret_cast<bf16 *>(p.out) + (int64_t)row * p.N + col, v + 16 * h16, p.N - col);
           else emit_residual16(reinterpret_cast<float *>(p.out) + (int64_t)row * p.N + col, v + 16 * h16, atomic, p.N - col);
         }
       }
@@ -266,14 +295,16 @@ __device__ __forceinline__ void drain_tile_staged(const KParams &p, const CUtens
     __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(a), __uint_as_float(b));
     return *reinterpret_cast<uint32_t *>(&t);
   };
-  if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
+  if (EPI == EPI_STORE || EPI == EPI_RESIDUAL || EPI == EPI_QKV_ROPE) {
     const int n = p.tile_n;
+    const int pos = (EPI == EPI_QKV_ROPE && row0 + lane < p.M) ? p.row_pos[row0 + lane] : 0;
     uint32_t va[32], vb[32];
     auto load = [&](uint32_t *v, int c) {
       if (n - c >= 32) ptx::tmem_ld_x32(taddr + c, v);
       else ptx::tmem_ld_x16(taddr + c, v);
     };
-    auto emit = [&](const uint32_t *v, int c) {   // 32 columns starting at c (the upper 16 may lie beyond the tile)
+    auto emit = [&](uint32_t *v, int c) {   // 32 columns starting at c (the upper 16 may lie beyond the tile)
+      if (EPI == EPI_QKV_ROPE) rope_pairs(p, v, nt * n + c, min(32, n - c), pos);
       if (EPI == EPI_RESIDUAL) {
         reuse();
 #pragma unroll
@@ -813,6 +844,9 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
   }
   p.out = g.out; p.bias = g.bias; p.part_m = g.part_m; p.part_s = g.part_s; p.part_i = g.part_i;
   p.rows_padded = g.rows_padded; p.logits = g.logits; p.status = g.status;
+  p.rope_cols = g.rope_cols; p.rope_dh = g.rope_dh; p.cs_stride = g.cs_stride; p.cs_table = g.cs_table; p.row_pos = g.row_pos;
+  if (g.epi == EPI_QKV_ROPE && (!g.cs_table || !g.row_pos || g.rope_dh < 2 || (g.rope_dh & (g.rope_dh - 1)) || (g.rope_cols % g.rope_dh)))
+    return cudaErrorInvalidValue;
   const int units = p.m_tiles * p.n_tiles * ks;
   if (units <= 0) return cudaSuccess;
   const int groups = num_sms / cg;
@@ -829,6 +863,7 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
   if (cg == 1) {
     switch (g.epi) {
       case EPI_STORE: L2PD_LAUNCH(gemm_tcgen05_kernel, EPI_STORE) break;
+      case EPI_QKV_ROPE: L2PD_LAUNCH(gemm_tcgen05_kernel, EPI_QKV_ROPE) break;
       case EPI_RESIDUAL: L2PD_LAUNCH(gemm_tcgen05_kernel, EPI_RESIDUAL) break;
       case EPI_SWIGLU: L2PD_LAUNCH(gemm_tcgen05_kernel, EPI_SWIGLU) break;
       case EPI_LMHEAD: L2PD_LAUNCH(gemm_tcgen05_kernel, EPI_LMHEAD) break;
@@ -837,6 +872,7 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
   } else {
     switch (g.epi) {
       case EPI_STORE: L2PD_LAUNCH(gemm_tcgen05_pair_kernel, EPI_STORE) break;
+      case EPI_QKV_ROPE: L2PD_LAUNCH(gemm_tcgen05_pair_kernel, EPI_QKV_ROPE) break;
       case EPI_RESIDUAL: L2PD_LAUNCH(gemm_tcgen05_pair_kernel, EPI_RESIDUAL) break;
       case EPI_SWIGLU: L2PD_LAUNCH(gemm_tcgen05_pair_kernel, EPI_SWIGLU) break;
       default: return cudaErrorInvalidValue;
