@@ -60,6 +60,10 @@ struct l2pd_ctx {
   StepSummary *d_summary = nullptr, *h_summary = nullptr;
   int32_t *d_status = nullptr, *h_status = nullptr;
   float2 *cs_table = nullptr;
+  // partial sums of the K slices of the O and down projections, [4][ksum_rows][d] fp32: summed in slice order by the
+  // RMSNorm that follows (bit-reproducible, unlike additions into x in completion order)
+  float *ksum = nullptr;
+  int64_t ksum_rows = 0;
   float2 *cs_table_t = nullptr;      // the same table as [pair][position] (fused rotation in the QKV epilogue)
 
   // TMA descriptors (bf16 path)
@@ -186,9 +190,12 @@ l2pd_status run_gemm_simt(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const 
   return L2PD_OK;
 }
 
+int64_t round_up(int64_t a, int64_t b);
+
 l2pd_status run_gemm_tc(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const TmaDesc *a, const TmaDesc *b,
                         const TmaDesc *b2, const TmaDesc *cm, void *out, int M, int N, int K, const GemmPlan &pl) {
   GemmArgs g{};
+  if (epi == EPI_RESIDUAL && c->ksum && effective_k_splits(K, pl.k_splits) > 1) { g.part = c->ksum; g.part_rows = (int)round_up(M, 512); }
   g.epi = epi; g.a = a; g.b = b; g.b2 = b2; g.c = cm; g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.out = out;
   g.cta_group = pl.cta_group; g.k_splits = pl.k_splits; g.slabs = pl.slabs;
   g.status = c->d_status;
@@ -214,10 +221,11 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     c->pl_qkv = plan_gemm(EPI_STORE, T_rows, 3 * hd, d, c->num_sms, 0);
     int box = c->pl_qkv.tile_n / c->pl_qkv.cta_group;
     if (box != c->box_qkv) { l2pd_status r = encode_weight_maps(c, c->tb_qkv, c->wqkv, 3 * hd, d, box); if (r) return r; c->box_qkv = box; }
-    c->pl_o = plan_gemm(EPI_RESIDUAL, T_rows, d, hd, c->num_sms, 0);
+    const int max_ks = (c->ksum == nullptr || T_rows <= c->ksum_rows) ? 4 : 1;   // K slices need their partial-sum area
+    c->pl_o = plan_gemm(EPI_RESIDUAL, T_rows, d, hd, c->num_sms, 0, max_ks);
     box = c->pl_o.tile_n / c->pl_o.cta_group;
     if (box != c->box_o) { l2pd_status r = encode_weight_maps(c, c->tb_o, c->wo, d, hd, box); if (r) return r; c->box_o = box; }
-    c->pl_down = plan_gemm(EPI_RESIDUAL, T_rows, d, F, c->num_sms, 0);
+    c->pl_down = plan_gemm(EPI_RESIDUAL, T_rows, d, F, c->num_sms, 0, max_ks);
     box = c->pl_down.tile_n / c->pl_down.cta_group;
     if (box != c->box_down) { l2pd_status r = encode_weight_maps(c, c->tb_down, c->w_down, d, F, box); if (r) return r; c->box_down = box; }
     c->pl_gu = plan_gemm(EPI_SWIGLU, T_rows, F, d, c->num_sms, 0);
@@ -238,9 +246,21 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     };
     if (c->tc_rows != T_rows) { c->tcw_qkv = c->tcw_o = c->tcw_h = c->tcw_down = 0; }
     l2pd_status r = out_map(c->tc_qkv, c->tcw_qkv, c->qkv, false, 3 * hd, c->pl_qkv.tile_n); if (r) return r;
-    r = out_map(c->tc_o, c->tcw_o, c->x, true, d, c->pl_o.tile_n); if (r) return r;
+    // K-split projections store per-slice partial sums: their map covers [slices * rows rounded up to a whole unit][d] of ksum
+    const int ks_o = c->ksum ? effective_k_splits(hd, c->pl_o.k_splits) : 1, ks_d = c->ksum ? effective_k_splits(F, c->pl_down.k_splits) : 1;
+    const int64_t mpad = round_up(T_rows, 512);
+    auto out_map_x = [&](TmaDesc &m, int &w_have, int ks, int w) -> l2pd_status {
+      if (ks <= 1) return out_map(m, w_have, c->x, true, d, w);
+      if ((w_have == w || w_have == -w) && c->tc_rows == T_rows) return L2PD_OK;
+      if (d < w) { w_have = -w; return L2PD_OK; }
+      l2pd_status r2 = make_tma_out_3d(&m, c->ksum, true, ks * mpad, d, w);
+      if (r2) return set_err(c, r2, "output tensor map encode failed (partial sums, tile %d)", w);
+      w_have = w;
+      return L2PD_OK;
+    };
+    r = out_map_x(c->tc_o, c->tcw_o, ks_o, c->pl_o.tile_n); if (r) return r;
     r = out_map(c->tc_h, c->tcw_h, c->h, false, F, c->pl_gu.tile_n / 2); if (r) return r;
-    r = out_map(c->tc_down, c->tcw_down, c->x, true, d, c->pl_down.tile_n); if (r) return r;
+    r = out_map_x(c->tc_down, c->tcw_down, ks_d, c->pl_down.tile_n); if (r) return r;
     c->tc_rows = T_rows;
   }
 
@@ -274,16 +294,29 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_O, EPI_RESIDUAL, &c->ta_att, &c->tb_o[l], nullptr, c->tcw_o > 0 ? &c->tc_o : nullptr, c->x, T_rows, d, hd, c->pl_o);
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_O, EPI_RESIDUAL, att, c->wo[l], nullptr, c->x, nullptr, T_rows, d, hd);
     if (r) return r;
-    CKLK(L2PD_K_RMSNORM, launch_rmsnorm<T>(s, c->x, c->norm2[l], f.rms_eps, n, T_rows, d));
+    {
+      const int ks = (tc && c->ksum) ? effective_k_splits(hd, c->pl_o.k_splits) : 1;
+      CKLK(L2PD_K_RMSNORM, launch_rmsnorm<T>(s, c->x, c->norm2[l], f.rms_eps, n, T_rows, d, c->ksum, ks > 1 ? ks : 0,
+                                            (int64_t)round_up(T_rows, 512) * d));
+    }
     if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_GATE_UP, EPI_SWIGLU, &c->ta_n, &c->tb_gate[l], &c->tb_up[l], c->tcw_h > 0 ? &c->tc_h : nullptr, hbuf, T_rows, F, d, c->pl_gu);
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_GATE_UP, EPI_SWIGLU, n, c->w_gate[l], c->w_up[l], hbuf, nullptr, T_rows, F, d);
     if (r) return r;
     if (tc) r = run_gemm_tc(c, s, L2PD_K_GEMM_DOWN, EPI_RESIDUAL, &c->ta_h, &c->tb_down[l], nullptr, c->tcw_down > 0 ? &c->tc_down : nullptr, c->x, T_rows, d, F, c->pl_down);
     else r = run_gemm_simt<T>(c, s, L2PD_K_GEMM_DOWN, EPI_RESIDUAL, hbuf, c->w_down[l], nullptr, c->x, nullptr, T_rows, d, F);
     if (r) return r;
+    // the down projection's K slices: summed by the next layer's RMSNorm, or right here when x is read by something else
+    int ks_pend = (tc && c->ksum) ? effective_k_splits(F, c->pl_down.k_splits) : 1;
+    const int64_t ks_stride = (int64_t)round_up(T_rows, 512) * d;
+    if (ks_pend > 1 && (c->cap || l + 1 == f.n_layers)) {
+      CKLK(L2PD_K_OTHER, launch_add_partials(s, c->x, c->ksum, ks_pend, ks_stride, T_rows, d));
+      ks_pend = 1;
+    }
     if (c->cap)
       CK(cudaMemcpyAsync(c->cap + (int64_t)(l + 1) * c->cap_stride, c->x, (size_t)T_rows * d * 4, cudaMemcpyDeviceToDevice, s));
-    if (l + 1 < f.n_layers) CKLK(L2PD_K_RMSNORM, launch_rmsnorm<T>(s, c->x, c->norm1[l + 1], f.rms_eps, n, T_rows, d));
+    if (l + 1 < f.n_layers)
+      CKLK(L2PD_K_RMSNORM, launch_rmsnorm<T>(s, c->x, c->norm1[l + 1], f.rms_eps, n, T_rows, d, c->ksum, ks_pend > 1 ? ks_pend : 0,
+                                            ks_stride));
   }
 
   // confidence head on the current block's rows
@@ -348,7 +381,7 @@ void free_all(l2pd_ctx *c) {
   cudaFree(c->x); cudaFree(c->n); cudaFree(c->qkv); cudaFree(c->q); cudaFree(c->att); cudaFree(c->h); cudaFree(c->nf);
   cudaFree(c->kc); cudaFree(c->vc); cudaFree(c->part); cudaFree(c->logits_f32);
   for (void *w : c->wqkv_perm) cudaFree(w);
-  cudaFree(c->d_row_pos); cudaFree(c->cs_table_t);
+  cudaFree(c->d_row_pos); cudaFree(c->cs_table_t); cudaFree(c->ksum);
   cudaFree(c->d_meta); cudaFree(c->d_row_slot); cudaFree(c->d_summary); cudaFree(c->d_status); cudaFree(c->cs_table);
   if (c->h_meta) cudaFreeHost(c->h_meta);
   if (c->h_summary) cudaFreeHost(c->h_summary);
@@ -452,6 +485,12 @@ l2pd_status l2pd_init(const l2pd_config *cfg, const l2pd_weights *w, int device,
   A(dev_alloc(c, &c->d_meta, (int64_t)f.max_batch));
   A(dev_alloc(c, &c->d_row_slot, mr));
   A(dev_alloc(c, &c->d_row_pos, mr));
+  // L2PD_ATOMIC_KSPLIT=1: no partial-sum area; K slices add into x in completion order (not bit-reproducible)
+  const char *ak = getenv("L2PD_ATOMIC_KSPLIT");
+  if (f.dtype == L2PD_BF16 && !(ak && ak[0] == '1')) {
+    c->ksum_rows = round_up(mr < 4096 ? mr : 4096, 512);   // a slice's area covers whole 512-row units
+    A(dev_alloc(c, &c->ksum, 4 * c->ksum_rows * d));
+  }
   A(dev_alloc(c, &c->d_summary, (int64_t)f.max_batch));
   A(dev_alloc(c, &c->d_status, (int64_t)1));
   A(dev_alloc(c, &c->cs_table, (int64_t)f.max_seq * (f.head_dim / 2)));

@@ -79,9 +79,13 @@ template <typename T>
 cudaError_t launch_embed_rmsnorm(cudaStream_t st, const int32_t *tokens, int64_t tok_stride,
                                  const SeqMeta *meta, const int32_t *row_slot, const T *emb,
                                  const float *gain, float eps, float *x, T *n, int rows, int d);
+// n = RMSNorm(x).  With n_part > 0, first x += part[0] + part[1] + ... (slice s at part + s * part_stride elements,
+// added in that order) and x is written back: the fixed-order end of a K-split projection.
 template <typename T>
-cudaError_t launch_rmsnorm(cudaStream_t st, const float *x, const float *gain, float eps, T *n,
-                           int rows, int d);
+cudaError_t launch_rmsnorm(cudaStream_t st, float *x, const float *gain, float eps, T *n,
+                           int rows, int d, const float *part = nullptr, int n_part = 0, int64_t part_stride = 0);
+// x += part[0] + part[1] + ... alone (where no RMSNorm follows directly)
+cudaError_t launch_add_partials(cudaStream_t st, float *x, const float *part, int n_part, int64_t part_stride, int rows, int d);
 template <typename T>
 cudaError_t launch_rope_scatter(cudaStream_t st, const T *qkv, const SeqMeta *meta,
                                 const int32_t *row_slot, const float2 *cs_table, T *q, T *kc, T *vc,
@@ -147,7 +151,8 @@ int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile);
 // drain is not overlapped with the next unit).
 // The B tensor map's box must be tile_n / cta_group rows (SwiGLU: tile_n / 2 for either group size).
 struct GemmPlan { int cta_group, tile_n, k_splits, slabs; };
-GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n);
+GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, int max_k_splits = 4);
+int effective_k_splits(int K, int k_splits);   // what the launcher makes of a requested K split
 struct GemmArgs {
   int epi;                 // EPI_STORE, EPI_RESIDUAL, EPI_SWIGLU, or EPI_LMHEAD
   const TmaDesc *a, *b, *b2;
@@ -159,6 +164,10 @@ struct GemmArgs {
   // LM head
   const float *bias; float *part_m, *part_s; int32_t *part_i; int rows_padded; float *logits;
   int32_t *status;         // device status word
+  // EPI_RESIDUAL with k_splits > 1 and part != null: instead of adding into `out`, slice s stores its partial sums
+  // at part[(s * part_rows + row) * N + col] (part_rows >= M rounded up to 512, a whole unit of rows; `c`, if given, must map that area);
+  // whoever reads X next adds them in slice order (launch_rmsnorm / launch_add_partials): bit-reproducible
+  float *part; int part_rows;
   // EPI_QKV_ROPE: columns [0, rope_cols) are rotated in adjacent pairs (2i, 2i + 1) by the angle of pair
   // ((column % dh) / 2) at the row's position; cs_table [dh/2][cs_stride] (cos, sin) indexed [pair][position], row_pos [M]
   int rope_cols, rope_dh, cs_stride; const float2 *cs_table; const int32_t *row_pos;

@@ -57,25 +57,39 @@ __device__ __forceinline__ void store4(bf16 *p, float a, float b, float c, float
 }
 
 // One block per row; rows up to 4 * 4 * blockDim floats stay in registers between the two passes.
+// n_part > 0: the row first takes in the partial sums of a K-split projection, slice after slice, and
+// the summed row is written back to x.
 template <typename T>
-__global__ void __launch_bounds__(256) rmsnorm_kernel(const float *x, const float *gain, float eps, T *n, int d) {
+__global__ void __launch_bounds__(256) rmsnorm_kernel(float *x, const float *gain, float eps, T *n, int d,
+                                                      const float *part, int n_part, int64_t part_stride) {
   grid_dep_launch();
   grid_dep_wait();
   __shared__ float red[32];
   const int row = blockIdx.x;
-  const float4 *xr = reinterpret_cast<const float4 *>(x + (int64_t)row * d);
+  float4 *xr = reinterpret_cast<float4 *>(x + (int64_t)row * d);
   const int d4 = d >> 2;
   constexpr int CACHE = 4;
   float4 v[CACHE];
   float ss = 0.f;
+  auto fetch = [&](int i) {
+    float4 w = xr[i];
+    if (n_part > 0) {
+      for (int s = 0; s < n_part; ++s) {
+        const float4 q = reinterpret_cast<const float4 *>(part + s * part_stride + (int64_t)row * d)[i];
+        w.x += q.x; w.y += q.y; w.z += q.z; w.w += q.w;
+      }
+      xr[i] = w;
+    }
+    return w;
+  };
 #pragma unroll
   for (int k = 0; k < CACHE; ++k) {
     const int i = threadIdx.x + k * blockDim.x;
-    v[k] = (i < d4) ? xr[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    v[k] = (i < d4) ? fetch(i) : make_float4(0.f, 0.f, 0.f, 0.f);
     ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
   }
   for (int i = threadIdx.x + CACHE * blockDim.x; i < d4; i += blockDim.x) {
-    float4 w = xr[i];
+    float4 w = fetch(i);
     ss += w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w;
   }
   const float tot = block_sum(ss, red);
@@ -91,9 +105,23 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float *x, const floa
     }
   }
   for (int i = threadIdx.x + CACHE * blockDim.x; i < d4; i += blockDim.x) {
-    const float4 w = xr[i];
+    const float4 w = xr[i];          // already summed and written back above, by this same thread
     const float4 g = g4[i];
     store4(nr + 4 * i, w.x * g.x * inv, w.y * g.y * inv, w.z * g.z * inv, w.w * g.w * inv);
+  }
+}
+
+__global__ void __launch_bounds__(256) add_partials_kernel(float *x, const float *part, int n_part, int64_t part_stride,
+                                                           int64_t n4) {
+  grid_dep_launch();
+  grid_dep_wait();
+  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+    float4 w = reinterpret_cast<float4 *>(x)[i];
+    for (int s = 0; s < n_part; ++s) {
+      const float4 q = reinterpret_cast<const float4 *>(part + s * part_stride)[i];
+      w.x += q.x; w.y += q.y; w.z += q.z; w.w += q.w;
+    }
+    reinterpret_cast<float4 *>(x)[i] = w;
   }
 }
 
@@ -297,9 +325,14 @@ cudaError_t launch_embed_rmsnorm(cudaStream_t st, const int32_t *tokens, int64_t
   return launch_kernel(embed_rmsnorm_kernel<T>, dim3(rows), dim3(256), 0, st, tokens, tok_stride, meta, row_slot, emb, gain, eps, x, n, d);
 }
 template <typename T>
-cudaError_t launch_rmsnorm(cudaStream_t st, const float *x, const float *gain, float eps, T *n,
-                           int rows, int d) {
-  return launch_kernel(rmsnorm_kernel<T>, dim3(rows), dim3(256), 0, st, x, gain, eps, n, d);
+cudaError_t launch_rmsnorm(cudaStream_t st, float *x, const float *gain, float eps, T *n,
+                           int rows, int d, const float *part, int n_part, int64_t part_stride) {
+  return launch_kernel(rmsnorm_kernel<T>, dim3(rows), dim3(256), 0, st, x, gain, eps, n, d, part, n_part, part_stride);
+}
+cudaError_t launch_add_partials(cudaStream_t st, float *x, const float *part, int n_part, int64_t part_stride, int rows, int d) {
+  const int64_t n4 = (int64_t)rows * d / 4;
+  const int grid = (int)((n4 + 255) / 256 < 2048 ? (n4 + 255) / 256 : 2048);
+  return launch_kernel(add_partials_kernel, dim3(grid), dim3(256), 0, st, x, part, n_part, part_stride, n4);
 }
 template <typename T>
 cudaError_t launch_rope_scatter(cudaStream_t st, const T *qkv, const SeqMeta *meta,
@@ -337,8 +370,8 @@ cudaError_t launch_gather_response(cudaStream_t st, const int32_t *tokens, int B
   template cudaError_t launch_embed_rmsnorm<T>(cudaStream_t, const int32_t *, int64_t,               \
                                                const SeqMeta *, const int32_t *, const T *,          \
                                                const float *, float, float *, T *, int, int);        \
-  template cudaError_t launch_rmsnorm<T>(cudaStream_t, const float *, const float *, float, T *,     \
-                                         int, int);                                                  \
+  template cudaError_t launch_rmsnorm<T>(cudaStream_t, float *, const float *, float, T *,           \
+                                         int, int, const float *, int, int64_t);                     \
   template cudaError_t launch_rope_scatter<T>(cudaStream_t, const T *, const SeqMeta *,              \
                                               const int32_t *, const float2 *, T *, T *, T *,        \
                                               int64_t, int, int, int);                               \

@@ -58,6 +58,7 @@ struct KParams {
   int out_tma;          // 1: the epilogue may stage its output in shared memory and store it through tmC
   int out_full_tiles;   // column tiles that lie wholly inside the row (the others use direct stores)
   int gate;             // 1: every unit's epilogue is staged; the producer keeps off the staging area meanwhile
+  float *part; int part_rows;      // EPI_RESIDUAL with K slices: slice s stores its partial sums at part[s * part_rows + row][N]
   int rope_cols, rope_dh, cs_stride;   // EPI_QKV_ROPE, see GemmArgs
   const float2 *cs_table;
   const int32_t *row_pos;
@@ -86,11 +87,15 @@ __device__ __forceinline__ void emit_store16(bf16 *dst, const uint32_t *v, int v
     *reinterpret_cast<uint4 *>(dst + hseg * 8) = pk;
   }
 }
-__device__ __forceinline__ void emit_residual16(float *px, const uint32_t *v, bool atomic, int valid) {
+// mode 0: x += acc (read-modify-write), 1: atomic x += acc, 2: plain store (a K slice's partial sums)
+__device__ __forceinline__ void emit_residual16(float *px, const uint32_t *v, int mode, int valid) {
 #pragma unroll
   for (int g = 0; g < 4; ++g) {
     if (g * 4 >= valid) break;
-    if (atomic) {
+    if (mode == 2) {
+      *reinterpret_cast<float4 *>(px + 4 * g) = make_float4(__uint_as_float(v[4 * g + 0]), __uint_as_float(v[4 * g + 1]),
+                                                            __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3]));
+    } else if (mode == 1) {
       ptx::red_add_v4(px + 4 * g, __uint_as_float(v[4 * g + 0]), __uint_as_float(v[4 * g + 1]),
                       __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3]));
     } else {
@@ -146,9 +151,10 @@ __device__ __forceinline__ void rope_pairs(const KParams &p, uint32_t *v, int co
 // epilogue with per-thread stores (a thread owns one row).  The loads run one step ahead of the
 // arithmetic and stores: while chunk c is converted and written, chunk c + 1 is in flight
 // (tcgen05.wait::ld covers every load issued so far).
-// `atomic` (split-K residual): the partial sum is added to X with a vector reduction.
+// K slices of the residual epilogue either add into X (`res_mode` 1) or store their partial sums to
+// `res_base`, the slice's own [rows][N] area (`res_mode` 2), for a later fixed-order sum.
 template <int EPI>
-__device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int row, int nt, bool atomic) {
+__device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int row, int nt, int res_mode, float *res_base) {
   const bool row_ok = row < p.M;
   const int half_n = p.tile_n >> 1;
   if (EPI == EPI_STORE || EPI == EPI_RESIDUAL || EPI == EPI_QKV_ROPE) {
@@ -168,7 +174,7 @@ __device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int
         const int col = n0 + c + 16 * h16;
         if (c + 16 * h16 < n && col < p.N) {
           if (EPI != EPI_RESIDUAL) emit_store16(reinterpret_cast<bf16 *>(p.out) + (int64_t)row * p.N + col, v + 16 * h16, p.N - col);
-          else emit_residual16(reinterpret_cast<float *>(p.out) + (int64_t)row * p.N + col, v + 16 * h16, atomic, p.N - col);
+          else emit_residual16(res_base + (int64_t)row * p.N + col, v + 16 * h16, res_mode, p.N - col);
         }
       }
     };
@@ -265,7 +271,7 @@ __device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int
 constexpr int STAGE_BUFS = 2;
 template <int EPI>
 __device__ __forceinline__ void drain_tile_staged(const KParams &p, const CUtensorMap *tmC, uint32_t taddr, int row0,
-                                                  int nt, uint32_t stage0, int lane) {
+                                                  int nt, uint32_t stage0, int lane, bool res_store) {
   const int half_n = p.tile_n >> 1;
   const uint32_t sw = (uint32_t)(lane & 7);
   int n_flush = 0;                       // staging tiles handed over so far; the current one is n_flush % STAGE_BUFS
@@ -278,7 +284,7 @@ __device__ __forceinline__ void drain_tile_staged(const KParams &p, const CUtens
     ptx::fence_proxy_async();
     __syncwarp();
     if (lane == 0) {
-      if (EPI == EPI_RESIDUAL) ptx::tma_reduce_add_3d(tmC, stage, c0, nt, row0);
+      if (EPI == EPI_RESIDUAL && !res_store) ptx::tma_reduce_add_3d(tmC, stage, c0, nt, row0);
       else ptx::tma_store_3d(tmC, stage, c0, nt, row0);
       ptx::bulk_commit();
     }
@@ -435,9 +441,11 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
   // group_m row tiles; inside a group the row tiles of one column tile are adjacent, then the next
   // column tile follows.  The CTAs running at the same time thus share a few weight tiles, and a
   // group's activation rows (sized to a fraction of L2) stay resident while its column tiles stream by.
+  int unit_ks = 0;   // K slice of the unit decoded last
   auto decode = [&](int u, int &mt, int &nt, int &kb0, int &kb1) {
     const int per_slice = p.m_tiles * p.n_tiles;
     const int ks = u / per_slice;
+    unit_ks = ks;
     const int r = u - ks * per_slice;
     const int per_group = p.group_m * p.n_tiles;
     const int g = r / per_group;
@@ -613,10 +621,14 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
       // the staging area is idle in a CTA's last unit (every load consumed, every MMA complete, in both
       // CTAs of a pair), and in earlier units when the producer is kept off it (p.gate)
       const bool last_unit = u + n_groups >= num_units;
+      const bool res_store = EPI == EPI_RESIDUAL && p.part != nullptr && p.k_splits > 1;
+      const int slice_row0 = res_store ? unit_ks * p.part_rows : 0;   // partial sums: the slice's own rows
       if (EPI != EPI_LMHEAD && p.out_tma && nt < p.out_full_tiles && (last_unit || p.gate))
-        drain_tile_staged<EPI>(p, tmC, taddr, row0, nt, sOut + (uint32_t)(warp - 3) * (4096u * STAGE_BUFS), lane);
+        drain_tile_staged<EPI>(p, tmC, taddr, slice_row0 + row0, nt, sOut + (uint32_t)(warp - 3) * (4096u * STAGE_BUFS), lane,
+                               res_store);
       else
-        drain_tile<EPI>(p, taddr, row0 + lane, nt, p.k_splits > 1);
+        drain_tile<EPI>(p, taddr, row0 + lane, nt, res_store ? 2 : (p.k_splits > 1 ? 1 : 0),
+                        res_store ? p.part + (int64_t)slice_row0 * p.N : reinterpret_cast<float *>(p.out));
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) {
@@ -774,12 +786,13 @@ static double plan_cost(int M, int N, int K, int num_sms, int cg, int slabs, int
   const double per_kb = fmax(fmax(2.0 * tile_n * slabs, 620.0), bytes / INGEST) * 1.06;
   // emptying the accumulators: bf16 stores leave an SM at ~34 B per cycle; fp32 additions into X are bound
   // by L2's atomic units, ~2500 B per cycle for the whole chip, i.e. ~17 B per cycle and SM when all drain at once
-  const double drain = (double)TILE_M * slabs * unit_n * (is_residual ? 4.0 / 17.0 : 2.0 / 34.0) + 1500.0;
+  // (K slices store their partial sums plainly: twice the rate of the additions)
+  const double drain = (double)TILE_M * slabs * unit_n * (is_residual ? (ks > 1 ? 4.0 / 34.0 : 4.0 / 17.0) : 2.0 / 34.0) + 1500.0;
   const double exposed = slabs == 2 ? drain : 0.3 * drain;
   return waves * (kb * per_kb + 6000.0 + exposed) + (slabs == 2 ? 0.0 : 0.7 * drain);
 }
 
-GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n) {
+GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, int max_k_splits) {
   GemmPlan best{1, 256, 1, 1};
   double best_cost = 1e300;
   const bool swiglu = epi == EPI_SWIGLU;
@@ -792,7 +805,7 @@ GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n) 
       for (int tn = 256; tn >= 64; tn -= step) {
         if (force_tile_n && tn != force_tile_n) continue;
         const int unit_n = swiglu ? tn / 2 : tn;
-        const int max_ks = (epi == EPI_RESIDUAL) ? 4 : 1;
+        const int max_ks = (epi == EPI_RESIDUAL) ? (max_k_splits < 4 ? max_k_splits : 4) : 1;
         for (int ks = 1; ks <= max_ks; ++ks) {
           if (ceil_div(K, TILE_K) < 8 * ks) break;
           const double c = plan_cost(M, N, K, num_sms, cg, slabs, unit_n, tn, ks, epi == EPI_RESIDUAL);
@@ -810,14 +823,18 @@ int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile) {
   return plan_gemm(EPI_LMHEAD, M, N, 4096, num_sms, 0).tile_n;
 }
 
+int effective_k_splits(int K, int k_splits) {
+  // every K slice must hold at least one k-block (an empty slice would add an unwritten accumulator)
+  int ks = k_splits > 1 ? k_splits : 1;
+  const int num_kb = ceil_div(K, TILE_K);
+  while (ks > 1 && ceil_div(num_kb, ks) * (ks - 1) >= num_kb) --ks;
+  return ks;
+}
+
 cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms) {
   const int cg = g.cta_group == 2 ? 2 : 1;
-  int ks = g.k_splits > 1 ? g.k_splits : 1;
-  if (ks > 1 && g.epi != EPI_RESIDUAL) return cudaErrorInvalidValue;
-  {   // every K slice must hold at least one k-block (an empty slice would add an unwritten accumulator)
-    const int num_kb = ceil_div(g.K, TILE_K);
-    while (ks > 1 && ceil_div(num_kb, ks) * (ks - 1) >= num_kb) --ks;
-  }
+  if (g.k_splits > 1 && g.epi != EPI_RESIDUAL) return cudaErrorInvalidValue;
+  const int ks = effective_k_splits(g.K, g.k_splits);
   KParams p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.tile_n = g.tile_n;
   p.b_stage_bytes = g.tile_n * 128 / cg;
@@ -844,6 +861,7 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
   }
   p.out = g.out; p.bias = g.bias; p.part_m = g.part_m; p.part_s = g.part_s; p.part_i = g.part_i;
   p.rows_padded = g.rows_padded; p.logits = g.logits; p.status = g.status;
+  p.part = g.part; p.part_rows = g.part_rows;
   p.rope_cols = g.rope_cols; p.rope_dh = g.rope_dh; p.cs_stride = g.cs_stride; p.cs_table = g.cs_table; p.row_pos = g.row_pos;
   if (g.epi == EPI_QKV_ROPE && (!g.cs_table || !g.row_pos || g.rope_dh < 2 || (g.rope_dh & (g.rope_dh - 1)) || (g.rope_cols % g.rope_dh)))
     return cudaErrorInvalidValue;
