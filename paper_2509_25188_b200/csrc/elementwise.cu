@@ -59,9 +59,10 @@ __device__ __forceinline__ void store4(bf16 *p, float a, float b, float c, float
 // One block per row; rows up to 4 * 4 * blockDim floats stay in registers between the two passes.
 // n_part > 0: the row first takes in the partial sums of a K-split projection, slice after slice, and
 // the summed row is written back to x.
-template <typename T>
+// NPART is a compile-time count so that all loads of a row chunk are issued before the first addition.
+template <typename T, int NPART>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(float *x, const float *gain, float eps, T *n, int d,
-                                                      const float *part, int n_part, int64_t part_stride) {
+                                                      const float *part, int64_t part_stride) {
   grid_dep_launch();
   grid_dep_wait();
   __shared__ float red[32];
@@ -73,11 +74,12 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(float *x, const float *gai
   float ss = 0.f;
   auto fetch = [&](int i) {
     float4 w = xr[i];
-    if (n_part > 0) {
-      for (int s = 0; s < n_part; ++s) {
-        const float4 q = reinterpret_cast<const float4 *>(part + s * part_stride + (int64_t)row * d)[i];
-        w.x += q.x; w.y += q.y; w.z += q.z; w.w += q.w;
-      }
+    if (NPART > 0) {
+      float4 q[NPART > 0 ? NPART : 1];
+#pragma unroll
+      for (int s = 0; s < NPART; ++s) q[s] = reinterpret_cast<const float4 *>(part + s * part_stride + (int64_t)row * d)[i];
+#pragma unroll
+      for (int s = 0; s < NPART; ++s) { w.x += q[s].x; w.y += q[s].y; w.z += q[s].z; w.w += q[s].w; }
       xr[i] = w;
     }
     return w;
@@ -327,7 +329,13 @@ cudaError_t launch_embed_rmsnorm(cudaStream_t st, const int32_t *tokens, int64_t
 template <typename T>
 cudaError_t launch_rmsnorm(cudaStream_t st, float *x, const float *gain, float eps, T *n,
                            int rows, int d, const float *part, int n_part, int64_t part_stride) {
-  return launch_kernel(rmsnorm_kernel<T>, dim3(rows), dim3(256), 0, st, x, gain, eps, n, d, part, n_part, part_stride);
+  switch (n_part) {
+    case 0: return launch_kernel(rmsnorm_kernel<T, 0>, dim3(rows), dim3(256), 0, st, x, gain, eps, n, d, part, part_stride);
+    case 2: return launch_kernel(rmsnorm_kernel<T, 2>, dim3(rows), dim3(256), 0, st, x, gain, eps, n, d, part, part_stride);
+    case 3: return launch_kernel(rmsnorm_kernel<T, 3>, dim3(rows), dim3(256), 0, st, x, gain, eps, n, d, part, part_stride);
+    case 4: return launch_kernel(rmsnorm_kernel<T, 4>, dim3(rows), dim3(256), 0, st, x, gain, eps, n, d, part, part_stride);
+    default: return cudaErrorInvalidValue;
+  }
 }
 cudaError_t launch_add_partials(cudaStream_t st, float *x, const float *part, int n_part, int64_t part_stride, int rows, int d) {
   const int64_t n4 = (int64_t)rows * d / 4;
