@@ -37,6 +37,20 @@ choices; the arithmetic of every function below is pinned by tests):
     position with the highest confidence is committed;
   * EoTP truncates at the committing step and decoding continues until the
     masked positions before [EoT] in the current block are done.
+
+Comparison policies (the strategies the paper measures Learn2PD against; same loop,
+another test inside it), selected by DecodeConfig.rule:
+  * "confidence": a masked position is committed when its confidence (Eq. 4)
+    exceeds a fixed threshold (the confidence-threshold parallel decoding the
+    related-work section cites); with the threshold at 1 nothing passes and the
+    fallback commits one position per step, i.e. low-confidence remasking with one
+    token per step, the paper's vanilla decoding (Section 3.1: s steps per block);
+  * "egp": Extremely Greedy Parallel, Section 3.1: unmask position j if and only
+    if the prediction equals the reference answer r_j (Algorithm 1's test).
+    Unpinned reading: when no masked position of the block matches, the masked
+    position with the highest confidence is committed WITH ITS REFERENCE TOKEN, so
+    that the loop ends and the response equals the reference, as the section says
+    of the oracle.  egp_labels() gives Algorithm 1's targets y_j for a step.
 """
 from __future__ import annotations
 
@@ -226,10 +240,35 @@ def unmask_rule(p: np.ndarray, conf: np.ndarray, masked: np.ndarray, tau: float)
     return unmask, forced
 
 
+def confidence_rule(conf: np.ndarray, masked: np.ndarray, threshold: float):
+    """Fixed-threshold policy: commit masked positions whose confidence exceeds the threshold
+    (strict); same progress fallback as unmask_rule."""
+    return unmask_rule(conf, conf, masked, threshold)
+
+
+def egp_labels(pred: np.ndarray, ref: np.ndarray) -> np.ndarray:
+    """Algorithm 1: y_j = 1 where the prediction equals the reference token, else 0."""
+    return np.asarray(pred) == np.asarray(ref)
+
+
+def egp_rule(pred: np.ndarray, ref: np.ndarray, conf: np.ndarray, masked: np.ndarray):
+    """Section 3.1 (EGP): unmask j iff pred_j == r_j.  Returns (unmask, forced); on a forced step the
+    caller commits the reference token at the chosen position (see the module header)."""
+    unmask = masked & egp_labels(pred, ref)
+    forced = False
+    if masked.any() and not unmask.any():
+        cand = np.where(masked)[0]
+        unmask[cand[np.argmax(conf[cand])]] = True
+        forced = True
+    return unmask, forced
+
+
 @dataclass
 class DecodeConfig:
     block_len: int
     tau: float = 0.96
+    rule: str = "filter"         # "filter" (Learn2PD, Algorithm 2), "confidence", "egp"
+    conf_threshold: float = 0.9  # rule "confidence"
     use_filter: bool = True      # False: nothing passes the threshold (one token per step)
     use_eotp: bool = True
     kv_cache: bool = False       # block-level prefix cache
@@ -297,7 +336,7 @@ def block_logits(m: Model, st: SeqState, cfg: DecodeConfig) -> np.ndarray:
 
 def decide(m: Model, filt: Dict[str, np.ndarray], st: SeqState, cfg: DecodeConfig,
            pred: np.ndarray, conf: np.ndarray, gap: Optional[np.ndarray] = None,
-           logits: Optional[np.ndarray] = None) -> StepRecord:
+           logits: Optional[np.ndarray] = None, ref: Optional[np.ndarray] = None) -> StepRecord:
     """Everything after M(X) in one step: filter, threshold, in-place commit, EoTP, block advance.
 
     pred/conf hold the n_rows block positions that are inside L_eff, in position order.
@@ -317,15 +356,29 @@ def decide(m: Model, filt: Dict[str, np.ndarray], st: SeqState, cfg: DecodeConfi
     conf_full = np.zeros(s, dtype=np.float64)
     conf_full[:n_rows] = conf
 
-    if cfg.use_filter:
+    if cfg.use_filter and cfg.rule == "filter":
         p = sigmoid(filter_logits(filt, c))
     else:
         p = np.zeros(s, dtype=np.float64)
-    unmask, forced = unmask_rule(p, conf_full, blk_masked, cfg.tau)
+    commit = np.full(s, -1, dtype=np.int64)     # token written at each committed position
+    commit[:n_rows] = pred
+    if cfg.rule == "filter":
+        unmask, forced = unmask_rule(p, conf_full, blk_masked, cfg.tau)
+    elif cfg.rule == "confidence":
+        unmask, forced = confidence_rule(conf_full, blk_masked, cfg.conf_threshold)
+    elif cfg.rule == "egp":
+        r_blk = np.asarray(ref, dtype=np.int64)[g0: g0 + s]
+        pred_full = np.full(s, -1, dtype=np.int64)
+        pred_full[:n_rows] = pred
+        unmask, forced = egp_rule(pred_full, r_blk, conf_full, blk_masked)
+        if forced:
+            commit = np.where(unmask, r_blk, commit)
+    else:
+        raise ValueError("unknown rule %r" % (cfg.rule,))
 
     for j in np.where(unmask)[0]:
         st.masked[g0 + j] = False
-        st.tokens[st.P + g0 + j] = pred[j]
+        st.tokens[st.P + g0 + j] = commit[j]
     st.forced += int(forced)
 
     # EoTP: earliest committed [EoT] in the generation region cuts the sequence there
@@ -351,7 +404,7 @@ def decide(m: Model, filt: Dict[str, np.ndarray], st: SeqState, cfg: DecodeConfi
 
 
 def denoise_step(m: Model, filt: Dict[str, np.ndarray], st: SeqState, cfg: DecodeConfig,
-                 keep_logits: bool = False, predictor=None) -> StepRecord:
+                 keep_logits: bool = False, predictor=None, ref: Optional[np.ndarray] = None) -> StepRecord:
     """One iteration of the while loop of Algorithm 2 for one sequence.
 
     predictor(m, st, cfg) -> logits[n_rows, V] replaces the transformer when given
@@ -361,7 +414,7 @@ def denoise_step(m: Model, filt: Dict[str, np.ndarray], st: SeqState, cfg: Decod
     st.steps += 1
     logits = (predictor or block_logits)(m, st, cfg)
     pred, conf, gap = confidence_head(logits)
-    return decide(m, filt, st, cfg, pred, conf, gap, logits if keep_logits else None)
+    return decide(m, filt, st, cfg, pred, conf, gap, logits if keep_logits else None, ref)
 
 
 @dataclass
@@ -375,14 +428,17 @@ class DecodeResult:
 
 def decode(m: Model, filt: Dict[str, np.ndarray], prompt: Sequence[int], G: int,
            cfg: DecodeConfig, keep_trace: bool = True, keep_logits: bool = False,
-           predictor=None) -> DecodeResult:
-    """Algorithm 2 with Algorithm 3's end-of-text break, for one prompt."""
+           predictor=None, ref: Optional[np.ndarray] = None) -> DecodeResult:
+    """Algorithm 2 with Algorithm 3's end-of-text break, for one prompt.  `ref` [G]: the reference
+    answer of rule "egp" (Algorithm 1's decode, without the filter update)."""
+    if cfg.rule == "egp" and (ref is None or len(ref) != G):
+        raise ValueError("rule 'egp' needs a reference answer of G tokens")
     if G % cfg.block_len != 0:
         raise ValueError("generation length must be a multiple of the block length")
     st = init_state(m, prompt, G)
     trace = []
     while not st.done:
-        rec = denoise_step(m, filt, st, cfg, keep_logits, predictor)
+        rec = denoise_step(m, filt, st, cfg, keep_logits, predictor, ref)
         if keep_trace:
             trace.append(rec)
     out_len = st.eot_pos + 1 if st.eot_pos >= 0 else G

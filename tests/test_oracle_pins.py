@@ -546,3 +546,112 @@ def test_linear_is_x_times_w_transposed():
         for o in range(4):
             assert y[t, o] == pytest.approx(sum(x[t, i] * float(w[o, i]) for i in range(5)), abs=1e-13)
     assert np.array_equal(orc.linear(x, np.eye(5, dtype=np.float32)), x)
+
+
+# ----------------------------------------------------------------------------- comparison policies
+
+def test_confidence_rule_closed_form_and_vanilla_limit():
+    """Fixed-threshold policy on one-hot logits: conf = e^a / (e^a + V - 1) in closed form, so which
+    positions pass 0.9 is known by hand; with the threshold at 1 nothing passes and the decode takes
+    s steps per block (Section 3.1's vanilla count), ending in the same tokens."""
+    s, V = 8, 12
+    m = _toy_model(V)
+    peaks = np.array([6.0, 1.0, 5.0, 2.0, 7.0, 0.5, 4.0, 3.0])
+    ids = np.array([3, 1, 4, 1, 5, 9, 2, 6])
+    logits = np.zeros((s, V))
+    logits[np.arange(s), ids] = peaks
+    conf = np.exp(peaks) / (np.exp(peaks) + V - 1)
+    first = conf > 0.9
+    assert first.sum() == 3                                   # peaks 6, 5, 7 (4 gives 0.832)
+    cfg = orc.DecodeConfig(block_len=s, rule="confidence", conf_threshold=0.9)
+    r = orc.decode(m, const_filter(s, 50.0), [0], s, cfg, predictor=_table_predictor([logits]))
+    assert np.array_equal(r.trace[0].unmask, first) and not r.trace[0].forced
+    assert (r.trace[0].p == 0).all()                          # the filter takes no part
+    # afterwards nothing passes: one forced commit per step, highest confidence first
+    rest = [int(np.where(t.unmask)[0][0]) for t in r.trace[1:]]
+    assert rest == [6, 7, 3, 1, 5] and all(t.forced for t in r.trace[1:])
+    assert r.steps == 1 + 5 and np.array_equal(r.response, ids)
+    van = orc.decode(m, None, [0], s, orc.DecodeConfig(block_len=s, rule="confidence", conf_threshold=1.0),
+                     predictor=_table_predictor([logits]))
+    assert van.steps == s and van.forced == s and np.array_equal(van.response, ids)
+    off = orc.decode(m, None, [0], s, orc.DecodeConfig(block_len=s, use_filter=False),
+                     predictor=_table_predictor([logits]))
+    assert [np.where(t.unmask)[0][0] for t in van.trace] == [np.where(t.unmask)[0][0] for t in off.trace]
+
+
+def _chain_predictor(ref, V, wrong):
+    """Predicts the reference at block position j only once position j-1 of the block is committed
+    (position 0 at once); elsewhere it predicts `wrong`."""
+    def f(m, st, cfg):
+        s = cfg.block_len
+        g0 = st.cur_block * s
+        ids = np.full(s, wrong)
+        for j in range(s):
+            if j == 0 or not st.masked[g0 + j - 1]:
+                ids[j] = ref[g0 + j]
+        return _one_hot_logits(ids, V)
+    return f
+
+
+def test_egp_unmasks_on_first_match_and_reproduces_the_reference():
+    """Section 3.1: a position is committed at the first step whose prediction equals the reference,
+    never earlier and never later; the response is the reference."""
+    s, G, V = 4, 8, 12
+    m = _toy_model(V)
+    ref = np.array([1, 2, 3, 4, 5, 6, 7, 8])
+    cfg = orc.DecodeConfig(block_len=s, rule="egp")
+    # (a) every prediction right at once: one step per block
+    table = [_one_hot_logits(ref[b * s:(b + 1) * s], V) for b in range(G // s)]
+    r = orc.decode(m, None, [0], G, cfg, predictor=_table_predictor(table), ref=ref)
+    assert r.steps == G // s and r.forced == 0 and np.array_equal(r.response, ref)
+    # (b) a prediction turns right only after its left neighbour is committed: step k of a block
+    #     commits position k alone, no fallback is needed, the labels are Algorithm 1's
+    r = orc.decode(m, None, [0], G, cfg, predictor=_chain_predictor(ref, V, wrong=0), ref=ref)
+    assert r.steps == G and r.forced == 0 and np.array_equal(r.response, ref)
+    for k, t in enumerate(r.trace):
+        want = np.zeros(s, bool)
+        want[k % s] = True
+        assert np.array_equal(t.unmask, want)
+        labels = orc.egp_labels(t.pred, ref[t.block * s:(t.block + 1) * s])
+        assert np.array_equal(labels[k % s:], want[k % s:])   # right of k: still wrong
+        assert labels[:k % s + 1].all()                        # committed positions stay right
+    with pytest.raises(ValueError):
+        orc.decode(m, None, [0], G, cfg, predictor=_table_predictor(table))
+
+
+def test_egp_fallback_commits_the_reference_token():
+    """Where the model never predicts the reference, the loop still ends and still returns the
+    reference: each such step commits the most confident masked position with its reference token."""
+    s, V = 4, 12
+    m = _toy_model(V)
+    ref = np.array([1, 2, 3, 4])
+    ids = np.array([1, 9, 3, 9])                 # positions 1 and 3 never match
+    logits = np.zeros((s, V))
+    logits[np.arange(s), ids] = [5.0, 2.0, 5.0, 3.0]
+    r = orc.decode(m, None, [0], s, orc.DecodeConfig(block_len=s, rule="egp"),
+                   predictor=_table_predictor([logits]), ref=ref)
+    assert np.array_equal(r.trace[0].unmask, [True, False, True, False]) and not r.trace[0].forced
+    assert [int(np.where(t.unmask)[0][0]) for t in r.trace[1:]] == [3, 1]
+    assert r.steps == 3 and r.forced == 2 and np.array_equal(r.response, ref)
+
+
+def test_egp_with_the_models_own_answer_as_reference_skips_repeats():
+    """Section 3.1 defines the reference as the answer of the standard decode; under EGP with that
+    reference the small transformer needs no more steps than the standard decode and every
+    step's commits are exactly the masked positions where pred == reference."""
+    shape = small_shape()
+    w = wl.make_weights(shape, seed=5)
+    m = oracle_model(shape, w)
+    s, G = 8, 16
+    prompt = wl.make_prompts(1, 6, shape, seed=1)[0]
+    van = orc.decode(m, None, prompt, G, orc.DecodeConfig(block_len=s, use_filter=False, use_eotp=False))
+    egp = orc.decode(m, None, prompt, G, orc.DecodeConfig(block_len=s, rule="egp", use_eotp=False),
+                     ref=van.response)
+    assert egp.steps <= van.steps and np.array_equal(egp.response, van.response)
+    masked = np.ones(G, bool)
+    for t in egp.trace:
+        blk = slice(t.block * s, (t.block + 1) * s)
+        if not t.forced:
+            assert np.array_equal(t.unmask, masked[blk] & orc.egp_labels(t.pred, van.response[blk]))
+        masked[blk] &= ~t.unmask
+    assert not masked.any()
