@@ -163,6 +163,28 @@ l2pd_status l2pd_decode(l2pd_ctx *ctx, void *stream, const int32_t *d_prompts,
                         int32_t B, int32_t P, int32_t G, int32_t *d_out_tokens,
                         int32_t *h_out_len, int32_t *h_steps, int32_t *h_total_steps);
 
+/*
+ * Comparison policies of Section 3.1: which test a masked position of the current block must
+ * pass to be committed.  The rest of the step (forward pass, confidence, progress fallback,
+ * EoTP, block advance) is unchanged.
+ *   L2PD_RULE_FILTER      Algorithm 2: sigmoid(filter output) > tau (the state after l2pd_init).
+ *   L2PD_RULE_CONFIDENCE  confidence (Eq. 4) > conf_threshold, strict, conf_threshold in [0, 1];
+ *                         at 1 nothing passes and every step commits only the most confident masked
+ *                         position: the one-token-per-step decoding the paper counts speed-ups against.
+ *   L2PD_RULE_EGP         Extremely Greedy Parallel: prediction == reference token.  d_reference:
+ *                         DEVICE int32 [ref_rows, ref_len], borrowed until the rule is set again or the
+ *                         context is destroyed; sequence i of a reset reads row i, so a reset needs
+ *                         B <= ref_rows and G == ref_len (else L2PD_ERR_SHAPE).  The ids are
+ *                         range-checked here (L2PD_ERR_TOKEN_RANGE; the call synchronises).  A step in
+ *                         which no masked position matches commits the most confident masked position
+ *                         WITH ITS REFERENCE TOKEN, so the decode ends and returns the reference.
+ * The filter output p is reported as 0 under the last two rules.  Any decode in progress is
+ * dropped: call l2pd_state_reset (or l2pd_decode) next.  Unused arguments are ignored.
+ */
+enum { L2PD_RULE_FILTER = 0, L2PD_RULE_CONFIDENCE = 1, L2PD_RULE_EGP = 2 };
+l2pd_status l2pd_set_unmask_rule(l2pd_ctx *ctx, void *stream, int32_t rule, float conf_threshold,
+                                 const int32_t *d_reference, int32_t ref_rows, int32_t ref_len);
+
 /* Number of sequences that still need steps (0 before the first reset). */
 int32_t l2pd_num_active(const l2pd_ctx *ctx);
 

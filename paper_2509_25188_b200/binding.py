@@ -55,7 +55,7 @@ class StepOut(C.Structure):
 
 
 EXPORTS = ["l2pd_init", "l2pd_state_reset", "l2pd_denoise_step", "l2pd_decode", "l2pd_num_active",
-           "l2pd_state_tokens", "l2pd_state_masked", "l2pd_set_capture", "l2pd_last_step_rows",
+           "l2pd_state_tokens", "l2pd_state_masked", "l2pd_set_unmask_rule", "l2pd_set_capture", "l2pd_last_step_rows",
            "l2pd_launch_count", "l2pd_last_step_ms", "l2pd_profile_enable", "l2pd_profile_read", "l2pd_last_error", "l2pd_destroy",
            "l2pd_gemm_bf16", "l2pd_gemm_bf16_residual", "l2pd_gemm_bf16_swiglu", "l2pd_lm_head_bf16",
            "l2pd_lm_head_scratch_elems", "l2pd_attention_bf16", "l2pd_lm_head_bf16_static"]
@@ -81,6 +81,7 @@ def _load() -> C.CDLL:
     lib.l2pd_state_masked.argtypes = [vp]
     lib.l2pd_state_masked.restype = vp
     lib.l2pd_set_capture.argtypes = [vp, vp, i64]
+    lib.l2pd_set_unmask_rule.argtypes = [vp, vp, i32, f32, vp, i32, i32]
     lib.l2pd_last_step_rows.argtypes = [vp]
     lib.l2pd_launch_count.argtypes = [vp]
     lib.l2pd_launch_count.restype = i64
@@ -259,6 +260,22 @@ class Decoder:
         _check(lib.l2pd_decode(self.ctx, _stream(), d_prompts.data_ptr(), B, P, int(G), d_out.data_ptr(),
                                out_len.ctypes.data, steps.ctypes.data, C.addressof(total)), self.ctx)
         return out_len, steps, int(total.value)
+
+    RULES = {"filter": 0, "confidence": 1, "egp": 2}
+
+    def set_unmask_rule(self, rule: str, conf_threshold: float = 0.9, reference=None):
+        """rule: "filter" | "confidence" | "egp" (reference: int ids [rows, G], kept alive here)."""
+        ref = None
+        if rule == "egp":
+            r = reference if isinstance(reference, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(reference))
+            ref = r.to("cuda:%d" % self.device, torch.int32).contiguous()
+            if ref.dim() != 2:
+                raise ValueError("reference answers must be [rows, G]")
+        _check(lib.l2pd_set_unmask_rule(self.ctx, _stream(), self.RULES[rule], float(conf_threshold),
+                                        ref.data_ptr() if ref is not None else None,
+                                        int(ref.shape[0]) if ref is not None else 0,
+                                        int(ref.shape[1]) if ref is not None else 0), self.ctx)
+        self._reference = ref
 
     # ---- state and instrumentation -------------------------------------------------------------
     @property

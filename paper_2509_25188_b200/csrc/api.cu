@@ -36,6 +36,10 @@ struct l2pd_ctx {
 
   // decode state
   int B = 0, P = 0, G = 0;
+  int rule = L2PD_RULE_FILTER;          // test applied to masked positions (l2pd_set_unmask_rule)
+  float conf_threshold = 0.9f;
+  const int32_t *d_ref = nullptr;       // EGP: reference answers [ref_rows, ref_len], borrowed
+  int ref_rows = 0, ref_len = 0;
   bool has_state = false;
   int32_t *d_tokens = nullptr;
   uint8_t *d_masked = nullptr;
@@ -371,6 +375,7 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
   a.w1 = c->fw1; a.b1 = c->fb1; a.w2 = c->fw2; a.b2 = c->fb2; a.tau = f.tau;
   a.use_filter = f.use_filter; a.use_eotp = f.use_eotp; a.committed_conf_mode = f.committed_conf_mode;
   a.eot_id = f.eot_id; a.summary = c->d_summary;
+  a.rule = c->rule; a.conf_threshold = c->conf_threshold; a.ref = c->d_ref;
   if (out) { a.o_conf = out->d_conf; a.o_pred = out->d_pred; a.o_p = out->d_p; a.o_unmask = out->d_unmask; }
   CKLK(L2PD_K_DECIDE, launch_decide(s, a, n_slots));
   return L2PD_OK;
@@ -579,6 +584,8 @@ l2pd_status l2pd_state_reset(l2pd_ctx *c, void *stream, const int32_t *d_prompts
   if (B < 1 || B > f.max_batch) return set_err(c, L2PD_ERR_SHAPE, "batch %d outside [1, %d]", B, f.max_batch);
   if (P < 1 || G < 1 || P + G > f.max_seq) return set_err(c, L2PD_ERR_SHAPE, "P + G = %d exceeds max_seq %d (or P, G < 1)", P + G, f.max_seq);
   if (G % f.block_len) return set_err(c, L2PD_ERR_SHAPE, "generation length %d is not a multiple of the block length %d", G, f.block_len);
+  if (c->rule == L2PD_RULE_EGP && (B > c->ref_rows || G != c->ref_len))
+    return set_err(c, L2PD_ERR_SHAPE, "reference answers are [%d, %d]; the reset asks for B = %d, G = %d", c->ref_rows, c->ref_len, B, G);
   cudaStream_t s = (cudaStream_t)stream;
   CK(cudaSetDevice(c->device));
   c->has_state = false;
@@ -671,6 +678,34 @@ l2pd_status l2pd_decode(l2pd_ctx *c, void *stream, const int32_t *d_prompts, int
     if (h_steps) h_steps[i] = c->h_steps[i];
   }
   if (h_total_steps) *h_total_steps = c->total_steps;
+  return L2PD_OK;
+}
+
+l2pd_status l2pd_set_unmask_rule(l2pd_ctx *c, void *stream, int32_t rule, float conf_threshold,
+                                 const int32_t *d_reference, int32_t ref_rows, int32_t ref_len) {
+  if (!c) return L2PD_ERR_ARG;
+  if (rule != L2PD_RULE_FILTER && rule != L2PD_RULE_CONFIDENCE && rule != L2PD_RULE_EGP)
+    return set_err(c, L2PD_ERR_ARG, "unknown rule %d", rule);
+  if (rule == L2PD_RULE_CONFIDENCE && !(conf_threshold >= 0.f && conf_threshold <= 1.f))
+    return set_err(c, L2PD_ERR_ARG, "confidence threshold %g outside [0, 1]", (double)conf_threshold);
+  if (rule == L2PD_RULE_EGP) {
+    if (!d_reference || ref_rows < 1 || ref_len < 1) return set_err(c, L2PD_ERR_ARG, "rule EGP needs reference answers");
+    cudaStream_t s = (cudaStream_t)stream;
+    CK(cudaSetDevice(c->device));
+    CK(cudaMemsetAsync(c->d_status, 0, 4, s));
+    CKL(launch_check_ids(s, d_reference, (int64_t)ref_rows * ref_len, c->cfg.vocab, c->cfg.mask_id, c->d_status));
+    CK(cudaMemcpyAsync(c->h_status, c->d_status, 4, cudaMemcpyDeviceToHost, s));
+    CK(cudaMemsetAsync(c->d_status, 0, 4, s));
+    CK(cudaStreamSynchronize(s));
+    if (*c->h_status) return set_err(c, L2PD_ERR_TOKEN_RANGE, "a reference id is outside [0, vocab) or equals mask_id");
+  }
+  c->has_state = false;   // the next decode starts from a reset
+  c->n_active = 0;
+  c->rule = rule;
+  if (rule == L2PD_RULE_CONFIDENCE) c->conf_threshold = conf_threshold;
+  c->d_ref = rule == L2PD_RULE_EGP ? d_reference : nullptr;
+  c->ref_rows = rule == L2PD_RULE_EGP ? ref_rows : 0;
+  c->ref_len = rule == L2PD_RULE_EGP ? ref_len : 0;
   return L2PD_OK;
 }
 

@@ -100,6 +100,7 @@ cudaError_t launch_build_row_map(cudaStream_t st, const SeqMeta *meta, int n_slo
 cudaError_t launch_permute_qkv_rows(cudaStream_t st, const bf16 *src, bf16 *dst, int H, int dh, int d);
 cudaError_t launch_state_reset(cudaStream_t st, const int32_t *prompts, int B, int P, int G, int vocab,
                                int mask_id, int32_t *tokens, uint8_t *masked, SeqState s, int32_t *bad);
+cudaError_t launch_check_ids(cudaStream_t st, const int32_t *ids, int64_t n, int vocab, int mask_id, int32_t *bad);
 cudaError_t launch_gather_response(cudaStream_t st, const int32_t *tokens, int B, int P, int G,
                                    int32_t *out);
 
@@ -128,6 +129,9 @@ struct DecideArgs {
   const float *w1, *b1, *w2, *b2;
   float tau;
   int use_filter, use_eotp, committed_conf_mode, eot_id;
+  int rule;                       // 0 filter (Algorithm 2), 1 fixed confidence threshold, 2 EGP (Section 3.1)
+  float conf_threshold;           // rule 1
+  const int32_t *ref;             // rule 2: reference answers [B, G]
   StepSummary *summary;           // [max_batch], indexed by sequence
   float *o_conf; int32_t *o_pred; float *o_p; uint8_t *o_unmask;   // optional [B, s]
 };

@@ -5,6 +5,9 @@
 //     p = sigmoid(z) (Section 3.2);
 //   * Algorithm 2: every masked position with p > tau (strict) is committed in place; if none
 //     passes, the masked position with the highest confidence is committed so the loop advances;
+//     (comparison policies of Section 3.1 replace the test: confidence above a fixed threshold, or
+//     Extremely Greedy Parallel, prediction == reference token; an EGP step in which nothing
+//     matches commits the reference token at the most confident masked position);
 //   * EoTP (Section 3.3): the earliest committed [EoT] cuts the sequence; later positions leave
 //     the mask set and read as [EoT];
 //   * block advance / stop (Algorithm 3: no block after one that holds [EoT]).
@@ -25,6 +28,7 @@ __global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
   __shared__ float s_p[MAX_S];
   __shared__ int s_masked[MAX_S];
   __shared__ int s_unmask[MAX_S];
+  __shared__ int s_commit[MAX_S];
   __shared__ int s_any, s_e, s_left;
 
   grid_dep_launch();
@@ -81,7 +85,7 @@ __global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
     s_c[j] = c;
   }
   __syncthreads();
-  if (a.use_filter) {
+  if (a.use_filter && a.rule == 0) {
     if (threadIdx.x < s) {
       int j = threadIdx.x;
       float h = a.b1[j];
@@ -103,7 +107,12 @@ __global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
   // ---- threshold, progress fallback ------------------------------------------------------------------
   if (threadIdx.x < s) {
     int j = threadIdx.x;
-    if (s_masked[j] && s_p[j] > a.tau) { s_unmask[j] = 1; s_any = 1; }
+    bool pass;
+    if (a.rule == 0) pass = s_p[j] > a.tau;
+    else if (a.rule == 1) pass = s_conf[j] > a.conf_threshold;
+    else pass = s_pred[j] == a.ref[(int64_t)seq * a.G + g0 + j];   // dead rows hold -1, never a token id
+    s_commit[j] = s_pred[j];
+    if (s_masked[j] && pass) { s_unmask[j] = 1; s_any = 1; }
   }
   __syncthreads();
   int forced = 0;
@@ -113,7 +122,10 @@ __global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
       float bc = -1.f;
       for (int j = 0; j < s; ++j)
         if (s_masked[j] && s_conf[j] > bc) { bc = s_conf[j]; best = j; }
-      if (best >= 0) { s_unmask[best] = 1; s_any = 2; }
+      if (best >= 0) {
+        s_unmask[best] = 1; s_any = 2;
+        if (a.rule == 2) s_commit[best] = a.ref[(int64_t)seq * a.G + g0 + best];
+      }
     }
     __syncthreads();
     forced = (s_any == 2);
@@ -123,10 +135,10 @@ __global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
   if (threadIdx.x < s) {
     int j = threadIdx.x;
     if (s_unmask[j]) {
-      a.tokens[(int64_t)seq * a.tok_stride + m.blk_start + j] = s_pred[j];
+      a.tokens[(int64_t)seq * a.tok_stride + m.blk_start + j] = s_commit[j];
       a.masked[(int64_t)seq * a.G + g0 + j] = 0;
       s_masked[j] = 0;
-      if (a.use_eotp && s_pred[j] == a.eot_id) atomicMin(&s_e, g0 + j);
+      if (a.use_eotp && s_commit[j] == a.eot_id) atomicMin(&s_e, g0 + j);
     }
     if (a.o_conf) a.o_conf[(int64_t)seq * s + j] = s_conf[j];
     if (a.o_pred) a.o_pred[(int64_t)seq * s + j] = s_pred[j];

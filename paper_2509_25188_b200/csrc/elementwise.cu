@@ -310,6 +310,14 @@ __global__ void state_reset_kernel(const int32_t *prompts, int P, int G, int voc
   }
 }
 
+// Sets *bad when an id is outside [0, vocab) or is the mask token.
+__global__ void check_ids_kernel(const int32_t *ids, int64_t n, int vocab, int mask_id, int32_t *bad) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    int t = ids[i];
+    if (t < 0 || t >= vocab || t == mask_id) atomicExch(bad, 1);
+  }
+}
+
 __global__ void gather_response_kernel(const int32_t *tokens, int P, int G, int32_t *out) {
   grid_dep_launch();
   grid_dep_wait();
@@ -368,6 +376,12 @@ cudaError_t launch_permute_qkv_rows(cudaStream_t st, const bf16 *src, bf16 *dst,
 cudaError_t launch_state_reset(cudaStream_t st, const int32_t *prompts, int B, int P, int G, int vocab,
                                int mask_id, int32_t *tokens, uint8_t *masked, SeqState s, int32_t *bad) {
   return launch_kernel(state_reset_kernel, dim3(B), dim3(256), 0, st, prompts, P, G, vocab, mask_id, tokens, masked, s, bad);
+}
+cudaError_t launch_check_ids(cudaStream_t st, const int32_t *ids, int64_t n, int vocab, int mask_id, int32_t *bad) {
+  int blocks = (int)((n + 255) / 256);
+  blocks = blocks < 1 ? 1 : (blocks > 592 ? 592 : blocks);
+  check_ids_kernel<<<blocks, 256, 0, st>>>(ids, n, vocab, mask_id, bad);
+  return cudaGetLastError();
 }
 cudaError_t launch_gather_response(cudaStream_t st, const int32_t *tokens, int B, int P, int G,
                                    int32_t *out) {

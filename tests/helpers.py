@@ -49,7 +49,7 @@ def _sync_oracle_state(st, m, toks, msk, l_eff, done, cur_block):
 
 
 def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, conf_margin=None,
-             check_logits=True, max_steps=None, replay_margin=1e-5, oracle_when=None):
+             check_logits=True, max_steps=None, replay_margin=1e-5, oracle_when=None, refs=None):
     """Runs the CUDA decoder step by step; before every step the oracle is put in the decoder's
     state (teacher forcing), then both take the step and are compared:
       logits  |gpu - orc| <= logit_rtol * max|orc row|
@@ -63,12 +63,23 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
     oracle_when(i, step_of_sequence_i, state) -> bool selects the (sequence, step) pairs on which the
     oracle's forward pass is run and compared (default: all of them); the decision replay runs on
     every step of every sequence either way, since it needs no forward pass.
+    Under cfg.rule "confidence" the margins apply to |conf - conf_threshold| instead of |p - tau|;
+    under "egp" (refs[i] = reference answer of sequence i) the test is an integer comparison and the
+    oracle's own decision is compared where every prediction of the block is sure.
     Returns counters; asserts on any violation.
     """
     import copy
 
     if conf_margin is None:
         conf_margin = 2 * conf_atol
+
+    def boundary_distance(r, blk_masked, n):
+        if cfg.rule == "filter":
+            return np.abs(r.p - cfg.tau)[blk_masked]
+        if cfg.rule == "confidence":
+            return np.abs(r.conf - cfg.conf_threshold)[blk_masked[:n]]
+        return np.zeros(0)
+
     prompts = np.asarray(prompts)
     B, P = prompts.shape
     s = cfg.block_len
@@ -88,6 +99,7 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
         out = dec.denoise_step(want_logits=need_logits)
         stat["steps"] += 1
         stat["trace"].append({k: np.array(out[k]) for k in ("block", "masks_left", "l_eff", "done", "forced")})
+        replayed = {}
         for i in active:
             st = states[i]
             pre = copy.deepcopy(st)
@@ -99,7 +111,7 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
             assert (out["pred"][i, n:] == -1).all() and (out["conf"][i, n:] == 0).all()
             rec = None
             if want_oracle[i]:
-                rec = orc.denoise_step(m, filt, st, cfg, keep_logits=True)
+                rec = orc.denoise_step(m, filt, st, cfg, keep_logits=True, ref=None if refs is None else refs[i])
                 stat["oracle_steps"] += 1
                 assert rec.block == blk and rec.n_rows == n
                 row_max = np.abs(rec.logits).max(axis=-1)
@@ -119,9 +131,9 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
             rp.steps += 1
             gpred = out["pred"][i, :n].astype(np.int64)
             gconf = out["conf"][i, :n].astype(np.float64)
-            rrec = orc.decide(m, filt, rp, cfg, gpred, gconf)
+            rrec = orc.decide(m, filt, rp, cfg, gpred, gconf, ref=None if refs is None else refs[i])
             blk_masked = pre.masked[blk * s: blk * s + s]
-            near = np.abs(rrec.p - cfg.tau)[blk_masked]
+            near = boundary_distance(rrec, blk_masked, n)
             replay_ok = (len(near) == 0 or near.min() > replay_margin)
             if replay_ok:
                 stat["replay_checked"] += 1
@@ -130,12 +142,15 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
                 assert out["forced"][i] == int(rrec.forced)
                 assert out["masks_left"][i] == int(rp.masked[blk * s: blk * s + s].sum())
                 assert np.abs(out["p"][i] - rrec.p).max() < 1e-4
+                replayed[i] = rp
 
             if rec is None:
                 continue
             # the oracle's own decision, where it is clear of the margins
-            near_o = np.abs(rec.p - cfg.tau)[blk_masked]
+            near_o = boundary_distance(rec, blk_masked, n)
             clear = len(near_o) == 0 or near_o.min() > p_margin
+            if cfg.rule == "egp":
+                clear = bool(sure.all())
             if rec.forced:
                 cm = np.sort(rec.conf[blk_masked[:n]])[::-1]
                 clear = clear and (len(cm) < 2 or cm[0] - cm[1] > conf_margin)
@@ -145,6 +160,8 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
                 assert out["forced"][i] == int(rec.forced)
                 stat["forced"] += int(rec.forced)
         toks, msk = dec.tokens(), dec.masked()
+        for i, rp in replayed.items():     # the committed ids and the mask set after the step
+            assert np.array_equal(rp.tokens, toks[i]) and np.array_equal(rp.masked, msk[i])
         for i in active:
             blk = out["block"][i]
             nxt = blk + 1 if (out["masks_left"][i] == 0 and not out["done"][i]) else blk
