@@ -37,6 +37,13 @@ choices; the arithmetic of every function below is pinned by tests):
     position with the highest confidence is committed;
   * EoTP truncates at the committing step and decoding continues until the
     masked positions before [EoT] in the current block are done.
+  * KV caches (Section 4.3 names a prefix cache and a dual cache and gives no rule):
+    the first step of a block is a full forward pass that stores K (rotated) and V
+    per layer; the block's other steps recompute rows from the block start to the
+    end of the sequence against stored prefix ++ fresh keys (prefix cache), or only
+    the block's own rows against stored prefix ++ fresh block ++ stored positions
+    after the block (dual cache).  Stored entries go stale as tokens are committed:
+    both are approximations for more than one layer and exact for one.
 
 Comparison policies (the strategies the paper measures Learn2PD against; same loop,
 another test inside it), selected by DecodeConfig.rule:
@@ -137,12 +144,14 @@ def silu(x: np.ndarray) -> np.ndarray:
 
 def layer_forward(m: Model, layer: Dict[str, np.ndarray], x: np.ndarray, pos: np.ndarray,
                   k_prefix: Optional[np.ndarray] = None, v_prefix: Optional[np.ndarray] = None,
-                  kv_out: Optional[list] = None) -> np.ndarray:
+                  kv_out: Optional[list] = None,
+                  k_suffix: Optional[np.ndarray] = None, v_suffix: Optional[np.ndarray] = None) -> np.ndarray:
     """One pre-norm block on rows x[T, d] at positions pos[T].
 
     k_prefix / v_prefix [Tp, H, dh] (k already rotated) are put before this
-    call's keys and values (prefix-cache rule).  kv_out, if a list, receives
-    (k_rotated, v) of this call's rows.
+    call's keys and values (prefix-cache rule), k_suffix / v_suffix [Ts, H, dh]
+    after them (dual-cache rule).  kv_out, if a list, receives (k_rotated, v) of
+    this call's rows.
     """
     H, dh = m.n_heads, m.head_dim
     T = x.shape[0]
@@ -158,6 +167,9 @@ def layer_forward(m: Model, layer: Dict[str, np.ndarray], x: np.ndarray, pos: np
     if k_prefix is not None:
         k = np.concatenate([k_prefix, k], axis=0)
         v = np.concatenate([v_prefix, v], axis=0)
+    if k_suffix is not None:
+        k = np.concatenate([k, k_suffix], axis=0)
+        v = np.concatenate([v, v_suffix], axis=0)
     a = attention(q, k, v).reshape(T, H * dh)
     x = x + linear(a, layer["wo"])
     n = rmsnorm(x, layer["norm2"], m.rms_eps)
@@ -166,12 +178,14 @@ def layer_forward(m: Model, layer: Dict[str, np.ndarray], x: np.ndarray, pos: np
 
 
 def forward_hidden(m: Model, tokens: np.ndarray, pos0: int = 0,
-                   prefix_kv: Optional[list] = None, kv_out: Optional[list] = None) -> np.ndarray:
+                   prefix_kv: Optional[list] = None, kv_out: Optional[list] = None,
+                   suffix_kv: Optional[list] = None) -> np.ndarray:
     """Residual stream after the last layer for `tokens` placed at positions pos0...
 
     Weights: tok_emb[V,d], layers[l]{wqkv[3Hdh,d], wo[d,Hdh], w_gate[F,d], w_up[F,d],
     w_down[d,F], norm1[d], norm2[d]}, final_norm[d], lm_head[V,d]; all [out, in].
-    prefix_kv[l] = (k, v) of earlier positions for layer l, or None.
+    prefix_kv[l] = (k, v) of earlier positions for layer l, or None; suffix_kv[l] the
+    same for later positions.
     kv_out, if a list, receives one (k, v) per layer for this call's rows.
     """
     w = m.weights
@@ -179,7 +193,8 @@ def forward_hidden(m: Model, tokens: np.ndarray, pos0: int = 0,
     pos = pos0 + np.arange(len(tokens))
     for l, layer in enumerate(w["layers"]):
         kp, vp = (prefix_kv[l] if prefix_kv is not None else (None, None))
-        x = layer_forward(m, layer, x, pos, kp, vp, kv_out)
+        ks, vs = (suffix_kv[l] if suffix_kv is not None else (None, None))
+        x = layer_forward(m, layer, x, pos, kp, vp, kv_out, ks, vs)
     return x
 
 
@@ -272,6 +287,7 @@ class DecodeConfig:
     use_filter: bool = True      # False: nothing passes the threshold (one token per step)
     use_eotp: bool = True
     kv_cache: bool = False       # block-level prefix cache
+    dual_cache: bool = False     # with kv_cache: the positions after the block are cached as well
     committed_conf_mode: int = 0  # 0: model confidence at committed positions, 1: 1.0 there
 
 
@@ -288,6 +304,7 @@ class SeqState:
     forced: int = 0
     eot_pos: int = -1            # generation index of the earliest committed [EoT], -1 if none
     prefix_kv: Optional[list] = None     # prefix cache of the current block
+    all_kv: Optional[list] = None        # dual cache: K, V of every position at the block's first step
     cache_block: int = -1                # block the cache was filled for
 
 
@@ -327,8 +344,16 @@ def block_logits(m: Model, st: SeqState, cfg: DecodeConfig) -> np.ndarray:
         kv: list = []
         x = forward_hidden(m, st.tokens[: st.L_eff], kv_out=kv)
         st.prefix_kv = [(k[:S_b].copy(), v[:S_b].copy()) for (k, v) in kv]
+        st.all_kv = kv if cfg.dual_cache else None
         st.cache_block = st.cur_block
         return lm_head_logits(m, x[S_b: S_b + n_rows])
+    if cfg.dual_cache:
+        # later steps, dual cache: only the block's rows; keys = cached prefix ++ fresh block rows ++
+        # cached positions after the block (those still inside L_eff)
+        end = S_b + n_rows
+        suffix = [(k[end: st.L_eff], v[end: st.L_eff]) for (k, v) in st.all_kv]
+        x = forward_hidden(m, st.tokens[S_b: end], pos0=S_b, prefix_kv=st.prefix_kv, suffix_kv=suffix)
+        return lm_head_logits(m, x)
     # later steps of the block: only rows [S_b, L_eff), keys = cached prefix ++ fresh rows
     x = forward_hidden(m, st.tokens[S_b: st.L_eff], pos0=S_b, prefix_kv=st.prefix_kv)
     return lm_head_logits(m, x[:n_rows])

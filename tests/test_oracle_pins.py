@@ -12,7 +12,7 @@ import torch
 
 from oracle import l2pd_oracle as orc
 from paper_2509_25188_b200 import workloads as wl
-from tests.helpers import const_filter, identity_filter, oracle_model, small_shape
+from tests.helpers import const_filter, find_eot_bias, identity_filter, oracle_model, small_shape
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "paper_constants.txt")
 
@@ -476,11 +476,11 @@ def test_prefix_cache_is_exact_for_one_layer():
     decode equals the uncached one."""
     shape, m = _cache_models(1)
     s, G = 4, 12
-    filt = wl.make_filter(s, seed=2)
+    filt = const_filter(s, -50.0)                             # one commit per step: most steps read the store
     p = wl.make_prompts(1, 5, shape, seed=3)[0]
     a = orc.decode(m, filt, p, G, orc.DecodeConfig(block_len=s), keep_logits=True)
     b = orc.decode(m, filt, p, G, orc.DecodeConfig(block_len=s, kv_cache=True), keep_logits=True)
-    assert a.steps == b.steps and np.array_equal(a.response, b.response)
+    assert a.steps == b.steps > G // s and np.array_equal(a.response, b.response)
     for ra, rb in zip(a.trace, b.trace):
         assert np.allclose(ra.logits, rb.logits, atol=1e-10)
 
@@ -505,6 +505,82 @@ def test_prefix_cache_first_step_of_each_block_is_the_full_forward():
             differs = True                       # stale prefix K/V: an approximation for NL > 1
     assert differs
     del cfg_u
+
+
+def test_dual_cache_is_exact_for_one_layer_and_uses_block_rows_only():
+    """One layer: K/V of a position depend on its own token alone, so reading the positions before
+    AND after the block from the store changes nothing as long as their tokens are unchanged
+    (they are: only the current block's positions are committed, and those rows are fresh)."""
+    shape, m = _cache_models(1)
+    s, G = 4, 12
+    filt = const_filter(s, -50.0)
+    p = wl.make_prompts(1, 5, shape, seed=3)[0]
+    a = orc.decode(m, filt, p, G, orc.DecodeConfig(block_len=s), keep_logits=True)
+    b = orc.decode(m, filt, p, G, orc.DecodeConfig(block_len=s, kv_cache=True, dual_cache=True), keep_logits=True)
+    assert a.steps == b.steps and np.array_equal(a.response, b.response)
+    assert a.steps > G // s                                   # some steps did read the store
+    for ra, rb in zip(a.trace, b.trace):
+        assert np.allclose(ra.logits, rb.logits, atol=1e-10)
+
+
+def test_dual_cache_two_layers_brute_force_and_eotp():
+    """Two layers: a later step of a block equals a by-hand evaluation in which layer 2's keys and
+    values outside the block are the ones of the block's first step (stale), inside it fresh; the
+    first step of each block is the full forward.  Runs with an [EoT] bias so the sequence is cut."""
+    shape, m = _cache_models(2)
+    s, G = 4, 12
+    filt = const_filter(s, -50.0)
+    cfg = orc.DecodeConfig(block_len=s, kv_cache=True, dual_cache=True)
+    seed, bias, _ = find_eot_bias(m, shape, filt, G, cfg, 5, grid=np.arange(5.0, 120.0, 5.0))
+    m.lm_head_bias = wl.make_eot_bias(shape, bias)
+    p = wl.make_prompts(1, 5, shape, seed=seed)[0]
+    st = orc.init_state(m, p, G)
+    H, dh = m.n_heads, m.head_dim
+    layers = m.weights["layers"]
+    stale = None
+    later = 0
+    while not st.done:
+        first = st.cache_block != st.cur_block
+        S_b = st.P + st.cur_block * s
+        L = st.L_eff
+        n = min(s, L - S_b)
+        # by hand: layer 1 over every position (its K/V do not depend on other tokens' state)
+        x0 = orc.widen(m.weights["tok_emb"][st.tokens[:L]])
+        pos = np.arange(L)
+        kv1 = []
+        x1 = orc.layer_forward(m, layers[0], x0, pos, kv_out=kv1)
+        if first:
+            kv2 = []
+            x2 = orc.layer_forward(m, layers[1], x1, pos, kv_out=kv2)
+            stale = (x0.copy(), kv1[0], kv2[0])
+            want = orc.lm_head_logits(m, x2[S_b: S_b + n])
+        else:
+            later += 1
+            x0_old, (k1o, v1o), (k2o, v2o) = stale
+            blk = slice(S_b, S_b + n)
+            # layer 1 on the block rows: keys of the other positions from the first step
+            k1 = np.concatenate([k1o[:S_b], kv1[0][0][blk], k1o[S_b + n: L]])
+            v1 = np.concatenate([v1o[:S_b], kv1[0][1][blk], v1o[S_b + n: L]])
+
+            def block_layer(layer, xin, k_all, v_all):
+                nn = orc.rmsnorm(xin, layer["norm1"], m.rms_eps)
+                q = orc.rope(orc.linear(nn, layer["wqkv"])[:, : H * dh].reshape(n, H, dh), pos[blk], m.rope_theta)
+                xo = xin + orc.linear(orc.attention(q, k_all, v_all).reshape(n, H * dh), layer["wo"])
+                nn = orc.rmsnorm(xo, layer["norm2"], m.rms_eps)
+                return xo + orc.linear(orc.silu(orc.linear(nn, layer["w_gate"])) * orc.linear(nn, layer["w_up"]), layer["w_down"])
+
+            xb1 = block_layer(layers[0], x0[blk], k1, v1)
+            nn = orc.rmsnorm(xb1, layers[1]["norm1"], m.rms_eps)
+            qkv = orc.linear(nn, layers[1]["wqkv"])
+            kf = orc.rope(qkv[:, H * dh: 2 * H * dh].reshape(n, H, dh), pos[blk], m.rope_theta)
+            vf = qkv[:, 2 * H * dh:].reshape(n, H, dh)
+            k2 = np.concatenate([k2o[:S_b], kf, k2o[S_b + n: L]])
+            v2 = np.concatenate([v2o[:S_b], vf, v2o[S_b + n: L]])
+            xb2 = block_layer(layers[1], xb1, k2, v2)
+            want = orc.lm_head_logits(m, xb2)
+        rec = orc.denoise_step(m, filt, st, cfg, keep_logits=True)
+        assert rec.n_rows == n and np.allclose(rec.logits, want, atol=1e-9)
+    assert later >= 2 and 0 <= st.eot_pos < G - 1            # cut before the end
 
 
 # ----------------------------------------------------------------------------- planted mistakes
