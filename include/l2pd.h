@@ -72,7 +72,11 @@ typedef struct {
                                     step of a block runs all positions and stores K (rotated) and V of
                                     the positions before the block; the block's other steps compute
                                     only positions from the block start on and attend to
-                                    stored ++ fresh keys) */
+                                    stored ++ fresh keys).
+                                 2: dual cache (same section): the first step of a block also stores K, V
+                                    of the positions after the block; the block's other steps compute
+                                    the block's s rows only and attend to stored prefix ++ fresh block
+                                    ++ stored positions after the block (up to L_eff) */
   int32_t committed_conf_mode;/* what the filter reads at block positions already committed:
                                  0 = the model's confidence recomputed this step, 1 = 1.0 */
   int32_t max_batch;          /* most sequences a reset may start */
@@ -125,7 +129,7 @@ typedef struct {
 
 /*
  * Create a context on `device`: validates the configuration, records the weight
- * pointers, allocates state, workspace and (kv_cache_mode = 1) the cache for
+ * pointers, allocates state, workspace and (kv_cache_mode != 0) the cache for
  * max_batch x max_seq.  Errors: L2PD_ERR_ARG / L2PD_ERR_SHAPE (d_model, d_ff,
  * n_heads*head_dim multiples of 8; head_dim 64 or 128 for bf16, even and <= 256 for
  * fp32; block_len in [1, 64]; ids inside the vocabulary), L2PD_ERR_OOM, L2PD_ERR_CUDA.

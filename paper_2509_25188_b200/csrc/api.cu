@@ -410,7 +410,7 @@ l2pd_status validate(const l2pd_config *f, const l2pd_weights *w, std::string *w
     return bad("mask_id / eot_id outside the vocabulary or equal");
   if (f->max_batch < 1 || f->max_seq < 2) return bad("max_batch / max_seq too small");
   if (!(f->tau >= 0.f && f->tau <= 1.f)) { *why = "tau outside [0, 1]"; return L2PD_ERR_ARG; }
-  if (f->kv_cache_mode != 0 && f->kv_cache_mode != 1) { *why = "kv_cache_mode must be 0 or 1"; return L2PD_ERR_ARG; }
+  if (f->kv_cache_mode < 0 || f->kv_cache_mode > 2) { *why = "kv_cache_mode must be 0, 1 or 2"; return L2PD_ERR_ARG; }
   if (f->committed_conf_mode != 0 && f->committed_conf_mode != 1) { *why = "committed_conf_mode must be 0 or 1"; return L2PD_ERR_ARG; }
   if (!(f->rms_eps >= 0.f) || !(f->rope_theta > 0.f)) { *why = "rms_eps / rope_theta"; return L2PD_ERR_ARG; }
   if (!w->tok_emb || !w->lm_head || !w->final_norm) { *why = "null weight pointer"; return L2PD_ERR_ARG; }
@@ -616,10 +616,13 @@ l2pd_status l2pd_denoise_step(l2pd_ctx *c, void *stream, const l2pd_step_out *ou
     if (c->h_done[i]) continue;
     SeqMeta &m = c->h_meta[n_slots++];
     const int b = c->h_cur_block[i], S_b = c->P + b * sb, L = c->h_l_eff[i];
-    const bool cached = f.kv_cache_mode == 1 && c->h_cache_block[i] == b;
+    const bool cached = f.kv_cache_mode != 0 && c->h_cache_block[i] == b;
     m.seq = i; m.row0 = T_rows; m.pos0 = cached ? S_b : 0; m.n_rows = L - m.pos0; m.kv_len = L;
     m.blk_start = S_b; m.n_blk_rows = (L - S_b < sb) ? (L - S_b) : sb; m.block = b;
-    if (f.kv_cache_mode == 1) c->h_cache_block[i] = b;
+    // dual cache: a cached step computes the block's rows only; their K/V overwrite the store in place and the
+    // positions after the block are read as the block's first step left them
+    if (cached && f.kv_cache_mode == 2) m.n_rows = m.n_blk_rows;
+    if (f.kv_cache_mode != 0) c->h_cache_block[i] = b;
     T_rows += m.n_rows;
     if (m.n_rows > max_q) max_q = m.n_rows;
     if (L > max_kv) max_kv = L;

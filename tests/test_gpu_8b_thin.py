@@ -47,7 +47,7 @@ def _run(thin8b, *, B, P, G, kv_cache, eot_bias, seed, sample, max_steps=None):
     m = oracle_model(SHAPE, w, lm_head_bias=bias)
     filt = wl.make_filter(s, 0.96, seed=0)
     prompts = wl.make_prompts(B, P, SHAPE, seed=seed)
-    cfg = orc.DecodeConfig(block_len=s, kv_cache=kv_cache)
+    cfg = orc.DecodeConfig(block_len=s, kv_cache=bool(kv_cache), dual_cache=kv_cache == 2)
     dec = binding.Decoder(SHAPE, dev, filt, block_len=s, max_batch=B, max_seq=P + G, kv_cache=kv_cache,
                           lm_head_bias=bias)
     # spread logits (row maxima ~32): |d conf| <= 0.5 max|d logit|, and a logit error of 6e-3 of the row maximum allows 0.1
@@ -119,5 +119,25 @@ def test_batch_of_8_prefix_cache(thin8b):
 
     st, toks, out_len, steps, total = _run(thin8b, B=8, P=1024, G=1024, kv_cache=True, eot_bias=15.0, seed=31,
                                            sample=sample)
+    assert st["oracle_steps"] == 2
+    assert st["replay_checked"] >= 0.9 * sum(st["seq_steps"])
+
+
+def test_dual_cache_single_sequence_and_batch(thin8b):
+    """Dual cache at the 8B widths: in-block steps run 32 rows per sequence (the small-M launch shapes).
+    The oracle follows the first (full) step and two stored-key steps, among them one after [EoT]."""
+    seen = {"eot": False}
+
+    def sample(i, k, state):
+        if i == 0 and state.eot_pos >= 0 and not seen["eot"]:
+            seen["eot"] = True
+            return True
+        return i == 0 and k in (0, 1, 2)
+
+    st, toks, out_len, steps, total = _run(thin8b, B=1, P=256, G=256, kv_cache=2, eot_bias=14.0, seed=11,
+                                           sample=sample)
+    assert st["oracle_steps"] >= 3 and st["replay_checked"] >= 0.9 * st["steps"]
+    st, toks, out_len, steps, total = _run(thin8b, B=8, P=1024, G=1024, kv_cache=2, eot_bias=15.0, seed=31,
+                                           sample=lambda i, k, state: i == 0 and k in (0, 1))
     assert st["oracle_steps"] == 2
     assert st["replay_checked"] >= 0.9 * sum(st["seq_steps"])

@@ -161,27 +161,48 @@ def test_batch_is_independent_and_finished_sequences_drop_out():
     dec.close()
 
 
-def test_prefix_cache_matches_oracle_with_the_same_rule():
+@pytest.mark.parametrize("mode", [1, 2])
+def test_kv_cache_matches_oracle_with_the_same_rule(mode):
+    """mode 1: prefix cache, 2: dual cache (Section 4.3)."""
     shape, w = _tiny()
     s, P, G, B = 16, 40, 64, 2
     filt = wl.make_filter(s, 0.96, seed=3)
     prompts = wl.make_prompts(B, P, shape, seed=21)
     m = oracle_model(shape, w)
-    cfg = orc.DecodeConfig(block_len=s, kv_cache=True)
+    cfg = orc.DecodeConfig(block_len=s, kv_cache=True, dual_cache=mode == 2)
     refs = orc.decode_batch(m, filt, prompts, G, cfg, keep_trace=False)
     b = _b()
-    dec = b.Decoder(shape, w, filt, block_len=s, max_batch=B, max_seq=P + G, kv_cache=True)
+    dec = b.Decoder(shape, w, filt, block_len=s, max_batch=B, max_seq=P + G, kv_cache=mode)
     toks, out_len, steps, _ = dec.decode(prompts, G)
     for i, r in enumerate(refs):
         assert np.array_equal(toks[i], r.response) and steps[i] == r.steps
     st = lockstep(dec, m, filt, cfg, prompts, G, logit_rtol=1e-4, conf_atol=1e-3, p_margin=1e-4)
     assert st["replay_checked"] > 0
-    # cached steps process only the rows from the block start on
+    # cached steps process only the rows from the block start on (dual cache: the block's rows)
     dec.state_reset(prompts, G)
     dec.denoise_step(outputs=False)
     assert dec.last_step_rows == B * (P + G)
     dec.denoise_step(outputs=False)
-    assert dec.last_step_rows == B * G
+    assert dec.last_step_rows == (B * G if mode == 1 else B * s)
+    dec.close()
+
+
+def test_dual_cache_one_token_per_step_with_eot_cut():
+    """Dual cache with the filter off (every step but a block's first reads the store) and an [EoT]
+    bias that cuts the sequence in mid-block, so stored positions beyond L_eff drop out of the keys."""
+    shape, w = _tiny()
+    s, P, G = 16, 40, 64
+    filt = const_filter(s, -50.0)
+    m = oracle_model(shape, w)
+    cfg = orc.DecodeConfig(block_len=s, kv_cache=True, dual_cache=True)
+    seed, bias, want = find_eot_bias(m, shape, filt, G, cfg, P)
+    prompts = wl.make_prompts(1, P, shape, seed=seed)
+    dec = _b().Decoder(shape, w, filt, block_len=s, max_batch=1, max_seq=P + G, kv_cache=2,
+                       lm_head_bias=m.lm_head_bias)
+    toks, out_len, steps, _ = dec.decode(prompts, G)
+    assert np.array_equal(toks[0], want.response) and steps[0] == want.steps and out_len[0] == want.out_len
+    st = lockstep(dec, m, filt, cfg, prompts, G, logit_rtol=1e-4, conf_atol=1e-3, p_margin=1e-4, conf_margin=1e-6)
+    assert st["replay_checked"] == st["steps"] and st["forced"] > 0
     dec.close()
 
 
@@ -247,7 +268,7 @@ def _bf16_shape(**kw):
 
 
 @pytest.mark.parametrize("spread", [False, True])
-@pytest.mark.parametrize("kv_cache", [False, True])
+@pytest.mark.parametrize("kv_cache", [0, 1, 2])
 def test_bf16_small_model_lockstep(spread, kv_cache):
     shape = _bf16_shape()
     w = wl.make_weights(shape, seed=0, final_norm_gain=wl.spread_gain(shape) if spread else 1.0)
@@ -255,7 +276,7 @@ def test_bf16_small_model_lockstep(spread, kv_cache):
     filt = wl.make_filter(s, 0.96, seed=0)
     prompts = wl.make_prompts(B, P, shape, seed=31)
     m = oracle_model(shape, w, lm_head_bias=wl.make_eot_bias(shape, 6.0) if spread else None)
-    cfg = orc.DecodeConfig(block_len=s, kv_cache=kv_cache)
+    cfg = orc.DecodeConfig(block_len=s, kv_cache=kv_cache > 0, dual_cache=kv_cache == 2)
     b = _b()
     dec = b.Decoder(shape, w, filt, block_len=s, max_batch=B, max_seq=P + G, kv_cache=kv_cache,
                     lm_head_bias=m.lm_head_bias)
