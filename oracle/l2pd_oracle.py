@@ -475,3 +475,86 @@ def decode_batch(m: Model, filt: Dict[str, np.ndarray], prompts: np.ndarray, G: 
                  cfg: DecodeConfig, **kw) -> List[DecodeResult]:
     """Sequences are independent: each prompt is decoded on its own."""
     return [decode(m, filt, p, G, cfg, **kw) for p in prompts]
+
+
+# ----------------------------------------------------------------------------
+# Filter training (Algorithm 1, Eq. 5-6, Section 4.1)
+#
+# Stage 1 collects, under the EGP policy, one sample per decoding step: the filter's input
+# (the block's s confidences, as decide() feeds them) and Algorithm 1's targets y_j.  Stage 2
+# minimises the mean binary cross-entropy between sigmoid(f_theta(conf)) and y with AdamW.
+# Readings (the paper gives the optimiser, the learning rate 0.001 and the epoch count only):
+#   * the loss of a batch is the mean over its samples and all s positions (Eq. 6 with
+#     m = samples * s);
+#   * AdamW as published (Loshchilov & Hutter): decoupled weight decay, bias-corrected moments;
+#     beta1 0.9, beta2 0.999, eps 1e-8, weight decay 0.01 unless given;
+#   * an epoch visits the samples in the given order in consecutive batches (batch_size 0 = one
+#     batch holding every sample); the caller shuffles, if it wants to, before the call.
+
+def egp_samples(trace: List[StepRecord], ref: np.ndarray, s: int):
+    """Stage 1 for one decoded sequence: (C[n, s], Y[n, s]) from the steps of an EGP decode.
+    Positions cut off by EoTP carry pred = -1 and therefore the target 0."""
+    C = np.stack([t.filt_in for t in trace]).astype(np.float64)
+    Y = np.zeros((len(trace), s), dtype=np.float64)
+    for n, t in enumerate(trace):
+        pred = np.full(s, -1, dtype=np.int64)
+        pred[: t.n_rows] = t.pred
+        Y[n] = egp_labels(pred, np.asarray(ref)[t.block * s: (t.block + 1) * s])
+    return C, Y
+
+
+def bce_with_logits(z: np.ndarray, y: np.ndarray) -> float:
+    """Eq. 6: -mean[y log sigmoid(z) + (1 - y) log(1 - sigmoid(z))], in the overflow-free form
+    max(z, 0) - z y + log(1 + exp(-|z|))."""
+    return float(np.mean(np.maximum(z, 0.0) - z * y + np.log1p(np.exp(-np.abs(z)))))
+
+
+def filter_loss_and_grads(filt: Dict[str, np.ndarray], C: np.ndarray, Y: np.ndarray):
+    """Loss of Eq. 6 over the batch (C[n, s], Y[n, s]) and its gradient w.r.t. w1, b1, w2, b2."""
+    w1, b1, w2, b2 = (widen(filt[k]) for k in ("w1", "b1", "w2", "b2"))
+    pre = C @ w1.T + b1                       # [n, s]
+    h = np.maximum(pre, 0.0)
+    z = h @ w2.T + b2
+    loss = bce_with_logits(z, Y)
+    dz = (sigmoid(z) - Y) / z.size            # d loss / d z
+    g = {"w2": dz.T @ h, "b2": dz.sum(axis=0)}
+    dh = dz @ w2
+    dpre = dh * (pre > 0.0)
+    g["w1"] = dpre.T @ C
+    g["b1"] = dpre.sum(axis=0)
+    return loss, g
+
+
+def adamw_step(param: np.ndarray, grad: np.ndarray, m: np.ndarray, v: np.ndarray, t: int,
+               lr: float, beta1: float, beta2: float, eps: float, weight_decay: float):
+    """One AdamW update, step count t >= 1; returns (param, m, v)."""
+    param = param * (1.0 - lr * weight_decay)
+    m = beta1 * m + (1.0 - beta1) * grad
+    v = beta2 * v + (1.0 - beta2) * grad * grad
+    m_hat = m / (1.0 - beta1 ** t)
+    v_hat = v / (1.0 - beta2 ** t)
+    return param - lr * m_hat / (np.sqrt(v_hat) + eps), m, v
+
+
+def train_filter(filt0: Dict[str, np.ndarray], C: np.ndarray, Y: np.ndarray, epochs: int,
+                 lr: float = 1e-3, beta1: float = 0.9, beta2: float = 0.999, eps: float = 1e-8,
+                 weight_decay: float = 0.01, batch_size: int = 0):
+    """Stage 2 of Algorithm 1.  Returns (filter, losses): the trained parameters (fp64) and the
+    loss of every update's batch, measured before the update."""
+    names = ("w1", "b1", "w2", "b2")
+    filt = {k: widen(filt0[k]).copy() for k in names}
+    mom = {k: np.zeros_like(filt[k]) for k in names}
+    var = {k: np.zeros_like(filt[k]) for k in names}
+    N = len(C)
+    bs = N if batch_size <= 0 else batch_size
+    losses = []
+    t = 0
+    for _ in range(epochs):
+        for lo in range(0, N, bs):
+            loss, g = filter_loss_and_grads(filt, C[lo: lo + bs], Y[lo: lo + bs])
+            losses.append(loss)
+            t += 1
+            for k in names:
+                filt[k], mom[k], var[k] = adamw_step(filt[k], g[k], mom[k], var[k], t, lr, beta1, beta2, eps,
+                                                     weight_decay)
+    return filt, np.asarray(losses)

@@ -731,3 +731,107 @@ def test_egp_with_the_models_own_answer_as_reference_skips_repeats():
             assert np.array_equal(t.unmask, masked[blk] & orc.egp_labels(t.pred, van.response[blk]))
         masked[blk] &= ~t.unmask
     assert not masked.any()
+
+
+# ----------------------------------------------------------------------------- filter training (Algorithm 1)
+
+def _train_data(s=8, n=40, seed=0):
+    rng = np.random.default_rng(seed)
+    C = rng.uniform(0.0, 1.0, size=(n, s))
+    Y = (C + 0.15 * rng.normal(size=(n, s)) > 0.6).astype(np.float64)      # high confidence -> mostly "unmask"
+    return C, Y
+
+
+def test_bce_at_zero_logits_is_log_two_and_matches_the_definition():
+    """Eq. 5/6: with p = 1/2 everywhere the loss is ln 2 = 0.693 (the paper's curve starts at 0.68);
+    the overflow-free form equals the printed definition where that one is finite."""
+    y = np.array([[0.0, 1.0, 1.0, 0.0]])
+    assert abs(orc.bce_with_logits(np.zeros((1, 4)), y) - math.log(2.0)) < 1e-15
+    z = np.array([[-3.0, 0.5, 2.0, 7.0]])
+    p = 1.0 / (1.0 + np.exp(-z))
+    want = -np.mean(y * np.log(p) + (1 - y) * np.log(1 - p))
+    assert abs(orc.bce_with_logits(z, y) - want) < 1e-12
+    assert np.isfinite(orc.bce_with_logits(np.array([[800.0, -800.0]]), np.array([[0.0, 1.0]])))
+
+
+def test_filter_gradients_match_central_differences():
+    s = 6
+    C, Y = _train_data(s, 12, seed=1)
+    filt = {k: v.astype(np.float64) for k, v in wl.make_filter(s, seed=5).items()}
+    loss, g = orc.filter_loss_and_grads(filt, C, Y)
+    eps = 1e-6
+    rng = np.random.default_rng(2)
+    for k in ("w1", "b1", "w2", "b2"):
+        for _ in range(6):
+            idx = tuple(rng.integers(0, n) for n in filt[k].shape)
+            up = {a: b.copy() for a, b in filt.items()}
+            dn = {a: b.copy() for a, b in filt.items()}
+            up[k][idx] += eps
+            dn[k][idx] -= eps
+            num = (orc.filter_loss_and_grads(up, C, Y)[0] - orc.filter_loss_and_grads(dn, C, Y)[0]) / (2 * eps)
+            assert abs(num - g[k][idx]) < 1e-7, (k, idx, num, g[k][idx])
+
+
+@pytest.mark.parametrize("batch_size", [0, 16])
+def test_training_matches_torch_adamw(batch_size):
+    """The same network, loss and optimiser built from torch's CPU library (nn.Linear,
+    binary_cross_entropy_with_logits, optim.AdamW) in fp64: parameters and loss curve agree."""
+    s = 8
+    C, Y = _train_data(s, 40, seed=3)
+    f0 = wl.make_filter(s, seed=7)
+    epochs = 25
+    filt, losses = orc.train_filter(f0, C, Y, epochs, lr=1e-2, weight_decay=0.05, batch_size=batch_size)
+    l1, l2 = torch.nn.Linear(s, s).double(), torch.nn.Linear(s, s).double()
+    with torch.no_grad():
+        l1.weight.copy_(torch.from_numpy(f0["w1"].astype(np.float64))); l1.bias.copy_(torch.from_numpy(f0["b1"].astype(np.float64)))
+        l2.weight.copy_(torch.from_numpy(f0["w2"].astype(np.float64))); l2.bias.copy_(torch.from_numpy(f0["b2"].astype(np.float64)))
+    opt = torch.optim.AdamW(list(l1.parameters()) + list(l2.parameters()), lr=1e-2, betas=(0.9, 0.999), eps=1e-8,
+                            weight_decay=0.05)
+    tc, ty = torch.from_numpy(C), torch.from_numpy(Y)
+    bs = len(C) if batch_size == 0 else batch_size
+    ref_losses = []
+    for _ in range(epochs):
+        for lo in range(0, len(C), bs):
+            opt.zero_grad()
+            z = l2(torch.relu(l1(tc[lo: lo + bs])))
+            loss = torch.nn.functional.binary_cross_entropy_with_logits(z, ty[lo: lo + bs])
+            loss.backward()
+            opt.step()
+            ref_losses.append(float(loss.detach()))
+    assert np.allclose(losses, ref_losses, rtol=0, atol=1e-10)
+    assert np.allclose(filt["w1"], l1.weight.detach().numpy(), atol=1e-9)
+    assert np.allclose(filt["b1"], l1.bias.detach().numpy(), atol=1e-9)
+    assert np.allclose(filt["w2"], l2.weight.detach().numpy(), atol=1e-9)
+    assert np.allclose(filt["b2"], l2.bias.detach().numpy(), atol=1e-9)
+    assert losses[-1] < losses[0]
+
+
+def test_first_adamw_step_moves_every_parameter_by_lr():
+    """Closed form: at t = 1 the bias-corrected ratio m_hat / sqrt(v_hat) is sign(g), so without
+    weight decay each parameter with a non-zero gradient moves by lr (up to eps)."""
+    p = np.array([0.5, -0.25, 2.0])
+    g = np.array([0.3, -4.0, 1e-3])
+    q, m, v = orc.adamw_step(p, g, np.zeros(3), np.zeros(3), 1, 1e-3, 0.9, 0.999, 1e-8, 0.0)
+    assert np.allclose(q, p - 1e-3 * np.sign(g), atol=1e-7)
+    q2, _, _ = orc.adamw_step(p, g, np.zeros(3), np.zeros(3), 1, 1e-3, 0.9, 0.999, 1e-8, 0.1)
+    assert np.allclose(q2 - q, -1e-3 * 0.1 * p, atol=1e-12)     # decay is decoupled from the gradient
+
+
+def test_egp_samples_are_algorithm_one_targets():
+    """Stage 1: the samples of an EGP decode are the filter inputs of its steps and pred == ref."""
+    s, G, V = 4, 8, 12
+    m = _toy_model(V)
+    ref = np.array([1, 2, 3, 4, 5, 6, 7, 8])
+    r = orc.decode(m, None, [0], G, orc.DecodeConfig(block_len=s, rule="egp"),
+                   predictor=_chain_predictor(ref, V, wrong=0), ref=ref)
+    C, Y = orc.egp_samples(r.trace, ref, s)
+    assert C.shape == Y.shape == (G, s)
+    for k in range(G):
+        want = np.zeros(s)
+        want[: k % s + 1] = 1.0                    # committed positions and the one that just turned right
+        assert np.array_equal(Y[k], want)
+        assert np.array_equal(C[k], r.trace[k].filt_in)
+    # the trained filter separates the two groups of this toy: its loss falls well below ln 2
+    f0 = wl.make_filter(s, seed=1)
+    _, losses = orc.train_filter(f0, C, Y, 300, lr=1e-2)
+    assert losses[0] > 0.3 and losses[-1] < 0.6 * losses[0]
