@@ -189,6 +189,36 @@ enum { L2PD_RULE_FILTER = 0, L2PD_RULE_CONFIDENCE = 1, L2PD_RULE_EGP = 2 };
 l2pd_status l2pd_set_unmask_rule(l2pd_ctx *ctx, void *stream, int32_t rule, float conf_threshold,
                                  const int32_t *d_reference, int32_t ref_rows, int32_t ref_len);
 
+/*
+ * Algorithm 1, stage 1 (data collection): while a sink is set, every denoising step appends one
+ * sample per sequence taking part in it, in step order and, within a step, in sequence order:
+ *   d_c [capacity, s] float  the filter's input of that step (the block's confidences as f_theta reads them)
+ *   d_y [capacity, s] uint8  the target y_j = 1 where the prediction equals the reference token (rule
+ *                            L2PD_RULE_EGP; 0 everywhere under the other rules and at positions cut off by EoTP)
+ * DEVICE arrays, borrowed until the sink is replaced or cleared (NULL, NULL, 0).  A step that would
+ * overflow the capacity returns L2PD_ERR_SHAPE and appends nothing.  Setting a sink resets the count.
+ */
+l2pd_status l2pd_set_collect(l2pd_ctx *ctx, float *d_c, uint8_t *d_y, int64_t capacity);
+int64_t l2pd_collect_count(const l2pd_ctx *ctx);
+
+/*
+ * Algorithm 1, stage 2 (Eq. 6; Section 4.1): trains the two-layer filter z = W2 relu(W1 c + b1) + b2 on N
+ * samples with AdamW (decoupled weight decay, bias-corrected moments, moments start at zero).  An epoch
+ * visits the samples in order in batches of batch_size (0 = all N in one batch); the loss of a batch is the
+ * mean over its samples and the s positions.  Arithmetic is fp32; a run is bit-reproducible on a given GPU.
+ * d_c [N, s] float, d_y [N, s] uint8 (0 / 1): DEVICE.  d_w1 [s, s], d_b1 [s], d_w2 [s, s], d_b2 [s]: DEVICE fp32,
+ * initial values in, trained values out.  h_losses: HOST [epochs * ceil(N / batch)] or NULL, the loss of every
+ * update's batch measured before the update.  Runs on the current device, allocates and frees its scratch,
+ * returns after the stream has finished.  s in [1, 64] (else L2PD_ERR_SHAPE); bad hyper-parameters L2PD_ERR_ARG.
+ */
+typedef struct {
+  float lr, beta1, beta2, eps, weight_decay;   /* the paper gives lr = 0.001; AdamW's published defaults: 0.9, 0.999, 1e-8, 0.01 */
+  int32_t epochs;                              /* the paper trains for 5,000 */
+  int32_t batch_size;                          /* 0: full batch */
+} l2pd_train_config;
+l2pd_status l2pd_filter_train(void *stream, int32_t s, int64_t N, const float *d_c, const uint8_t *d_y, float *d_w1,
+                              float *d_b1, float *d_w2, float *d_b2, const l2pd_train_config *cfg, float *h_losses);
+
 /* Number of sequences that still need steps (0 before the first reset). */
 int32_t l2pd_num_active(const l2pd_ctx *ctx);
 

@@ -47,6 +47,11 @@ class Weights(C.Structure):
                 ("filt_w1", C.c_void_p), ("filt_b1", C.c_void_p), ("filt_w2", C.c_void_p), ("filt_b2", C.c_void_p)]
 
 
+class TrainConfig(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("weight_decay", C.c_float), ("epochs", C.c_int32), ("batch_size", C.c_int32)]
+
+
 class StepOut(C.Structure):
     _fields_ = [("d_conf", C.c_void_p), ("d_pred", C.c_void_p), ("d_p", C.c_void_p),
                 ("d_unmask", C.c_void_p), ("d_logits", C.c_void_p),
@@ -55,7 +60,7 @@ class StepOut(C.Structure):
 
 
 EXPORTS = ["l2pd_init", "l2pd_state_reset", "l2pd_denoise_step", "l2pd_decode", "l2pd_num_active",
-           "l2pd_state_tokens", "l2pd_state_masked", "l2pd_set_unmask_rule", "l2pd_set_capture", "l2pd_last_step_rows",
+           "l2pd_state_tokens", "l2pd_state_masked", "l2pd_set_unmask_rule", "l2pd_set_collect", "l2pd_collect_count", "l2pd_filter_train", "l2pd_set_capture", "l2pd_last_step_rows",
            "l2pd_launch_count", "l2pd_last_step_ms", "l2pd_profile_enable", "l2pd_profile_read", "l2pd_last_error", "l2pd_destroy",
            "l2pd_gemm_bf16", "l2pd_gemm_bf16_residual", "l2pd_gemm_bf16_swiglu", "l2pd_lm_head_bf16",
            "l2pd_lm_head_scratch_elems", "l2pd_attention_bf16", "l2pd_lm_head_bf16_static"]
@@ -82,6 +87,10 @@ def _load() -> C.CDLL:
     lib.l2pd_state_masked.restype = vp
     lib.l2pd_set_capture.argtypes = [vp, vp, i64]
     lib.l2pd_set_unmask_rule.argtypes = [vp, vp, i32, f32, vp, i32, i32]
+    lib.l2pd_set_collect.argtypes = [vp, vp, vp, i64]
+    lib.l2pd_collect_count.argtypes = [vp]
+    lib.l2pd_collect_count.restype = i64
+    lib.l2pd_filter_train.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp, vp, C.POINTER(TrainConfig), vp]
     lib.l2pd_last_step_rows.argtypes = [vp]
     lib.l2pd_launch_count.argtypes = [vp]
     lib.l2pd_launch_count.restype = i64
@@ -277,6 +286,23 @@ class Decoder:
                                         int(ref.shape[1]) if ref is not None else 0), self.ctx)
         self._reference = ref
 
+    def set_collect(self, capacity: int):
+        """Starts (capacity > 0) or stops (0) collecting Algorithm 1's samples; returns the device sinks."""
+        if capacity <= 0:
+            _check(lib.l2pd_set_collect(self.ctx, None, None, 0), self.ctx)
+            self._sink = None
+            return None
+        dev = "cuda:%d" % self.device
+        c = torch.zeros(capacity, self.block_len, device=dev)
+        y = torch.zeros(capacity, self.block_len, dtype=torch.uint8, device=dev)
+        _check(lib.l2pd_set_collect(self.ctx, c.data_ptr(), y.data_ptr(), capacity), self.ctx)
+        self._sink = (c, y)
+        return c, y
+
+    @property
+    def collect_count(self) -> int:
+        return int(lib.l2pd_collect_count(self.ctx))
+
     # ---- state and instrumentation -------------------------------------------------------------
     @property
     def num_active(self) -> int:
@@ -393,3 +419,22 @@ def attention_bf16(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, H: int, dh
     _check(lib.l2pd_attention_bf16(_stream(), q.data_ptr(), k.data_ptr(), v.data_ptr(), out.data_ptr(),
                                    Tq, Tk, H, dh, q.stride(0), k.stride(0), out.stride(0), impl, 1))
     return out
+
+
+def filter_train(filt: Dict[str, np.ndarray], C_in, Y_in, epochs: int, lr: float = 1e-3, beta1: float = 0.9,
+                 beta2: float = 0.999, eps: float = 1e-8, weight_decay: float = 0.01, batch_size: int = 0,
+                 device: int = 0):
+    """Algorithm 1, stage 2 on the GPU.  C_in [N, s] float, Y_in [N, s] 0/1 (numpy or device tensors).
+    Returns (trained filter as numpy fp32 arrays, losses [updates])."""
+    dev = "cuda:%d" % device
+    torch.cuda.set_device(device)
+    tc = (C_in if isinstance(C_in, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(C_in))).to(dev, torch.float32).contiguous()
+    ty = (Y_in if isinstance(Y_in, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(Y_in))).to(dev, torch.uint8).contiguous()
+    N, s = int(tc.shape[0]), int(tc.shape[1])
+    p = {k: torch.from_numpy(np.ascontiguousarray(filt[k], dtype=np.float32)).to(dev) for k in ("w1", "b1", "w2", "b2")}
+    bs = N if batch_size <= 0 else batch_size
+    losses = np.zeros(max(epochs * (-(-N // bs)), 1), np.float32)
+    cfg = TrainConfig(lr, beta1, beta2, eps, weight_decay, epochs, batch_size)
+    _check(lib.l2pd_filter_train(_stream(), s, N, tc.data_ptr(), ty.data_ptr(), p["w1"].data_ptr(), p["b1"].data_ptr(),
+                                 p["w2"].data_ptr(), p["b2"].data_ptr(), C.byref(cfg), losses.ctypes.data), None)
+    return {k: v.cpu().numpy() for k, v in p.items()}, losses[: epochs * (-(-N // bs))]

@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OUT = os.path.join(HERE, "libl2pd.so")
 OBJ = os.path.join(HERE, "_build")
-SOURCES = ["api.cu", "elementwise.cu", "simt.cu", "decide.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "lm_head_static.cu"]
+SOURCES = ["api.cu", "elementwise.cu", "simt.cu", "decide.cu", "gemm_tcgen05.cu", "attention.cu", "attention_tc.cu", "lm_head_static.cu", "filter_train.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC"]

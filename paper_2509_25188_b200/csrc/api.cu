@@ -40,6 +40,9 @@ struct l2pd_ctx {
   float conf_threshold = 0.9f;
   const int32_t *d_ref = nullptr;       // EGP: reference answers [ref_rows, ref_len], borrowed
   int ref_rows = 0, ref_len = 0;
+  float *collect_c = nullptr;           // sample sink of l2pd_set_collect
+  uint8_t *collect_y = nullptr;
+  int64_t collect_cap = 0, collect_n = 0;
   bool has_state = false;
   int32_t *d_tokens = nullptr;
   uint8_t *d_masked = nullptr;
@@ -376,6 +379,11 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
   a.use_filter = f.use_filter; a.use_eotp = f.use_eotp; a.committed_conf_mode = f.committed_conf_mode;
   a.eot_id = f.eot_id; a.summary = c->d_summary;
   a.rule = c->rule; a.conf_threshold = c->conf_threshold; a.ref = c->d_ref;
+  if (c->collect_c) {
+    if (c->collect_n + n_slots > c->collect_cap) return set_err(c, L2PD_ERR_SHAPE, "sample sink full (%lld of %lld)", (long long)c->collect_n, (long long)c->collect_cap);
+    a.collect_c = c->collect_c; a.collect_y = c->collect_y; a.collect_base = c->collect_n;
+    c->collect_n += n_slots;
+  }
   if (out) { a.o_conf = out->d_conf; a.o_pred = out->d_pred; a.o_p = out->d_p; a.o_unmask = out->d_unmask; }
   CKLK(L2PD_K_DECIDE, launch_decide(s, a, n_slots));
   return L2PD_OK;
@@ -710,6 +718,56 @@ l2pd_status l2pd_set_unmask_rule(l2pd_ctx *c, void *stream, int32_t rule, float 
   c->ref_rows = rule == L2PD_RULE_EGP ? ref_rows : 0;
   c->ref_len = rule == L2PD_RULE_EGP ? ref_len : 0;
   return L2PD_OK;
+}
+
+l2pd_status l2pd_set_collect(l2pd_ctx *c, float *d_c, uint8_t *d_y, int64_t capacity) {
+  if (!c) return L2PD_ERR_ARG;
+  if ((d_c == nullptr) != (d_y == nullptr) || (d_c && capacity < 1)) return set_err(c, L2PD_ERR_ARG, "sample sink: both arrays and a capacity, or neither");
+  c->collect_c = d_c; c->collect_y = d_y; c->collect_cap = d_c ? capacity : 0; c->collect_n = 0;
+  return L2PD_OK;
+}
+int64_t l2pd_collect_count(const l2pd_ctx *c) { return c ? c->collect_n : 0; }
+
+l2pd_status l2pd_filter_train(void *stream, int32_t s, int64_t N, const float *d_c, const uint8_t *d_y, float *d_w1,
+                              float *d_b1, float *d_w2, float *d_b2, const l2pd_train_config *t, float *h_losses) {
+  if (!d_c || !d_y || !d_w1 || !d_b1 || !d_w2 || !d_b2 || !t) return L2PD_ERR_ARG;
+  if (s < 1 || s > 64 || N < 1) return L2PD_ERR_SHAPE;
+  if (t->epochs < 0 || t->batch_size < 0 || !(t->lr > 0.f) || !(t->beta1 >= 0.f && t->beta1 < 1.f) ||
+      !(t->beta2 >= 0.f && t->beta2 < 1.f) || !(t->eps > 0.f) || !(t->weight_decay >= 0.f)) return L2PD_ERR_ARG;
+  cudaStream_t st = (cudaStream_t)stream;
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return L2PD_ERR_CUDA;
+  const int P = 2 * (s * s + s);
+  const int64_t bs = t->batch_size > 0 ? t->batch_size : N;
+  const int64_t per_epoch = (N + bs - 1) / bs, updates = per_epoch * t->epochs;
+  float *theta = nullptr, *gpart = nullptr, *losses = nullptr;
+  auto cleanup = [&]() { cudaFree(theta); cudaFree(gpart); cudaFree(losses); };
+  if (cudaMalloc(&theta, sizeof(float) * 3 * P) != cudaSuccess || cudaMalloc(&gpart, sizeof(float) * (size_t)sms * (P + 1)) != cudaSuccess ||
+      cudaMalloc(&losses, sizeof(float) * (size_t)(updates > 0 ? updates : 1)) != cudaSuccess) { cleanup(); return L2PD_ERR_OOM; }
+  float *m = theta + P, *v = theta + 2 * P;
+  const size_t ss = sizeof(float) * s * s, sv = sizeof(float) * s;
+  bool ok = cudaMemcpyAsync(theta, d_w1, ss, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+            cudaMemcpyAsync(theta + s * s, d_b1, sv, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+            cudaMemcpyAsync(theta + s * s + s, d_w2, ss, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+            cudaMemcpyAsync(theta + 2 * s * s + s, d_b2, sv, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+            cudaMemsetAsync(m, 0, sizeof(float) * 2 * P, st) == cudaSuccess;
+  FilterTrainHyper h{t->lr, t->beta1, t->beta2, t->eps, t->weight_decay};
+  double p1 = 1.0, p2 = 1.0;   // beta^t, carried in double
+  int64_t u = 0;
+  for (int e = 0; ok && e < t->epochs; ++e)
+    for (int64_t lo = 0; ok && lo < N; lo += bs, ++u) {
+      p1 *= t->beta1; p2 *= t->beta2;
+      ok = launch_filter_update(st, d_c, d_y, lo, (N - lo < bs ? N - lo : bs), s, theta, m, v, gpart, sms, h, 1.0 - p1, 1.0 - p2,
+                                losses + u) == cudaSuccess;
+    }
+  ok = ok && cudaMemcpyAsync(d_w1, theta, ss, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+       cudaMemcpyAsync(d_b1, theta + s * s, sv, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+       cudaMemcpyAsync(d_w2, theta + s * s + s, ss, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+       cudaMemcpyAsync(d_b2, theta + 2 * s * s + s, sv, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  if (ok && h_losses && updates > 0) ok = cudaMemcpyAsync(h_losses, losses, sizeof(float) * updates, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+  ok = (cudaStreamSynchronize(st) == cudaSuccess) && ok;
+  cleanup();
+  return ok ? L2PD_OK : L2PD_ERR_CUDA;
 }
 
 int32_t l2pd_num_active(const l2pd_ctx *c) { return c ? c->n_active : 0; }

@@ -132,10 +132,19 @@ struct DecideArgs {
   int rule;                       // 0 filter (Algorithm 2), 1 fixed confidence threshold, 2 EGP (Section 3.1)
   float conf_threshold;           // rule 1
   const int32_t *ref;             // rule 2: reference answers [B, G]
+  float *collect_c; uint8_t *collect_y; int64_t collect_base;   // optional: slot k appends (filter input, pred == ref) as sample collect_base + k
   StepSummary *summary;           // [max_batch], indexed by sequence
   float *o_conf; int32_t *o_pred; float *o_p; uint8_t *o_unmask;   // optional [B, s]
 };
 cudaError_t launch_decide(cudaStream_t st, const DecideArgs &a, int n_slots);
+
+// filter_train.cu : one AdamW update of the filter on the samples [n0, n0 + n) (Algorithm 1, Eq. 6).
+// theta / m / v: packed W1 [s*s], b1 [s], W2 [s*s], b2 [s]; gpart: [grid, 2*(s*s+s) + 1] scratch;
+// bc1 / bc2 = 1 - beta^t for this update's step count t; loss_out receives the batch's loss before the update.
+struct FilterTrainHyper { float lr, beta1, beta2, eps, weight_decay; };
+cudaError_t launch_filter_update(cudaStream_t st, const float *C, const uint8_t *Y, int64_t n0, int64_t n, int s,
+                                 float *theta, float *m, float *v, float *gpart, int grid, const FilterTrainHyper &h,
+                                 double bc1, double bc2, float *loss_out);
 
 // gemm_tcgen05.cu
 struct TmaDesc { CUtensorMap map; };

@@ -140,6 +140,11 @@ __global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
       s_masked[j] = 0;
       if (a.use_eotp && s_commit[j] == a.eot_id) atomicMin(&s_e, g0 + j);
     }
+    if (a.collect_c) {   // stage 1 of Algorithm 1: the filter's input and the target y_j = [pred_j == r_j]
+      const int64_t row = a.collect_base + slot;
+      a.collect_c[row * s + j] = s_c[j];
+      a.collect_y[row * s + j] = (a.rule == 2 && s_pred[j] == a.ref[(int64_t)seq * a.G + g0 + j]) ? 1 : 0;
+    }
     if (a.o_conf) a.o_conf[(int64_t)seq * s + j] = s_conf[j];
     if (a.o_pred) a.o_pred[(int64_t)seq * s + j] = s_pred[j];
     if (a.o_p) a.o_p[(int64_t)seq * s + j] = s_p[j];
