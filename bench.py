@@ -381,6 +381,24 @@ def run_ours(args):
                            "rows_per_s": rows / (t_in * 1e-3)}
             decx.close()
 
+        # filter training at the paper's scale (Section 4.1: 2,640 prompts, 5,000 epochs, lr 0.001): synthetic samples,
+        # one per decoding step of a 32-step-per-prompt EGP run; the whole of stage 2 on the device
+        n_samp = 2640 * 32
+        rng = np.random.default_rng(0)
+        c_s = rng.uniform(0.0, 1.0, size=(n_samp, s)).astype(np.float32)
+        y_s = (c_s + 0.15 * rng.normal(size=(n_samp, s)) > 0.6).astype(np.uint8)
+        tc_s, ty_s = torch.from_numpy(c_s).to(dev), torch.from_numpy(y_s).to(dev)
+        binding.filter_train(filt, tc_s, ty_s, 20)
+        ev0.record()
+        _, tr_losses = binding.filter_train(filt, tc_s, ty_s, 5000)
+        ev1.record()
+        torch.cuda.synchronize()
+        ms_tr = ev0.elapsed_time(ev1)
+        fl_epoch = 10.0 * n_samp * s * s        # two products forward, three backward, 2 flops per multiply-add
+        extra["filter_training"] = {"samples": n_samp, "block_len": s, "epochs": 5000, "batch": "full", "ms": ms_tr,
+                                    "us_per_epoch": 1e3 * ms_tr / 5000, "gflops": fl_epoch * 5000 / (ms_tr * 1e-3) / 1e9,
+                                    "loss_first": float(tr_losses[0]), "loss_last": float(tr_losses[-1])}
+
     if rank == 0:
         T, R = B * (P + G), B * s
         work = step_work(SHAPE, T, P + G, R)
