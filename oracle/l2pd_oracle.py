@@ -228,7 +228,18 @@ def confidence_head(logits: np.ndarray):
 
 
 def filter_logits(filt: Dict[str, np.ndarray], conf_block: np.ndarray) -> np.ndarray:
-    """f_theta: z = W2 relu(W1 c + b1) + b2 on the block's s confidences."""
+    """f_theta: z = W2 relu(W1 c + b1) + b2 on the block's s confidences (Section 3.2).
+
+    The depth study of Section 4.4 (one, two and four layers) uses filt["layers"], a list of
+    (W, b) pairs of Linear(s, s) layers with ReLU between consecutive layers and none after the last.
+    """
+    if "layers" in filt:
+        h = conf_block
+        for k, (w, b) in enumerate(filt["layers"]):
+            if k > 0:
+                h = np.maximum(h, 0.0)
+            h = widen(w) @ h + widen(b)
+        return h
     h = widen(filt["w1"]) @ conf_block + widen(filt["b1"])
     h = np.maximum(h, 0.0)
     return widen(filt["w2"]) @ h + widen(filt["b2"])

@@ -835,3 +835,29 @@ def test_egp_samples_are_algorithm_one_targets():
     f0 = wl.make_filter(s, seed=1)
     _, losses = orc.train_filter(f0, C, Y, 300, lr=1e-2)
     assert losses[0] > 0.3 and losses[-1] < 0.6 * losses[0]
+
+
+# ----------------------------------------------------------------------------- filter depth (Section 4.4)
+
+def test_filter_depth_variants():
+    """One layer is an affine map; the two-entry list equals the named two-layer filter; four layers
+    equal torch's Sequential of Linear / ReLU in fp64."""
+    s = 6
+    rng = np.random.default_rng(3)
+    c = rng.uniform(size=s)
+    f2 = wl.make_filter(s, seed=2)
+    two = {"layers": [(f2["w1"], f2["b1"]), (f2["w2"], f2["b2"])]}
+    assert np.allclose(orc.filter_logits(two, c), orc.filter_logits(f2, c), atol=0)
+    one = {"layers": [(f2["w1"], f2["b1"])]}
+    assert np.allclose(orc.filter_logits(one, c), f2["w1"].astype(np.float64) @ c + f2["b1"], atol=1e-15)
+    ws = [(rng.normal(size=(s, s)), rng.normal(size=s)) for _ in range(4)]
+    mods = []
+    for k, (w, b) in enumerate(ws):
+        lin = torch.nn.Linear(s, s).double()
+        with torch.no_grad():
+            lin.weight.copy_(torch.from_numpy(w)); lin.bias.copy_(torch.from_numpy(b))
+        mods += ([torch.nn.ReLU()] if k else []) + [lin]
+    want = torch.nn.Sequential(*mods)(torch.from_numpy(c)).detach().numpy()
+    assert np.allclose(orc.filter_logits({"layers": ws}, c), want, atol=1e-12)
+    # parameter counts of the three depths at s = 32: 1,056 / 2,112 (the printed count) / 4,224
+    assert [k * (32 * 32 + 32) for k in (1, 2, 4)] == [1056, int(paper_constants()["filter_params_at_block_32"]), 4224]
