@@ -190,6 +190,16 @@ l2pd_status l2pd_set_unmask_rule(l2pd_ctx *ctx, void *stream, int32_t rule, floa
                                  const int32_t *d_reference, int32_t ref_rows, int32_t ref_len);
 
 /*
+ * Filter depth (Section 4.4 compares one, two and four layers): replaces the two-layer filter given at
+ * init by n_layers Linear(s, s) layers, z = W_n relu(... relu(W_1 c + b_1) ...) + b_n, ReLU between
+ * consecutive layers, none after the last; p = sigmoid(z).  d_w, d_b: HOST arrays of n_layers DEVICE
+ * pointers ([s, s] row-major and [s], fp32), borrowed until replaced or the context is destroyed.
+ * n_layers = 0 goes back to the init-time filter; n_layers in [1, 4] also turns the filter on if the
+ * configuration had use_filter = 0.  May be called between steps.
+ */
+l2pd_status l2pd_set_filter(l2pd_ctx *ctx, int32_t n_layers, const float *const *d_w, const float *const *d_b);
+
+/*
  * Algorithm 1, stage 1 (data collection): while a sink is set, every denoising step appends one
  * sample per sequence taking part in it, in step order and, within a step, in sequence order:
  *   d_c [capacity, s] float  the filter's input of that step (the block's confidences as f_theta reads them)

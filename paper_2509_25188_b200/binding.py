@@ -60,7 +60,7 @@ class StepOut(C.Structure):
 
 
 EXPORTS = ["l2pd_init", "l2pd_state_reset", "l2pd_denoise_step", "l2pd_decode", "l2pd_num_active",
-           "l2pd_state_tokens", "l2pd_state_masked", "l2pd_set_unmask_rule", "l2pd_set_collect", "l2pd_collect_count", "l2pd_filter_train", "l2pd_set_capture", "l2pd_last_step_rows",
+           "l2pd_state_tokens", "l2pd_state_masked", "l2pd_set_unmask_rule", "l2pd_set_filter", "l2pd_set_collect", "l2pd_collect_count", "l2pd_filter_train", "l2pd_set_capture", "l2pd_last_step_rows",
            "l2pd_launch_count", "l2pd_last_step_ms", "l2pd_profile_enable", "l2pd_profile_read", "l2pd_last_error", "l2pd_destroy",
            "l2pd_gemm_bf16", "l2pd_gemm_bf16_residual", "l2pd_gemm_bf16_swiglu", "l2pd_lm_head_bf16",
            "l2pd_lm_head_scratch_elems", "l2pd_attention_bf16", "l2pd_lm_head_bf16_static"]
@@ -87,6 +87,7 @@ def _load() -> C.CDLL:
     lib.l2pd_state_masked.restype = vp
     lib.l2pd_set_capture.argtypes = [vp, vp, i64]
     lib.l2pd_set_unmask_rule.argtypes = [vp, vp, i32, f32, vp, i32, i32]
+    lib.l2pd_set_filter.argtypes = [vp, i32, vp, vp]
     lib.l2pd_set_collect.argtypes = [vp, vp, vp, i64]
     lib.l2pd_collect_count.argtypes = [vp]
     lib.l2pd_collect_count.restype = i64
@@ -285,6 +286,17 @@ class Decoder:
                                         int(ref.shape[0]) if ref is not None else 0,
                                         int(ref.shape[1]) if ref is not None else 0), self.ctx)
         self._reference = ref
+
+    def set_filter_layers(self, layers):
+        """layers: list of (W [s, s], b [s]) numpy arrays, 1 to 4 of them; [] restores the init-time filter."""
+        dev = "cuda:%d" % self.device
+        ws = [torch.from_numpy(np.ascontiguousarray(w, dtype=np.float32)).to(dev) for w, _ in layers]
+        bs = [torch.from_numpy(np.ascontiguousarray(b, dtype=np.float32)).to(dev) for _, b in layers]
+        n = len(layers)
+        pw = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in ws])
+        pb = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in bs])
+        _check(lib.l2pd_set_filter(self.ctx, n, pw, pb), self.ctx)
+        self._filter_layers = (ws, bs)
 
     def set_collect(self, capacity: int):
         """Starts (capacity > 0) or stops (0) collecting Algorithm 1's samples; returns the device sinks."""

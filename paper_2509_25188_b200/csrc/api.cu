@@ -40,6 +40,8 @@ struct l2pd_ctx {
   float conf_threshold = 0.9f;
   const int32_t *d_ref = nullptr;       // EGP: reference answers [ref_rows, ref_len], borrowed
   int ref_rows = 0, ref_len = 0;
+  int n_filter_layers = 0;              // l2pd_set_filter: 0 = the two-layer filter given at init
+  const float *flt_w[4] = {}, *flt_b[4] = {};
   float *collect_c = nullptr;           // sample sink of l2pd_set_collect
   uint8_t *collect_y = nullptr;
   int64_t collect_cap = 0, collect_n = 0;
@@ -379,6 +381,9 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
   a.use_filter = f.use_filter; a.use_eotp = f.use_eotp; a.committed_conf_mode = f.committed_conf_mode;
   a.eot_id = f.eot_id; a.summary = c->d_summary;
   a.rule = c->rule; a.conf_threshold = c->conf_threshold; a.ref = c->d_ref;
+  a.n_filter_layers = c->n_filter_layers;
+  for (int k = 0; k < 4; ++k) { a.fw[k] = c->flt_w[k]; a.fb[k] = c->flt_b[k]; }
+  if (c->n_filter_layers > 0) a.use_filter = 1;
   if (c->collect_c) {
     if (c->collect_n + n_slots > c->collect_cap) return set_err(c, L2PD_ERR_SHAPE, "sample sink full (%lld of %lld)", (long long)c->collect_n, (long long)c->collect_cap);
     a.collect_c = c->collect_c; a.collect_y = c->collect_y; a.collect_base = c->collect_n;
@@ -717,6 +722,16 @@ l2pd_status l2pd_set_unmask_rule(l2pd_ctx *c, void *stream, int32_t rule, float 
   c->d_ref = rule == L2PD_RULE_EGP ? d_reference : nullptr;
   c->ref_rows = rule == L2PD_RULE_EGP ? ref_rows : 0;
   c->ref_len = rule == L2PD_RULE_EGP ? ref_len : 0;
+  return L2PD_OK;
+}
+
+l2pd_status l2pd_set_filter(l2pd_ctx *c, int32_t n_layers, const float *const *d_w, const float *const *d_b) {
+  if (!c) return L2PD_ERR_ARG;
+  if (n_layers < 0 || n_layers > 4) return set_err(c, L2PD_ERR_ARG, "filter depth %d outside [0, 4]", n_layers);
+  for (int k = 0; k < n_layers; ++k)
+    if (!d_w || !d_b || !d_w[k] || !d_b[k]) return set_err(c, L2PD_ERR_ARG, "filter layer %d: null pointer", k);
+  c->n_filter_layers = n_layers;
+  for (int k = 0; k < 4; ++k) { c->flt_w[k] = k < n_layers ? d_w[k] : nullptr; c->flt_b[k] = k < n_layers ? d_b[k] : nullptr; }
   return L2PD_OK;
 }
 

@@ -127,6 +127,8 @@ struct DecideArgs {
   uint8_t *masked;                // [B, G]
   SeqState st;
   const float *w1, *b1, *w2, *b2;
+  int n_filter_layers;            // 0: the two-layer filter above; 1..4: fw[k] / fb[k], ReLU between layers (Section 4.4)
+  const float *fw[4], *fb[4];
   float tau;
   int use_filter, use_eotp, committed_conf_mode, eot_id;
   int rule;                       // 0 filter (Algorithm 2), 1 fixed confidence threshold, 2 EGP (Section 3.1)

@@ -25,6 +25,7 @@ __global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
   __shared__ int s_pred[MAX_S];
   __shared__ float s_c[MAX_S];
   __shared__ float s_h[MAX_S];
+  __shared__ float s_t[MAX_S];
   __shared__ float s_p[MAX_S];
   __shared__ int s_masked[MAX_S];
   __shared__ int s_unmask[MAX_S];
@@ -85,7 +86,22 @@ __global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
     s_c[j] = c;
   }
   __syncthreads();
-  if (a.use_filter && a.rule == 0) {
+  if (a.use_filter && a.rule == 0 && a.n_filter_layers > 0) {
+    // depth variants: x <- W_k x + b_k with ReLU between consecutive layers; s_h / s_t alternate as output
+    // (s_c, the filter's input, stays intact for the sample sink)
+    float *src = s_c, *dst = s_h;
+    for (int k = 0; k < a.n_filter_layers; ++k) {
+      if (threadIdx.x < s) {
+        const int j = threadIdx.x;
+        float z = a.fb[k][j];
+        for (int i = 0; i < s; ++i) z = fmaf(a.fw[k][j * s + i], k > 0 ? fmaxf(src[i], 0.f) : src[i], z);
+        dst[j] = z;
+        if (k + 1 == a.n_filter_layers) s_p[j] = 1.0f / (1.0f + expf(-z));
+      }
+      __syncthreads();
+      src = dst; dst = (dst == s_h) ? s_t : s_h;
+    }
+  } else if (a.use_filter && a.rule == 0) {
     if (threadIdx.x < s) {
       int j = threadIdx.x;
       float h = a.b1[j];

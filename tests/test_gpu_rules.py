@@ -117,3 +117,32 @@ def test_rule_errors():
     dec.set_unmask_rule("filter")
     dec.state_reset(prompts, d.gen_len)
     dec.close()
+
+
+@pytest.mark.parametrize("depth", [1, 2, 4])
+def test_filter_depth_variants(depth):
+    """Section 4.4: one-, two- and four-layer filters; decisions bit-exact against the oracle in lockstep."""
+    shape, w, d, filt, dec, m = _setup(batch=2)
+    s = d.block_len
+    rng = np.random.default_rng(depth)
+    base = wl.make_filter(s, d.tau, seed=depth)
+    layers = [(base["w1"], base["b1"])]
+    for k in range(1, depth):
+        layers.append(((rng.normal(size=(s, s)) * 0.3 + np.eye(s)).astype(np.float32), (0.1 * rng.normal(size=s)).astype(np.float32)))
+    if depth > 1:
+        layers[-1] = (base["w2"], base["b2"])
+    ofilt = {"layers": layers}
+    prompts = wl.make_prompts(2, d.prompt_len, shape, seed=7)
+    cfg = orc.DecodeConfig(block_len=s, tau=d.tau)
+    dec.set_filter_layers(layers)
+    st = lockstep(dec, m, ofilt, cfg, prompts, d.gen_len, logit_rtol=1e-4, conf_atol=1e-3, p_margin=1e-3,
+                  conf_margin=1e-5, replay_margin=1e-4)
+    assert st["replay_checked"] >= 0.8 * sum(st["seq_steps"])
+    if depth == 2:       # the list form of the init-time filter decodes exactly like it
+        toks, _, steps, _ = dec.decode(prompts, d.gen_len)
+        dec.set_filter_layers([])
+        dec2 = _b().Decoder(shape, w, base, block_len=s, tau=d.tau, max_batch=2, max_seq=d.prompt_len + d.gen_len)
+        toks2, _, steps2, _ = dec2.decode(prompts, d.gen_len)
+        assert np.array_equal(toks, toks2) and np.array_equal(steps, steps2)
+        dec2.close()
+    dec.close()
