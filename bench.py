@@ -34,8 +34,8 @@ SHAPE = wl.LLADA_8B
 DEC = wl.DECODES[WORKLOAD]
 METRIC, UNIT = "generated_tokens_per_s", "tokens/s"
 # DRAM bytes (read + write) of one gate/up launch at T = 512: dram__bytes_read.sum + dram__bytes_write.sum of
-# the ncu capture summarised in profiles/gemm_pair_T512_layer_shapes.md (208.2 MB + 3.6 MB)
-GATE_UP_DRAM_BYTES_PER_LAUNCH = 211.8e6
+# the ncu capture summarised in profiles/gemm_pair_T512_layer_shapes.md (209.0 MB + 4.2 MB)
+GATE_UP_DRAM_BYTES_PER_LAUNCH = 213.2e6
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -380,6 +380,28 @@ def run_ours(args):
                            "achieved_gbs": (wk["weight_bytes"] + wk["act_bytes"] + kv_bytes) / (t_in * 1e-3) / 1e9,
                            "rows_per_s": rows / (t_in * 1e-3)}
             decx.close()
+
+        # long generation (the setting of Section 4.3's EoTP study: generation length 1024, block 32): one sequence, the
+        # EoT logit biased so that the answer ends early; the same decode with and without EoTP
+        Pl, Gl, bias_l = 1024, 1024, 14.0
+        pl_ = torch.from_numpy(wl.make_prompts(1, Pl, SHAPE, seed=7)).to(dev)
+        out_l = torch.empty(1, Gl, dtype=torch.int32, device=dev)
+        rec = {"prompt_len": Pl, "gen_len": Gl, "eot_bias": bias_l}
+        for tag, eotp in (("eotp", True), ("no_eotp", False)):
+            decl = binding.Decoder(SHAPE, w, filt, block_len=s, tau=DEC.tau, max_batch=1, max_seq=Pl + Gl, device=local,
+                                   use_eotp=eotp, lm_head_bias=wl.make_eot_bias(SHAPE, bias_l))
+            decl.state_reset_device(pl_, Gl)
+            decl.denoise_step_host()                       # warm-up at this shape
+            ev0.record()
+            ol, st_l, tot_l = decl.decode_device(pl_, Gl, out_l)
+            ev1.record()
+            torch.cuda.synchronize()
+            first_eot = (out_l[0] == SHAPE.eot_id).nonzero()
+            rec[tag] = {"ms": ev0.elapsed_time(ev1), "steps": int(tot_l), "out_len": int(ol[0]),
+                        "first_eot": int(first_eot[0]) if len(first_eot) else -1}
+            decl.close()
+        rec["speedup_from_eotp"] = rec["no_eotp"]["ms"] / rec["eotp"]["ms"]
+        extra["long_generation"] = rec
 
         # filter training at the paper's scale (Section 4.1: 2,640 prompts, 5,000 epochs, lr 0.001): synthetic samples,
         # one per decoding step of a 32-step-per-prompt EGP run; the whole of stage 2 on the device

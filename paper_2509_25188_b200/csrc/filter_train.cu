@@ -7,7 +7,7 @@
 //                        dh = dz W2, dpre = dh [pre > 0], and adds dz^T h, dpre^T c and the bias sums into
 //                        accumulators its threads own; a block ends by writing its sums (not yet divided by
 //                        the batch's element count) and its loss sum to its own row of `gpart`;
-//   filter_adamw_kernel  one block adds the rows in block order (so a run is bit-reproducible), scales by
+//   filter_adamw_kernel  one thread per parameter adds the rows in block order (so a run is bit-reproducible), scales by
 //                        1 / (samples * s) and applies AdamW: decoupled weight decay, bias-corrected moments.
 // The whole problem (a few thousand parameters, samples of s floats) lives in shared memory and L2; the
 // arithmetic is fp32 on CUDA cores: K = s <= 64 is far too short a contraction for the tensor cores to matter.
@@ -142,14 +142,26 @@ struct AdamArgs {
   float *loss_out;                 // the batch's loss, measured before this update
 };
 
-__global__ void __launch_bounds__(1024) filter_adamw_kernel(AdamArgs a) {
+constexpr int ADAM_THREADS = 128;
+
+__global__ void __launch_bounds__(ADAM_THREADS) filter_adamw_kernel(AdamArgs a) {
   grid_dep_launch();
   grid_dep_wait();
-  for (int p = threadIdx.x; p <= a.P; p += blockDim.x) {
+  const int p = blockIdx.x * ADAM_THREADS + threadIdx.x;   // one parameter per thread; entry P is the loss
+  if (p <= a.P) {
+    // the rows are added in block order whatever the batching of the loads: eight loads in flight, then eight adds
     float g = 0.f;
-    for (int b = 0; b < a.n_blocks; ++b) g += a.gpart[(int64_t)b * (a.P + 1) + p];
+    int b = 0;
+    for (; b + 8 <= a.n_blocks; b += 8) {
+      float t[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t[i] = a.gpart[(int64_t)(b + i) * (a.P + 1) + p];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) g += t[i];
+    }
+    for (; b < a.n_blocks; ++b) g += a.gpart[(int64_t)b * (a.P + 1) + p];
     g *= a.inv_count;
-    if (p == a.P) { *a.loss_out = g; continue; }
+    if (p == a.P) { *a.loss_out = g; return; }
     const float th = a.theta[p] * (1.0f - a.lr * a.weight_decay);
     const float m = a.beta1 * a.m[p] + (1.0f - a.beta1) * g;
     const float v = a.beta2 * a.v[p] + (1.0f - a.beta2) * g * g;
@@ -182,7 +194,7 @@ cudaError_t launch_filter_update(cudaStream_t st, const float *C, const uint8_t 
   a.lr = h.lr; a.beta1 = h.beta1; a.beta2 = h.beta2; a.eps = h.eps; a.weight_decay = h.weight_decay;
   a.bc1 = (float)bc1; a.bc2 = (float)bc2;
   a.theta = theta; a.m = m; a.v = v; a.loss_out = loss_out;
-  return launch_kernel(filter_adamw_kernel, dim3(1), dim3(1024), 0, st, a);
+  return launch_kernel(filter_adamw_kernel, dim3((a.P + 1 + ADAM_THREADS - 1) / ADAM_THREADS), dim3(ADAM_THREADS), 0, st, a);
 }
 
 }  // namespace l2pd

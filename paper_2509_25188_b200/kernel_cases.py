@@ -9,6 +9,7 @@ Cases (LLaDA-8B layer shapes unless overridden with --d/--ff/--vocab/--heads):
   down     X[T,d]  += H[T,F] Wd^T                   residual epilogue
   lm_head  pred/conf over V for R = --rows rows     fused confidence head
   attn     bidirectional attention, --rows queries and keys, 32 heads x 128
+  train    filter training (Algorithm 1, stage 2): --rows samples of 32 confidences, --iters epochs per call
   step     whole denoising steps of a --layers deep model of these widths (batch 1, --rows / 2 prompt
            tokens + --rows / 2 masks, block 32): the small, self-ending case for profiling the
            memory-bound kernels (RMSNorm, RoPE/scatter, embedding, final norm, decision)
@@ -30,7 +31,7 @@ from . import binding as b
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", choices=["qkv", "o", "gate_up", "down", "lm_head", "attn", "step"])
+    ap.add_argument("case", choices=["qkv", "o", "gate_up", "down", "lm_head", "attn", "step", "train"])
     ap.add_argument("--rows", type=int, default=512)
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
@@ -72,6 +73,16 @@ def main():
             dec.denoise_step(outputs=False)
         per_layer = 2.0 * T * (4 * d * d + 3 * d * F) + 4.0 * T * T * d
         flops, byts = a.layers * per_layer + 2.0 * 32 * d * V, 2.0 * (a.layers * (4 * d * d + 3 * d * F) + V * d)
+    elif a.case == "train":
+        import numpy as np
+        from . import workloads as wl
+        rng = np.random.default_rng(0)
+        c_s = torch.from_numpy(rng.uniform(0.0, 1.0, size=(T, 32)).astype(np.float32)).to(dev)
+        y_s = (c_s + 0.15 * torch.randn_like(c_s) > 0.6).to(torch.uint8)
+        f0 = wl.make_filter(32, 0.96, seed=0)
+        epochs = 10
+        run = lambda i: b.filter_train(f0, c_s, y_s, epochs)
+        flops, byts = epochs * 10.0 * T * 32 * 32, epochs * 5.0 * T * 32
     elif a.case == "qkv":
         A, W = rnd(T, d, 1.0), ring(3 * d, d)
         Cc = torch.empty(T, 3 * d, dtype=torch.bfloat16, device=dev)
