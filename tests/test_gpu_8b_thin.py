@@ -141,3 +141,37 @@ def test_dual_cache_single_sequence_and_batch(thin8b):
                                            sample=lambda i, k, state: i == 0 and k in (0, 1))
     assert st["oracle_steps"] == 2
     assert st["replay_checked"] >= 0.9 * sum(st["seq_steps"])
+
+
+def test_comparison_policies_at_the_8b_widths(thin8b):
+    """Fixed confidence threshold and EGP (with a seeded synthetic reference: most steps take the
+    fallback and write reference ids) through the full-width kernels; every decision replayed, the
+    oracle's forward pass on sampled steps, and Algorithm 1's samples collected on the way."""
+    from paper_2509_25188_b200 import binding
+    w, dev = thin8b
+    s, B, P, G = 32, 2, 96, 64
+    bias = wl.make_eot_bias(SHAPE, 14.0)
+    m = oracle_model(SHAPE, w, lm_head_bias=bias)
+    filt = wl.make_filter(s, 0.96, seed=0)
+    prompts = wl.make_prompts(B, P, SHAPE, seed=41)
+    dec = binding.Decoder(SHAPE, dev, filt, block_len=s, max_batch=B, max_seq=P + G, lm_head_bias=bias)
+    sample = lambda i, k, state: i == 0 and k in (0, 3)
+    cfg = orc.DecodeConfig(block_len=s, rule="confidence", conf_threshold=0.6)
+    dec.set_unmask_rule("confidence", conf_threshold=0.6)
+    st = lockstep(dec, m, filt, cfg, prompts, G, logit_rtol=2e-2, conf_atol=0.1, p_margin=0.3, oracle_when=sample)
+    assert st["oracle_steps"] >= 1 and st["replay_checked"] >= 0.9 * sum(st["seq_steps"])
+    rng = np.random.default_rng(5)
+    refs = rng.integers(0, SHAPE.vocab - 2, size=(B, G))
+    cfg = orc.DecodeConfig(block_len=s, rule="egp")
+    dec.set_unmask_rule("egp", reference=refs)
+    sink_c, sink_y = dec.set_collect(B * G)
+    st = lockstep(dec, m, filt, cfg, prompts, G, logit_rtol=2e-2, conf_atol=0.1, p_margin=0.3, oracle_when=sample, refs=refs)
+    assert st["replay_checked"] == sum(st["seq_steps"])          # integer test: every step is replayed
+    n = dec.collect_count
+    assert n == sum(st["seq_steps"])
+    for i in range(B):
+        assert np.array_equal(st["states"][i].tokens[P:], refs[i])  # EGP ends in the reference
+    y = sink_y[:n].cpu().numpy()
+    c = sink_c[:n].cpu().numpy()
+    assert set(np.unique(y)) <= {0, 1} and (c >= 0).all() and (c <= 1.0 + 1e-6).all()
+    dec.close()
