@@ -277,7 +277,8 @@ l2pd_status l2pd_profile_read(const l2pd_ctx *ctx, int32_t kind, double *ms_tota
  * or a negative value if no step has run. */
 float l2pd_last_step_ms(const l2pd_ctx *ctx);
 
-const char *l2pd_last_error(const l2pd_ctx *ctx);   /* never NULL; "" when there is none */
+const char *l2pd_last_error(const l2pd_ctx *ctx);   /* never NULL; "" when there is none; ctx = NULL: what failed in
+                                                        the calling thread's last context-free call (GEMM, LM head, ...) */
 void l2pd_destroy(l2pd_ctx *ctx);                   /* NULL is allowed */
 
 /*

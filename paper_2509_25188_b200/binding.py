@@ -123,7 +123,7 @@ def _stream() -> int:
 
 def _check(status: int, ctx=None):
     if status != 0:
-        msg = lib.l2pd_last_error(ctx).decode() if ctx else ""
+        msg = lib.l2pd_last_error(ctx).decode()
         raise L2pdError(status, msg)
 
 

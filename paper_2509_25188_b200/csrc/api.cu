@@ -206,7 +206,7 @@ l2pd_status run_gemm_tc(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const Tm
   GemmArgs g{};
   if (epi == EPI_RESIDUAL && c->ksum && effective_k_splits(K, pl.k_splits) > 1) { g.part = c->ksum; g.part_rows = (int)round_up(M, 512); }
   g.epi = epi; g.a = a; g.b = b; g.b2 = b2; g.c = cm; g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.out = out;
-  g.cta_group = pl.cta_group; g.k_splits = pl.k_splits; g.slabs = pl.slabs;
+  g.cta_group = pl.cta_group; g.k_splits = pl.k_splits; g.slabs = pl.slabs; g.k_interleave = pl.k_interleave;
   g.status = c->d_status;
   if (epi == EPI_QKV_ROPE) {
     g.rope_cols = 2 * c->cfg.n_heads * c->cfg.head_dim; g.rope_dh = c->cfg.head_dim;
@@ -812,7 +812,7 @@ l2pd_status l2pd_profile_read(const l2pd_ctx *c, int32_t kind, double *ms_total,
   if (launches) *launches = c->prof_launches[kind];
   return L2PD_OK;
 }
-const char *l2pd_last_error(const l2pd_ctx *c) { return c ? c->err.c_str() : "null context"; }
+const char *l2pd_last_error(const l2pd_ctx *c);
 
 void l2pd_destroy(l2pd_ctx *c) {
   if (!c) return;
@@ -823,6 +823,13 @@ void l2pd_destroy(l2pd_ctx *c) {
 }
 
 // ---- stand-alone kernels --------------------------------------------------------------------------------
+
+// what failed in the calling thread's last stand-alone call (l2pd_last_error(NULL))
+static thread_local char g_standalone_err[160] = "";
+static l2pd_status standalone_cuda_error(const char *where, cudaError_t e) {
+  snprintf(g_standalone_err, sizeof(g_standalone_err), "%s: %s", where, cudaGetErrorString(e));
+  return L2PD_ERR_CUDA;
+}
 
 static int32_t *standalone_status() {
   static int32_t *p[64] = {};
@@ -845,8 +852,10 @@ static int device_sms() {
 static l2pd_status finish_standalone(cudaStream_t s, int32_t *status, int check) {
   if (!check) return L2PD_OK;
   int32_t h = 0;
-  if (cudaMemcpyAsync(&h, status, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2PD_ERR_CUDA;
-  if (cudaStreamSynchronize(s) != cudaSuccess) return L2PD_ERR_CUDA;
+  cudaError_t e = cudaMemcpyAsync(&h, status, 4, cudaMemcpyDeviceToHost, s);
+  if (e != cudaSuccess) return standalone_cuda_error("status read-back", e);
+  e = cudaStreamSynchronize(s);
+  if (e != cudaSuccess) return standalone_cuda_error("stream synchronisation", e);
   if (h != DEV_OK) { cudaMemsetAsync(status, 0, 4, s); return L2PD_ERR_TIMEOUT; }
   return L2PD_OK;
 }
@@ -857,7 +866,10 @@ static l2pd_status gemm_common(void *stream, int epi, const void *A, const void 
   if (M < 1 || N < 8 || K < 8 || (N % 8) || (K % 8)) return L2PD_ERR_SHAPE;
   if (tile_n < 0) return L2PD_ERR_SHAPE;
   const int sms = device_sms();
-  // tile_n = width + 1000 * cta_group + 10000 * k_splits + 100000 * slabs; any part 0 = chosen automatically
+  // tile_n = width + 1000 * cta_group + 10000 * k_splits + 100000 * slabs + 1000000 * k_interleave (1 = on, 2 = off);
+  // any part 0 = chosen automatically
+  const int want_kil = tile_n / 1000000;
+  tile_n %= 1000000;
   const int want_sl = tile_n / 100000, want_ks = (tile_n % 100000) / 10000, want_cg = (tile_n % 10000) / 1000,
             want_tn = tile_n % 1000;
   const int unit = 16;
@@ -868,6 +880,8 @@ static l2pd_status gemm_common(void *stream, int epi, const void *A, const void 
   if (want_cg) pl.cta_group = want_cg;
   if (want_ks) pl.k_splits = want_ks;
   if (want_sl) pl.slabs = want_sl;
+  if (want_kil == 1) pl.k_interleave = 1;
+  if (want_kil == 2 || pl.cta_group != 1 || pl.slabs != 1) pl.k_interleave = 0;
   if (pl.slabs == 2 && pl.cta_group != 2) return L2PD_ERR_SHAPE;
   if (pl.k_splits > ceil_div(K, 64)) pl.k_splits = ceil_div(K, 64);
   int32_t *status = standalone_status();
@@ -888,11 +902,13 @@ static l2pd_status gemm_common(void *stream, int epi, const void *A, const void 
   g.c = staged ? &tcm : nullptr;
   g.epi = epi; g.a = &ta; g.b = &tb; g.b2 = epi == EPI_SWIGLU ? &tb2 : nullptr;
   g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.cta_group = pl.cta_group; g.k_splits = pl.k_splits;
-  g.slabs = pl.slabs;
+  g.slabs = pl.slabs; g.k_interleave = pl.k_interleave;
   g.out = out; g.status = status;
-  if (launch_gemm_tcgen05((cudaStream_t)stream, g, sms) != cudaSuccess) return L2PD_ERR_CUDA;
+  { cudaError_t e = launch_gemm_tcgen05((cudaStream_t)stream, g, sms); if (e != cudaSuccess) return standalone_cuda_error("GEMM launch", e); }
   return finish_standalone((cudaStream_t)stream, status, check);
 }
+
+const char *l2pd_last_error(const l2pd_ctx *c) { return c ? c->err.c_str() : g_standalone_err; }
 
 l2pd_status l2pd_gemm_bf16(void *stream, const void *A, const void *W, void *C, int32_t M, int32_t N, int32_t K,
                            int32_t tile_n, int32_t check) {

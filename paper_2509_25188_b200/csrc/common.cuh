@@ -165,7 +165,9 @@ int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile);
 // tile, each slab with its own MMA-issuing thread; its accumulators fill tensor memory, so the
 // drain is not overlapped with the next unit).
 // The B tensor map's box must be tile_n / cta_group rows (SwiGLU: tile_n / 2 for either group size).
-struct GemmPlan { int cta_group, tile_n, k_splits, slabs; };
+// k_interleave = 1 (single CTA, one slab, few rows): the two MMA-issuing threads take alternate k-blocks of the
+// unit into two accumulators that the epilogue adds — halves the K loop where instruction issue bounds it
+struct GemmPlan { int cta_group, tile_n, k_splits, slabs, k_interleave; };
 GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, int max_k_splits = 4);
 int effective_k_splits(int K, int k_splits);   // what the launcher makes of a requested K split
 struct GemmArgs {
@@ -175,6 +177,7 @@ struct GemmArgs {
   int M, N, K, tile_n;
   int cta_group, k_splits; // 0 / 1 = single CTA, no split
   int slabs;               // 0 / 1 = one row slab per unit, 2 = two
+  int k_interleave;        // see GemmPlan
   void *out;               // bf16 C, fp32 X, or bf16 H
   // LM head
   const float *bias; float *part_m, *part_s; int32_t *part_i; int rows_padded; float *logits;

@@ -62,6 +62,7 @@ struct KParams {
   int rope_cols, rope_dh, cs_stride;   // EPI_QKV_ROPE, see GemmArgs
   const float2 *cs_table;
   const int32_t *row_pos;
+  int kil;   // 1: the unit's k-blocks alternate between the two MMA issuers (accumulators 0 and 1, added in the epilogue)
 };
 
 __device__ __forceinline__ void fail(int32_t *status, int code) {
@@ -154,7 +155,9 @@ __device__ __forceinline__ void rope_pairs(const KParams &p, uint32_t *v, int co
 // K slices of the residual epilogue either add into X (`res_mode` 1) or store their partial sums to
 // `res_base`, the slice's own [rows][N] area (`res_mode` 2), for a later fixed-order sum.
 template <int EPI>
-__device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int row, int nt, int res_mode, float *res_base) {
+// two_acc: the unit's sum is spread over two accumulators (ACC_COLS columns apart), added here.
+__device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int row, int nt, int res_mode, float *res_base,
+                                           bool two_acc = false) {
   const bool row_ok = row < p.M;
   const int half_n = p.tile_n >> 1;
   if (EPI == EPI_STORE || EPI == EPI_RESIDUAL || EPI == EPI_QKV_ROPE) {
@@ -178,6 +181,18 @@ __device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int
         }
       }
     };
+    if (two_acc) {
+      for (int c = 0; c < n; c += 32) {
+        load(va, c);
+        if (n - c >= 32) ptx::tmem_ld_x32(taddr + ACC_COLS + c, vb);
+        else ptx::tmem_ld_x16(taddr + ACC_COLS + c, vb);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) va[i] = __float_as_uint(__uint_as_float(va[i]) + __uint_as_float(vb[i]));
+        emit(va, c);
+      }
+      return;
+    }
     load(va, 0);
     for (int c = 0; c < n; c += 64) {
       ptx::tmem_ld_wait();
@@ -199,6 +214,21 @@ __device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int
     auto emit = [&](const uint32_t *g, const uint32_t *u, int c) {
       if (row_ok && n0 + c < p.N) emit_swiglu16(H + (int64_t)row * p.N + n0 + c, g, u, min(p.N - n0 - c, half_n - c));
     };
+    if (two_acc) {
+      for (int c = 0; c < half_n; c += 16) {
+        load(ga, ua, c);
+        ptx::tmem_ld_x16(taddr + ACC_COLS + c, gb);
+        ptx::tmem_ld_x16(taddr + ACC_COLS + half_n + c, ub);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          ga[i] = __float_as_uint(__uint_as_float(ga[i]) + __uint_as_float(gb[i]));
+          ua[i] = __float_as_uint(__uint_as_float(ua[i]) + __uint_as_float(ub[i]));
+        }
+        emit(ga, ua, c);
+      }
+      return;
+    }
     load(ga, ua, 0);
     for (int c = 0; c < half_n; c += 32) {
       ptx::tmem_ld_wait();
@@ -395,7 +425,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
   const uint32_t sB = base + p.n_stages * p.a_stage_bytes;
   const uint32_t sOut = sA + (uint32_t)(p.n_stages - 2) * p.a_stage_bytes;   // output staging: see drain_tile_staged
   const int slabs = p.slabs;
-  const int nbuf = slabs == 1 ? 2 : 1;            // accumulator buffers a unit can alternate between
+  const int nbuf = (slabs == 1 && !p.kil) ? 2 : 1;   // accumulator buffers a unit can alternate between
   const int unit_rows = TILE_M * CG * slabs;
   const uint32_t bar0 = ptx::smem_u32(bars);
   auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -406,7 +436,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.n_stages; ++s) { ptx::mbar_init(full_bar(s), 1); ptx::mbar_init(empty_bar(s), slabs); }
-    for (int b = 0; b < 2; ++b) { ptx::mbar_init(tfull_bar(b), slabs); ptx::mbar_init(tempty_bar(b), 4 * CG * slabs); }
+    for (int b = 0; b < 2; ++b) { ptx::mbar_init(tfull_bar(b), p.kil ? 2 : slabs); ptx::mbar_init(tempty_bar(b), 4 * CG * slabs); }
     ptx::mbar_init(sfree_bar, 4 * slabs);
     *abort_flag = 0;
     ptx::fence_barrier_init();
@@ -530,7 +560,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
     // warp 1 feeds slab 0, warp 2 slab 1: each slab has its own accumulator columns, so the two
     // instruction streams need no ordering between them; both count on the stage's `empty` barrier.
     const int sl = warp - 1;
-    if (lane == 0 && leader && sl < slabs) {
+    if (lane == 0 && leader && (sl < slabs || p.kil)) {
       const uint32_t idesc = ptx::idesc_bf16(TILE_M * CG, (uint32_t)p.tile_n);
       uint32_t phases = 0;
       int lt = 0;
@@ -545,13 +575,20 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
         const uint32_t d_tmem = tmem_base + (ab + sl) * ACC_COLS;   // slab sl of a two-slab unit: column sl * ACC_COLS
         int stage = 0;
         for (int kb = kb0; kb < kb1; ++kb) {
+          // Alternating issuers: the ring has an even number of stages and every unit starts at stage 0, so the
+          // stages of even k-blocks are the even ones.  Each stage's barriers thus have one consumer, which sees all of
+          // their phases in order (a thread that skipped phases could not tell a parity from the one two phases on).
+          if (p.kil && ((kb - kb0) & 1) != sl) {
+            if (++stage == p.n_stages) stage = 0;
+            continue;
+          }
           if (!ptx::mbar_wait(full_bar(stage), (phases >> stage) & 1u)) { fail(p.status, DEV_TIMEOUT_MMA); ok = false; break; }
           ptx::tc_fence_after_sync();
-          const uint64_t a_desc = ptx::smem_desc_sw128(sA + stage * p.a_stage_bytes + sl * A_STAGE_BYTES);
+          const uint64_t a_desc = ptx::smem_desc_sw128(sA + stage * p.a_stage_bytes + (p.kil ? 0 : sl * A_STAGE_BYTES));
           const uint64_t b_desc = ptx::smem_desc_sw128(sB + stage * p.b_stage_bytes);
 #pragma unroll
           for (int k = 0; k < TILE_K / 16; ++k) {   // 16 bf16 = 32 bytes per MMA: descriptor address += 2
-            const uint32_t acc = (kb > kb0 || k > 0) ? 1u : 0u;
+            const uint32_t acc = (kb > kb0 + (p.kil ? sl : 0) || k > 0) ? 1u : 0u;
             if (CG == 2) ptx::mma_bf16_ss_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, acc);
             else ptx::mma_bf16_ss(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, acc);
           }
@@ -628,7 +665,8 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
                                res_store);
       else
         drain_tile<EPI>(p, taddr, row0 + lane, nt, res_store ? 2 : (p.k_splits > 1 ? 1 : 0),
-                        res_store ? p.part + (int64_t)slice_row0 * p.N : reinterpret_cast<float *>(p.out));
+                        res_store ? p.part + (int64_t)slice_row0 * p.N : reinterpret_cast<float *>(p.out),
+                        p.kil && kb1 - kb0 >= 2);
       ptx::tc_fence_before_sync();
       __syncwarp();
       if (lane == 0) {
@@ -774,7 +812,7 @@ l2pd_status make_tma_out_3d(TmaDesc *out, void *ptr, bool fp32, int64_t rows, in
 // takes to issue its four MMAs and the stage hand-over; the bytes it must take in at INGEST bytes
 // per cycle.  A unit adds a fixed fill part and, when its accumulators are not double-buffered
 // (two slabs), the drain of the accumulator; times the number of waves over the SMs (or SM pairs).
-static double plan_cost(int M, int N, int K, int num_sms, int cg, int slabs, int unit_n, int tile_n, int ks, bool is_residual) {
+static double plan_cost(int M, int N, int K, int num_sms, int cg, int slabs, int unit_n, int tile_n, int ks, bool is_residual, bool kil) {
   const double INGEST = cg == 2 ? 58.0 : 68.0;   // measured: bytes per cycle an SM takes in from L2 through TMA
   const int groups = num_sms / cg;
   const int m_tiles = ceil_div(M, TILE_M * cg * slabs);
@@ -783,7 +821,7 @@ static double plan_cost(int M, int N, int K, int num_sms, int cg, int slabs, int
   const int waves = ceil_div(units, groups);
   const int kb = ceil_div(ceil_div(K, TILE_K), ks);
   const double bytes = (double)slabs * A_STAGE_BYTES + 128.0 * tile_n / cg;
-  const double per_kb = fmax(fmax(2.0 * tile_n * slabs, 620.0), bytes / INGEST) * 1.06;
+  const double per_kb = fmax(fmax(2.0 * tile_n * slabs, kil ? 330.0 : 620.0), bytes / INGEST) * 1.06;
   // emptying the accumulators: bf16 stores leave an SM at ~34 B per cycle; fp32 additions into X are bound
   // by L2's atomic units, ~2500 B per cycle for the whole chip, i.e. ~17 B per cycle and SM when all drain at once
   // (K slices store their partial sums plainly: twice the rate of the additions)
@@ -793,7 +831,7 @@ static double plan_cost(int M, int N, int K, int num_sms, int cg, int slabs, int
 }
 
 GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, int max_k_splits) {
-  GemmPlan best{1, 256, 1, 1};
+  GemmPlan best{1, 256, 1, 1, 0};
   double best_cost = 1e300;
   const bool swiglu = epi == EPI_SWIGLU;
   const int step = 16;   // SwiGLU: the gate and up halves are then multiples of 8 (one swizzle group of rows)
@@ -808,8 +846,10 @@ GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, 
         const int max_ks = (epi == EPI_RESIDUAL) ? (max_k_splits < 4 ? max_k_splits : 4) : 1;
         for (int ks = 1; ks <= max_ks; ++ks) {
           if (ceil_div(K, TILE_K) < 8 * ks) break;
-          const double c = plan_cost(M, N, K, num_sms, cg, slabs, unit_n, tn, ks, epi == EPI_RESIDUAL);
-          if (c < best_cost - 1e-9) { best_cost = c; best = GemmPlan{cg, tn, ks, slabs}; }
+          // few rows: one 128-row MMA per 132 cycles and issuer bounds the K loop; the idle second issuer takes every other k-block
+          const bool kil = M <= TILE_M && cg == 1 && slabs == 1 && epi != EPI_LMHEAD && epi != EPI_QKV_ROPE;
+          const double c = plan_cost(M, N, K, num_sms, cg, slabs, unit_n, tn, ks, epi == EPI_RESIDUAL, kil);
+          if (c < best_cost - 1e-9) { best_cost = c; best = GemmPlan{cg, tn, ks, slabs, kil ? 1 : 0}; }
         }
       }
     }
@@ -844,12 +884,15 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
   const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
   int stages = (SMEM_BUDGET - 2048) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
+  if (g.k_interleave) stages &= ~1;   // alternate k-blocks <-> alternate stages
   if (stages < 2) return cudaErrorInvalidValue;
   p.n_stages = stages;
   p.m_tiles = ceil_div(g.M, TILE_M * cg * p.slabs);
   const int n_per_tile = (g.epi == EPI_SWIGLU) ? g.tile_n / 2 : g.tile_n;
   // staged output: needs the output map and a staging area (the A part of the ring's last two stages)
-  p.out_tma = (g.c != nullptr && g.epi != EPI_LMHEAD && stages >= 3) ? 1 : 0;
+  p.kil = g.k_interleave ? 1 : 0;
+  if (p.kil && (cg != 1 || p.slabs != 1 || g.epi == EPI_LMHEAD || g.epi == EPI_QKV_ROPE)) return cudaErrorInvalidValue;
+  p.out_tma = (g.c != nullptr && g.epi != EPI_LMHEAD && stages >= 3 && !p.kil) ? 1 : 0;   // (the two-accumulator sum lives in the direct-store drain)
   p.out_full_tiles = p.out_tma ? g.N / n_per_tile : 0;
   p.gate = (p.out_tma && p.slabs == 2 && stages >= 4) ? 1 : 0;
   p.n_tiles = ceil_div(g.N, n_per_tile);

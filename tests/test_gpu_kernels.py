@@ -53,6 +53,11 @@ GEMM_SHAPES = [
     (300, 528, 1032, 202176),  # two slabs: the second one mostly empty, N and K tails
     (1100, 2048, 256, 202128), # two slabs: several units per pair, ragged last row tile
     (512, 12288, 320, 202256), # two slabs, full-width accumulators (all 512 tensor-memory columns)
+    (32, 1024, 4096, 1000096),  # few rows: the two MMA issuers take alternate k-blocks (two accumulators added in the epilogue)
+    (100, 528, 1032, 1001176),  # the same with an odd number of k-blocks, N and K tails
+    (128, 512, 320, 1000256),   # the same with both accumulators 256 columns wide
+    (32, 1024, 4096, 2000096),  # alternation switched off: one issuer
+    (32, 12288, 4096, 0),       # the QKV projection of a 32-row step, automatic plan
 ]
 
 
@@ -73,6 +78,10 @@ RESIDUAL_SHAPES = GEMM_SHAPES[:5] + [
     (512, 4096, 1024, 2240),    # pair, width 240
     (512, 4096, 4096, 232176),  # two slabs + three K slices
     (400, 1024, 12288, 222176), # two slabs + two K slices, ragged rows
+    (32, 4096, 4096, 1041112),  # few rows: four K slices, alternate k-blocks inside each
+    (64, 528, 4104, 1031064),   # three slices, the last one shorter, K tail
+    (100, 512, 192, 1031064),   # slices of a single k-block: the second issuer has nothing to add
+    (32, 4096, 12288, 0),       # the down projection of a 32-row step, automatic plan
 ]
 
 
@@ -94,7 +103,8 @@ def test_gemm_bf16_residual(M, N, K, tile_n):
                                           (200, 336, 192, 2064), (1000, 2048, 256, 2256),
                                           (512, 1408, 512, 202160), (300, 2048, 256, 202256),
                                           (512, 1408, 512, 202176), (200, 336, 192, 1176), (130, 1408, 128, 2144),
-                                          (512, 24576, 256, 0)])
+                                          (512, 24576, 256, 0), (32, 1408, 4096, 1000176), (90, 336, 192, 1000064),
+                                          (32, 12288, 4096, 0)])
 def test_gemm_bf16_swiglu(M, F, K, tile_n):
     b = _b()
     A = _bf16(3, 0, (M, K), 1.0)
