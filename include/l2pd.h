@@ -290,11 +290,13 @@ void l2pd_destroy(l2pd_ctx *ctx);                   /* NULL is allowed */
  */
 
 /* C[M,N] (bf16) = A[M,K] (bf16, row-major) x W[N,K]^T (bf16, row-major); tcgen05 path.
- * K and N multiples of 8.  tile_n = width + 1000 * cta_group + 10000 * k_splits + 100000 * slabs,
- * every part optional (0 = chosen automatically): width a multiple of 16 in [32, 256]; cta_group 1,
- * or 2 for a pair of SMs on one 256-row tile; k_splits (residual epilogue only) slices K, the
- * slices adding into X with floating-point reductions whose order is not fixed; slabs 2 (pairs
- * only) lets one unit cover two 256-row slabs against one load of the weight tile.
+ * K and N multiples of 8.  tile_n = width + 1000 * cta_group + 10000 * k_splits + 100000 * slabs
+ * + 1000000 * k_interleave, every part optional (0 = chosen automatically): width a multiple of 16 in
+ * [32, 256]; cta_group 1, or 2 for a pair of SMs on one 256-row tile; k_splits (residual epilogue only)
+ * slices K, the slices adding into X with floating-point reductions whose order is not fixed; slabs 2
+ * (pairs only) lets one unit cover two 256-row slabs against one load of the weight tile; k_interleave
+ * 1 (one slab only) has two threads issue the MMAs of alternate k-blocks into two accumulators that the
+ * epilogue adds (chosen automatically when the rows fit one slab), 2 switches it off.
  * A and the output follow stream order.  The weights W are requested before the kernel launched
  * just ahead of this one in the stream has completed (programmatic dependent launch): that kernel
  * must not be the one that writes them. */

@@ -881,7 +881,7 @@ static l2pd_status gemm_common(void *stream, int epi, const void *A, const void 
   if (want_ks) pl.k_splits = want_ks;
   if (want_sl) pl.slabs = want_sl;
   if (want_kil == 1) pl.k_interleave = 1;
-  if (want_kil == 2 || pl.cta_group != 1 || pl.slabs != 1) pl.k_interleave = 0;
+  if (want_kil == 2 || pl.slabs != 1) pl.k_interleave = 0;
   if (pl.slabs == 2 && pl.cta_group != 2) return L2PD_ERR_SHAPE;
   if (pl.k_splits > ceil_div(K, 64)) pl.k_splits = ceil_div(K, 64);
   int32_t *status = standalone_status();

@@ -847,7 +847,7 @@ GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, 
         for (int ks = 1; ks <= max_ks; ++ks) {
           if (ceil_div(K, TILE_K) < 8 * ks) break;
           // few rows: one 128-row MMA per 132 cycles and issuer bounds the K loop; the idle second issuer takes every other k-block
-          const bool kil = M <= TILE_M && cg == 1 && slabs == 1 && epi != EPI_LMHEAD && epi != EPI_QKV_ROPE;
+          const bool kil = M <= TILE_M * cg && slabs == 1 && epi != EPI_LMHEAD;
           const double c = plan_cost(M, N, K, num_sms, cg, slabs, unit_n, tn, ks, epi == EPI_RESIDUAL, kil);
           if (c < best_cost - 1e-9) { best_cost = c; best = GemmPlan{cg, tn, ks, slabs, kil ? 1 : 0}; }
         }
@@ -891,7 +891,7 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
   const int n_per_tile = (g.epi == EPI_SWIGLU) ? g.tile_n / 2 : g.tile_n;
   // staged output: needs the output map and a staging area (the A part of the ring's last two stages)
   p.kil = g.k_interleave ? 1 : 0;
-  if (p.kil && (cg != 1 || p.slabs != 1 || g.epi == EPI_LMHEAD || g.epi == EPI_QKV_ROPE)) return cudaErrorInvalidValue;
+  if (p.kil && (p.slabs != 1 || g.epi == EPI_LMHEAD)) return cudaErrorInvalidValue;
   p.out_tma = (g.c != nullptr && g.epi != EPI_LMHEAD && stages >= 3 && !p.kil) ? 1 : 0;   // (the two-accumulator sum lives in the direct-store drain)
   p.out_full_tiles = p.out_tma ? g.N / n_per_tile : 0;
   p.gate = (p.out_tma && p.slabs == 2 && stages >= 4) ? 1 : 0;

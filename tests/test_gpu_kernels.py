@@ -58,6 +58,8 @@ GEMM_SHAPES = [
     (128, 512, 320, 1000256),   # the same with both accumulators 256 columns wide
     (32, 1024, 4096, 2000096),  # alternation switched off: one issuer
     (32, 12288, 4096, 0),       # the QKV projection of a 32-row step, automatic plan
+    (256, 2048, 1032, 1002240), # alternate k-blocks on a pair of SMs (one 256-row slab), K tail
+    (200, 12288, 4096, 0),      # QKV at 200 rows, automatic plan
 ]
 
 
@@ -82,6 +84,8 @@ RESIDUAL_SHAPES = GEMM_SHAPES[:5] + [
     (64, 528, 4104, 1031064),   # three slices, the last one shorter, K tail
     (100, 512, 192, 1031064),   # slices of a single k-block: the second issuer has nothing to add
     (32, 4096, 12288, 0),       # the down projection of a 32-row step, automatic plan
+    (256, 4096, 12288, 1042240), # pair, four K slices, alternate k-blocks
+    (256, 4096, 12288, 0),
 ]
 
 
@@ -104,7 +108,7 @@ def test_gemm_bf16_residual(M, N, K, tile_n):
                                           (512, 1408, 512, 202160), (300, 2048, 256, 202256),
                                           (512, 1408, 512, 202176), (200, 336, 192, 1176), (130, 1408, 128, 2144),
                                           (512, 24576, 256, 0), (32, 1408, 4096, 1000176), (90, 336, 192, 1000064),
-                                          (32, 12288, 4096, 0)])
+                                          (32, 12288, 4096, 0), (256, 1408, 4096, 1002176), (256, 12288, 4096, 0)])
 def test_gemm_bf16_swiglu(M, F, K, tile_n):
     b = _b()
     A = _bf16(3, 0, (M, K), 1.0)
