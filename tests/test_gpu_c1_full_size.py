@@ -144,26 +144,29 @@ def test_c1_confidence_head_and_decision_match_oracle(c1, name):
         assert np.array_equal(out["unmask"][0].astype(bool)[clear], g[name + "_unmask"][clear])
 
 
-@pytest.mark.parametrize("name", ["C2", "C3", "C4"])
+@pytest.mark.parametrize("name", ["C2", "C3", "C4", "C2-dual", "C4-dual"])
 def test_full_depth_decodes_replay_every_decision(c1, name):
     """The decode configurations at full depth (32 layers): single sequence with an EoT bias, batch 16
-    (prompt 512 + generation 512) and batch 8 with the prefix cache (1024 + 1024).  The oracle's forward
+    (prompt 512 + generation 512) and batch 8 with the prefix cache (1024 + 1024); "-dual": the same
+    shapes with the dual cache (in-block steps of 32 rows per sequence).  The oracle's forward
     pass is out of reach here (minutes per step and sequence); what is checked on every step of every
     sequence is the decision logic — filter, threshold, fallback, commit, EoTP, block advance — replayed
     in fp64 on the decoder's own confidences, bit for bit, and the decode invariants at the end."""
     from paper_2509_25188_b200 import binding
     from tests.helpers import lockstep
     shape, _, dev, _, _ = c1
-    dsh = wl.DECODES[name]
+    dual = name.endswith("-dual")
+    dsh = wl.DECODES[name.split("-")[0]]
     B, P, G, s = dsh.batch, dsh.prompt_len, dsh.gen_len, dsh.block_len
+    kv_mode = 2 if dual else int(dsh.kv_cache)
     bias = wl.make_eot_bias(shape, 14.0)
     w = dict(dev, final_norm=np.full(shape.d_model, wl.spread_gain(shape), np.float32))
     filt = wl.make_filter(s, dsh.tau, seed=0)
     m = oracle_model(shape, {"layers": [], "final_norm": None, "tok_emb": None, "lm_head": None}, lm_head_bias=bias)
-    cfg = orc.DecodeConfig(block_len=s, tau=dsh.tau, kv_cache=dsh.kv_cache)
+    cfg = orc.DecodeConfig(block_len=s, tau=dsh.tau, kv_cache=kv_mode > 0, dual_cache=dual)
     prompts = wl.make_prompts(B, P, shape, seed=41)
     dec = binding.Decoder(shape, w, filt, block_len=s, tau=dsh.tau, max_batch=B, max_seq=P + G,
-                          kv_cache=dsh.kv_cache, lm_head_bias=bias)
+                          kv_cache=kv_mode, lm_head_bias=bias)
     st = lockstep(dec, m, filt, cfg, prompts, G, logit_rtol=2e-2, conf_atol=0.1, p_margin=0.3,
                   oracle_when=lambda i, k, state: False)
     dec.close()
