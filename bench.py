@@ -403,6 +403,32 @@ def run_ours(args):
         rec["speedup_from_eotp"] = rec["no_eotp"]["ms"] / rec["eotp"]["ms"]
         extra["long_generation"] = rec
 
+        # threshold sweep (Section 4.4 studies tau = 0.9 ... 0.99) and the comparison policies on the C2 decode: steps and
+        # generated tokens per second of one sequence with the same synthetic model, filter and EoT bias
+        sweep = {}
+        d_out2 = torch.empty(B, G, dtype=torch.int32, device=dev)
+        for tag, kw, rule in [("tau_0.90", {"tau": 0.90}, None), ("tau_0.96", {"tau": 0.96}, None), ("tau_0.99", {"tau": 0.99}, None),
+                              ("confidence_0.9", {"tau": DEC.tau}, ("confidence", 0.9)),
+                              ("one_token_per_step", {"tau": DEC.tau}, ("confidence", 1.0))]:
+            decs = binding.Decoder(SHAPE, w, filt, block_len=s, max_batch=B, max_seq=P + G, device=local,
+                                   lm_head_bias=wl.make_eot_bias(SHAPE, 14.0), **kw)
+            if rule:
+                decs.set_unmask_rule(rule[0], conf_threshold=rule[1])
+            decs.state_reset_device(d_prompts, G)
+            decs.denoise_step_host()
+            ev0.record()
+            ol, st_s, tot_s = decs.decode_device(d_prompts, G, d_out2)
+            ev1.record()
+            torch.cuda.synchronize()
+            ms_s = ev0.elapsed_time(ev1)
+            sweep[tag] = {"steps": int(tot_s), "out_len": int(ol[0]), "ms": ms_s,
+                          "generated_tokens_per_s": float(np.sum(ol)) / (ms_s * 1e-3)}
+            decs.close()
+        base_steps = sweep["one_token_per_step"]["steps"]
+        for v in sweep.values():
+            v["steps_vs_one_token_per_step"] = base_steps / max(v["steps"], 1)
+        extra["policy_sweep_C2"] = sweep
+
         # filter training at the paper's scale (Section 4.1: 2,640 prompts, 5,000 epochs, lr 0.001): synthetic samples,
         # one per decoding step of a 32-step-per-prompt EGP run; the whole of stage 2 on the device
         n_samp = 2640 * 32
