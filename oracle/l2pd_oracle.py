@@ -520,6 +520,55 @@ def bce_with_logits(z: np.ndarray, y: np.ndarray) -> float:
     return float(np.mean(np.maximum(z, 0.0) - z * y + np.log1p(np.exp(-np.abs(z)))))
 
 
+def filter_layers_loss_and_grads(layers, C: np.ndarray, Y: np.ndarray):
+    """The same for the depth variants of Section 4.4: layers = [(W, b), ...], ReLU between consecutive
+    layers.  Returns (loss, [(dW, db), ...])."""
+    acts = [C]                                   # input of layer k
+    pres = []
+    x = C
+    for k, (w, b) in enumerate(layers):
+        if k > 0:
+            x = np.maximum(x, 0.0)
+            acts.append(x)
+        x = x @ widen(w).T + widen(b)
+        pres.append(x)
+    z = x
+    loss = bce_with_logits(z, Y)
+    delta = (sigmoid(z) - Y) / z.size            # d loss / d (output of the last layer)
+    grads = [None] * len(layers)
+    for k in range(len(layers) - 1, -1, -1):
+        grads[k] = (delta.T @ acts[k], delta.sum(axis=0))
+        if k > 0:
+            delta = (delta @ widen(layers[k][0])) * (pres[k - 1] > 0.0)
+    return loss, grads
+
+
+def train_filter_layers(layers0, C: np.ndarray, Y: np.ndarray, epochs: int, lr: float = 1e-3, beta1: float = 0.9,
+                        beta2: float = 0.999, eps: float = 1e-8, weight_decay: float = 0.01, batch_size: int = 0):
+    """train_filter for a filter given as a list of (W, b) layers; returns (layers, losses)."""
+    layers = [(widen(w).copy(), widen(b).copy()) for (w, b) in layers0]
+    mom = [(np.zeros_like(w), np.zeros_like(b)) for (w, b) in layers]
+    var = [(np.zeros_like(w), np.zeros_like(b)) for (w, b) in layers]
+    N = len(C)
+    bs = N if batch_size <= 0 else batch_size
+    losses = []
+    t = 0
+    for _ in range(epochs):
+        for lo in range(0, N, bs):
+            loss, g = filter_layers_loss_and_grads(layers, C[lo: lo + bs], Y[lo: lo + bs])
+            losses.append(loss)
+            t += 1
+            for k in range(len(layers)):
+                new = []
+                for q in range(2):
+                    p, m, v = adamw_step(layers[k][q], g[k][q], mom[k][q], var[k][q], t, lr, beta1, beta2, eps, weight_decay)
+                    new.append((p, m, v))
+                layers[k] = (new[0][0], new[1][0])
+                mom[k] = (new[0][1], new[1][1])
+                var[k] = (new[0][2], new[1][2])
+    return layers, np.asarray(losses)
+
+
 def filter_loss_and_grads(filt: Dict[str, np.ndarray], C: np.ndarray, Y: np.ndarray):
     """Loss of Eq. 6 over the batch (C[n, s], Y[n, s]) and its gradient w.r.t. w1, b1, w2, b2."""
     w1, b1, w2, b2 = (widen(filt[k]) for k in ("w1", "b1", "w2", "b2"))

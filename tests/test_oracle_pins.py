@@ -861,3 +861,42 @@ def test_filter_depth_variants():
     assert np.allclose(orc.filter_logits({"layers": ws}, c), want, atol=1e-12)
     # parameter counts of the three depths at s = 32: 1,056 / 2,112 (the printed count) / 4,224
     assert [k * (32 * 32 + 32) for k in (1, 2, 4)] == [1056, int(paper_constants()["filter_params_at_block_32"]), 4224]
+
+
+@pytest.mark.parametrize("depth", [1, 2, 4])
+def test_depth_variant_training_matches_torch_and_the_two_layer_form(depth):
+    """Backpropagation through 1, 2 and 4 layers against torch autograd + optim.AdamW in fp64; at depth 2 the
+    list form also reproduces train_filter."""
+    s = 6
+    C, Y = _train_data(s, 30, seed=11)
+    rng = np.random.default_rng(depth)
+    layers0 = [((rng.normal(size=(s, s)) * 0.5).astype(np.float32), (0.1 * rng.normal(size=s)).astype(np.float32))
+               for _ in range(depth)]
+    epochs = 20
+    got, losses = orc.train_filter_layers(layers0, C, Y, epochs, lr=1e-2, weight_decay=0.02, batch_size=16)
+    mods = []
+    lins = []
+    for k, (w, b) in enumerate(layers0):
+        lin = torch.nn.Linear(s, s).double()
+        with torch.no_grad():
+            lin.weight.copy_(torch.from_numpy(w.astype(np.float64))); lin.bias.copy_(torch.from_numpy(b.astype(np.float64)))
+        lins.append(lin)
+        mods += ([torch.nn.ReLU()] if k else []) + [lin]
+    net = torch.nn.Sequential(*mods)
+    opt = torch.optim.AdamW(net.parameters(), lr=1e-2, betas=(0.9, 0.999), eps=1e-8, weight_decay=0.02)
+    tc, ty = torch.from_numpy(C), torch.from_numpy(Y)
+    ref_losses = []
+    for _ in range(epochs):
+        for lo in range(0, len(C), 16):
+            opt.zero_grad()
+            loss = torch.nn.functional.binary_cross_entropy_with_logits(net(tc[lo: lo + 16]), ty[lo: lo + 16])
+            loss.backward()
+            opt.step()
+            ref_losses.append(float(loss.detach()))
+    assert np.allclose(losses, ref_losses, rtol=0, atol=1e-10)
+    for (w, b), lin in zip(got, lins):
+        assert np.allclose(w, lin.weight.detach().numpy(), atol=1e-9) and np.allclose(b, lin.bias.detach().numpy(), atol=1e-9)
+    if depth == 2:
+        f0 = {"w1": layers0[0][0], "b1": layers0[0][1], "w2": layers0[1][0], "b2": layers0[1][1]}
+        two, l2 = orc.train_filter(f0, C, Y, epochs, lr=1e-2, weight_decay=0.02, batch_size=16)
+        assert np.allclose(l2, losses, atol=1e-12) and np.allclose(two["w2"], got[1][0], atol=1e-12)
