@@ -228,6 +228,12 @@ typedef struct {
 } l2pd_train_config;
 l2pd_status l2pd_filter_train(void *stream, int32_t s, int64_t N, const float *d_c, const uint8_t *d_y, float *d_w1,
                               float *d_b1, float *d_w2, float *d_b2, const l2pd_train_config *cfg, float *h_losses);
+/* The same for the depth variants of Section 4.4: n_layers in [1, 4] Linear(s, s) layers with ReLU between
+ * consecutive layers.  d_w, d_b: HOST arrays of n_layers DEVICE pointers ([s, s] row-major, [s]; fp32), initial values
+ * in, trained values out.  n_layers outside [1, 4] or a null entry: L2PD_ERR_ARG. */
+l2pd_status l2pd_filter_train_layers(void *stream, int32_t s, int32_t n_layers, int64_t N, const float *d_c,
+                                     const uint8_t *d_y, float *const *d_w, float *const *d_b,
+                                     const l2pd_train_config *cfg, float *h_losses);
 
 /* Number of sequences that still need steps (0 before the first reset). */
 int32_t l2pd_num_active(const l2pd_ctx *ctx);

@@ -60,7 +60,7 @@ class StepOut(C.Structure):
 
 
 EXPORTS = ["l2pd_init", "l2pd_state_reset", "l2pd_denoise_step", "l2pd_decode", "l2pd_num_active",
-           "l2pd_state_tokens", "l2pd_state_masked", "l2pd_set_unmask_rule", "l2pd_set_filter", "l2pd_set_collect", "l2pd_collect_count", "l2pd_filter_train", "l2pd_set_capture", "l2pd_last_step_rows",
+           "l2pd_state_tokens", "l2pd_state_masked", "l2pd_set_unmask_rule", "l2pd_set_filter", "l2pd_set_collect", "l2pd_collect_count", "l2pd_filter_train", "l2pd_filter_train_layers", "l2pd_set_capture", "l2pd_last_step_rows",
            "l2pd_launch_count", "l2pd_last_step_ms", "l2pd_profile_enable", "l2pd_profile_read", "l2pd_last_error", "l2pd_destroy",
            "l2pd_gemm_bf16", "l2pd_gemm_bf16_residual", "l2pd_gemm_bf16_swiglu", "l2pd_lm_head_bf16",
            "l2pd_lm_head_scratch_elems", "l2pd_attention_bf16", "l2pd_lm_head_bf16_static"]
@@ -92,6 +92,7 @@ def _load() -> C.CDLL:
     lib.l2pd_collect_count.argtypes = [vp]
     lib.l2pd_collect_count.restype = i64
     lib.l2pd_filter_train.argtypes = [vp, i32, i64, vp, vp, vp, vp, vp, vp, C.POINTER(TrainConfig), vp]
+    lib.l2pd_filter_train_layers.argtypes = [vp, i32, i32, i64, vp, vp, vp, vp, C.POINTER(TrainConfig), vp]
     lib.l2pd_last_step_rows.argtypes = [vp]
     lib.l2pd_launch_count.argtypes = [vp]
     lib.l2pd_launch_count.restype = i64
@@ -450,3 +451,25 @@ def filter_train(filt: Dict[str, np.ndarray], C_in, Y_in, epochs: int, lr: float
     _check(lib.l2pd_filter_train(_stream(), s, N, tc.data_ptr(), ty.data_ptr(), p["w1"].data_ptr(), p["b1"].data_ptr(),
                                  p["w2"].data_ptr(), p["b2"].data_ptr(), C.byref(cfg), losses.ctypes.data), None)
     return {k: v.cpu().numpy() for k, v in p.items()}, losses[: epochs * (-(-N // bs))]
+
+
+def filter_train_layers(layers, C_in, Y_in, epochs: int, lr: float = 1e-3, beta1: float = 0.9, beta2: float = 0.999,
+                        eps: float = 1e-8, weight_decay: float = 0.01, batch_size: int = 0, device: int = 0):
+    """filter_train for a filter given as a list of 1 to 4 (W [s, s], b [s]) layers; returns (layers, losses)."""
+    dev = "cuda:%d" % device
+    torch.cuda.set_device(device)
+    tc = (C_in if isinstance(C_in, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(C_in))).to(dev, torch.float32).contiguous()
+    ty = (Y_in if isinstance(Y_in, torch.Tensor) else torch.from_numpy(np.ascontiguousarray(Y_in))).to(dev, torch.uint8).contiguous()
+    N, s = int(tc.shape[0]), int(tc.shape[1])
+    ws = [torch.from_numpy(np.ascontiguousarray(w, dtype=np.float32)).to(dev) for w, _ in layers]
+    bs_ = [torch.from_numpy(np.ascontiguousarray(b_, dtype=np.float32)).to(dev) for _, b_ in layers]
+    n = len(layers)
+    pw = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in ws])
+    pb = (C.c_void_p * max(n, 1))(*[t.data_ptr() for t in bs_])
+    bsz = N if batch_size <= 0 else batch_size
+    updates = epochs * (-(-N // bsz))
+    losses = np.zeros(max(updates, 1), np.float32)
+    cfg = TrainConfig(lr, beta1, beta2, eps, weight_decay, epochs, batch_size)
+    _check(lib.l2pd_filter_train_layers(_stream(), s, n, N, tc.data_ptr(), ty.data_ptr(), pw, pb, C.byref(cfg),
+                                        losses.ctypes.data), None)
+    return [(w.cpu().numpy(), b_.cpu().numpy()) for w, b_ in zip(ws, bs_)], losses[:updates]

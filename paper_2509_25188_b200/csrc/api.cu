@@ -743,16 +743,18 @@ l2pd_status l2pd_set_collect(l2pd_ctx *c, float *d_c, uint8_t *d_y, int64_t capa
 }
 int64_t l2pd_collect_count(const l2pd_ctx *c) { return c ? c->collect_n : 0; }
 
-l2pd_status l2pd_filter_train(void *stream, int32_t s, int64_t N, const float *d_c, const uint8_t *d_y, float *d_w1,
-                              float *d_b1, float *d_w2, float *d_b2, const l2pd_train_config *t, float *h_losses) {
-  if (!d_c || !d_y || !d_w1 || !d_b1 || !d_w2 || !d_b2 || !t) return L2PD_ERR_ARG;
+static l2pd_status filter_train_impl(void *stream, int32_t s, int32_t L, int64_t N, const float *d_c, const uint8_t *d_y,
+                                     float *const *w, float *const *b, const l2pd_train_config *t, float *h_losses) {
+  if (!d_c || !d_y || !w || !b || !t) return L2PD_ERR_ARG;
+  if (L < 1 || L > 4) return L2PD_ERR_ARG;
+  for (int k = 0; k < L; ++k) if (!w[k] || !b[k]) return L2PD_ERR_ARG;
   if (s < 1 || s > 64 || N < 1) return L2PD_ERR_SHAPE;
   if (t->epochs < 0 || t->batch_size < 0 || !(t->lr > 0.f) || !(t->beta1 >= 0.f && t->beta1 < 1.f) ||
       !(t->beta2 >= 0.f && t->beta2 < 1.f) || !(t->eps > 0.f) || !(t->weight_decay >= 0.f)) return L2PD_ERR_ARG;
   cudaStream_t st = (cudaStream_t)stream;
   int dev = 0, sms = 148;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return L2PD_ERR_CUDA;
-  const int P = 2 * (s * s + s);
+  const int per = s * s + s, P = L * per;
   const int64_t bs = t->batch_size > 0 ? t->batch_size : N;
   const int64_t per_epoch = (N + bs - 1) / bs, updates = per_epoch * t->epochs;
   float *theta = nullptr, *gpart = nullptr, *losses = nullptr;
@@ -761,28 +763,37 @@ l2pd_status l2pd_filter_train(void *stream, int32_t s, int64_t N, const float *d
       cudaMalloc(&losses, sizeof(float) * (size_t)(updates > 0 ? updates : 1)) != cudaSuccess) { cleanup(); return L2PD_ERR_OOM; }
   float *m = theta + P, *v = theta + 2 * P;
   const size_t ss = sizeof(float) * s * s, sv = sizeof(float) * s;
-  bool ok = cudaMemcpyAsync(theta, d_w1, ss, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
-            cudaMemcpyAsync(theta + s * s, d_b1, sv, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
-            cudaMemcpyAsync(theta + s * s + s, d_w2, ss, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
-            cudaMemcpyAsync(theta + 2 * s * s + s, d_b2, sv, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
-            cudaMemsetAsync(m, 0, sizeof(float) * 2 * P, st) == cudaSuccess;
+  bool ok = cudaMemsetAsync(m, 0, sizeof(float) * 2 * P, st) == cudaSuccess;
+  for (int k = 0; ok && k < L; ++k)
+    ok = cudaMemcpyAsync(theta + k * per, w[k], ss, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+         cudaMemcpyAsync(theta + k * per + s * s, b[k], sv, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
   FilterTrainHyper h{t->lr, t->beta1, t->beta2, t->eps, t->weight_decay};
   double p1 = 1.0, p2 = 1.0;   // beta^t, carried in double
   int64_t u = 0;
   for (int e = 0; ok && e < t->epochs; ++e)
     for (int64_t lo = 0; ok && lo < N; lo += bs, ++u) {
       p1 *= t->beta1; p2 *= t->beta2;
-      ok = launch_filter_update(st, d_c, d_y, lo, (N - lo < bs ? N - lo : bs), s, theta, m, v, gpart, sms, h, 1.0 - p1, 1.0 - p2,
+      ok = launch_filter_update(st, d_c, d_y, lo, (N - lo < bs ? N - lo : bs), s, L, theta, m, v, gpart, sms, h, 1.0 - p1, 1.0 - p2,
                                 losses + u) == cudaSuccess;
     }
-  ok = ok && cudaMemcpyAsync(d_w1, theta, ss, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
-       cudaMemcpyAsync(d_b1, theta + s * s, sv, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
-       cudaMemcpyAsync(d_w2, theta + s * s + s, ss, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
-       cudaMemcpyAsync(d_b2, theta + 2 * s * s + s, sv, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
+  for (int k = 0; ok && k < L; ++k)
+    ok = cudaMemcpyAsync(w[k], theta + k * per, ss, cudaMemcpyDeviceToDevice, st) == cudaSuccess &&
+         cudaMemcpyAsync(b[k], theta + k * per + s * s, sv, cudaMemcpyDeviceToDevice, st) == cudaSuccess;
   if (ok && h_losses && updates > 0) ok = cudaMemcpyAsync(h_losses, losses, sizeof(float) * updates, cudaMemcpyDeviceToHost, st) == cudaSuccess;
   ok = (cudaStreamSynchronize(st) == cudaSuccess) && ok;
   cleanup();
   return ok ? L2PD_OK : L2PD_ERR_CUDA;
+}
+
+l2pd_status l2pd_filter_train(void *stream, int32_t s, int64_t N, const float *d_c, const uint8_t *d_y, float *d_w1,
+                              float *d_b1, float *d_w2, float *d_b2, const l2pd_train_config *t, float *h_losses) {
+  float *w[2] = {d_w1, d_w2}, *b[2] = {d_b1, d_b2};
+  return filter_train_impl(stream, s, 2, N, d_c, d_y, w, b, t, h_losses);
+}
+
+l2pd_status l2pd_filter_train_layers(void *stream, int32_t s, int32_t n_layers, int64_t N, const float *d_c, const uint8_t *d_y,
+                                     float *const *d_w, float *const *d_b, const l2pd_train_config *t, float *h_losses) {
+  return filter_train_impl(stream, s, n_layers, N, d_c, d_y, d_w, d_b, t, h_losses);
 }
 
 int32_t l2pd_num_active(const l2pd_ctx *c) { return c ? c->n_active : 0; }

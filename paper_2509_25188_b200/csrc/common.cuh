@@ -141,10 +141,10 @@ struct DecideArgs {
 cudaError_t launch_decide(cudaStream_t st, const DecideArgs &a, int n_slots);
 
 // filter_train.cu : one AdamW update of the filter on the samples [n0, n0 + n) (Algorithm 1, Eq. 6).
-// theta / m / v: packed W1 [s*s], b1 [s], W2 [s*s], b2 [s]; gpart: [grid, 2*(s*s+s) + 1] scratch;
+// theta / m / v: packed per layer W_k [s*s], b_k [s] (n_layers of them, 1 .. 4); gpart: [grid, n_layers*(s*s+s) + 1] scratch;
 // bc1 / bc2 = 1 - beta^t for this update's step count t; loss_out receives the batch's loss before the update.
 struct FilterTrainHyper { float lr, beta1, beta2, eps, weight_decay; };
-cudaError_t launch_filter_update(cudaStream_t st, const float *C, const uint8_t *Y, int64_t n0, int64_t n, int s,
+cudaError_t launch_filter_update(cudaStream_t st, const float *C, const uint8_t *Y, int64_t n0, int64_t n, int s, int n_layers,
                                  float *theta, float *m, float *v, float *gpart, int grid, const FilterTrainHyper &h,
                                  double bc1, double bc2, float *loss_out);
 

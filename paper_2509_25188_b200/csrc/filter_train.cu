@@ -6,10 +6,11 @@
 //   filter_grad_warp_kernel (s <= 32)  a warp per sample, lane j = block position j: the lane keeps row j of W1 and
 //                        W2 and the accumulators of row j of both gradients in registers; the sample's vectors
 //                        (c, h, dz) pass between lanes through 128-byte shared-memory slots read as broadcasts;
-//   filter_grad_kernel (s > 32)  every block walks tiles of 32 samples: forward (pre, h, z), dz = sigmoid(z) - y,
-//                        dh = dz W2, dpre = dh [pre > 0], and adds dz^T h, dpre^T c and the bias sums into
-//                        accumulators its threads own; a block ends by writing its sums (not yet divided by
-//                        the batch's element count) and its loss sum to its own row of `gpart`;
+//   filter_grad_kernel (s > 32, or the depth variants of Section 4.4: 1 to 4 layers)  every block walks tiles of
+//                        32 samples: forward through the layers, dz = sigmoid(z) - y, then layer by layer
+//                        downwards dW_k += delta_k^T x_k, db_k += sum delta_k, delta_{k-1} = (delta_k W_k) [x_k > 0],
+//                        into accumulators its threads own; a block ends by writing its sums (not yet divided
+//                        by the batch's element count) and its loss sum to its own row of `gpart`;
 //   filter_adamw_kernel  one thread per parameter adds the rows in block order (so a run is bit-reproducible), scales by
 //                        1 / (samples * s) and applies AdamW: decoupled weight decay, bias-corrected moments.
 // The whole problem (a few thousand parameters, samples of s floats) lives in shared memory and L2; the
@@ -30,37 +31,41 @@ struct GradArgs {
   const uint8_t *Y;        // [N, s] targets (0 / 1)
   int64_t n0, n;           // the batch: samples [n0, n0 + n)
   int s;
-  const float *theta;      // packed: W1 [s*s], b1 [s], W2 [s*s], b2 [s]
+  int n_layers;            // 1 .. 4 Linear(s, s) layers, ReLU between consecutive layers
+  const float *theta;      // packed per layer: W_k [s*s], b_k [s]
   float *gpart;            // [gridDim.x, P + 1]: gradient sums, then the loss sum
 };
 
+constexpr int MAX_LAYERS = 4;
+
+// Any depth, any s <= 64: every block walks tiles of 32 samples held in shared memory.
 __global__ void __launch_bounds__(GRAD_THREADS) filter_grad_kernel(GradArgs a) {
   extern __shared__ float sm[];
-  const int s = a.s, sp = s + 1;     // padded row stride: rows read side by side fall into different banks
-  float *W1 = sm;                    // [s][sp]
-  float *W2 = W1 + s * sp;           // [s][sp]
-  float *b1 = W2 + s * sp;           // [s]
-  float *b2 = b1 + s;                // [s]
-  float *Ct = b2 + s;                // [TB][sp] inputs of the tile
-  float *Ht = Ct + TB * sp;          // [TB][sp] hidden activations
-  float *Zt = Ht + TB * sp;          // [TB][sp] dz
-  float *Pt = Zt + TB * sp;          // [TB][sp] pre-activations, then dpre
+  const int s = a.s, sp = s + 1, L = a.n_layers;   // padded row stride: rows read side by side fall into different banks
+  float *W = sm;                      // [L][s][sp]
+  float *Bv = W + L * s * sp;         // [L][s]
+  float *X = Bv + L * s;              // [L][TB][sp]: X[0] the inputs, X[k] = relu(output of layer k - 1)
+  float *D0 = X + L * TB * sp;        // [TB][sp] delta of the layer being differentiated
+  float *D1 = D0 + TB * sp;           // [TB][sp] delta of the layer below
   __shared__ float red[GRAD_THREADS / 32];
 
   grid_dep_launch();
   grid_dep_wait();
   const int tid = threadIdx.x;
-  const int P = 2 * (s * s + s);
-  for (int e = tid; e < s * s; e += GRAD_THREADS) {
-    W1[(e / s) * sp + e % s] = a.theta[e];
-    W2[(e / s) * sp + e % s] = a.theta[s * s + s + e];
+  const int per = s * s + s, P = L * per;
+  for (int k = 0; k < L; ++k) {
+    for (int e = tid; e < s * s; e += GRAD_THREADS) W[(k * s + e / s) * sp + e % s] = a.theta[k * per + e];
+    if (tid < s) Bv[k * s + tid] = a.theta[k * per + s * s + tid];
   }
-  if (tid < s) { b1[tid] = a.theta[s * s + tid]; b2[tid] = a.theta[2 * s * s + s + tid]; }
 
-  float acc1[MAX_OWN], acc2[MAX_OWN];
+  float acc[MAX_LAYERS][MAX_OWN], gb[MAX_LAYERS];
 #pragma unroll
-  for (int k = 0; k < MAX_OWN; ++k) { acc1[k] = 0.f; acc2[k] = 0.f; }
-  float gb1 = 0.f, gb2 = 0.f, loss = 0.f;
+  for (int k = 0; k < MAX_LAYERS; ++k) {
+    gb[k] = 0.f;
+#pragma unroll
+    for (int q = 0; q < MAX_OWN; ++q) acc[k][q] = 0.f;
+  }
+  float loss = 0.f;
 
   const int64_t n_tiles = (a.n + TB - 1) / TB;
   for (int64_t tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
@@ -69,62 +74,77 @@ __global__ void __launch_bounds__(GRAD_THREADS) filter_grad_kernel(GradArgs a) {
     __syncthreads();                                   // the previous tile's buffers are no longer read
     for (int e = tid; e < TB * s; e += GRAD_THREADS) {
       const int n = e / s, i = e - n * s;
-      Ct[n * sp + i] = n < rows ? a.C[(base + n) * s + i] : 0.f;
+      X[n * sp + i] = n < rows ? a.C[(base + n) * s + i] : 0.f;
     }
     __syncthreads();
-    for (int o = tid; o < TB * s; o += GRAD_THREADS) {   // pre = W1 c + b1, h = relu(pre)
-      const int n = o / s, j = o - n * s;
-      float v = b1[j];
-      for (int i = 0; i < s; ++i) v = fmaf(W1[j * sp + i], Ct[n * sp + i], v);
-      Pt[n * sp + j] = v;
-      Ht[n * sp + j] = fmaxf(v, 0.f);
-    }
-    __syncthreads();
-    for (int o = tid; o < TB * s; o += GRAD_THREADS) {   // z = W2 h + b2; dz and the loss of Eq. 6
-      const int n = o / s, j = o - n * s;
-      float z = b2[j];
-      for (int i = 0; i < s; ++i) z = fmaf(W2[j * sp + i], Ht[n * sp + i], z);
-      float dz = 0.f;
-      if (n < rows) {
-        const float y = (float)a.Y[(base + n) * s + j];
-        dz = 1.0f / (1.0f + expf(-z)) - y;
-        loss += fmaxf(z, 0.f) - z * y + log1pf(expf(-fabsf(z)));
-      }
-      Zt[n * sp + j] = dz;
-    }
-    __syncthreads();
-    for (int o = tid; o < TB * s; o += GRAD_THREADS) {   // dpre = (dz W2) [pre > 0]
-      const int n = o / s, i = o - n * s;
-      float v = 0.f;
-      for (int j = 0; j < s; ++j) v = fmaf(Zt[n * sp + j], W2[j * sp + i], v);
-      Pt[n * sp + i] = Pt[n * sp + i] > 0.f ? v : 0.f;   // each thread replaces the pre-activation it alone reads
-    }
-    __syncthreads();
-#pragma unroll
-    for (int k = 0; k < MAX_OWN; ++k) {                  // dW2 += dz^T h, dW1 += dpre^T c
-      const int e = tid + k * GRAD_THREADS;
-      if (e < s * s) {
-        const int j = e / s, i = e - j * s;
-        float v1 = acc1[k], v2 = acc2[k];
-        for (int n = 0; n < TB; ++n) {
-          v2 = fmaf(Zt[n * sp + j], Ht[n * sp + i], v2);
-          v1 = fmaf(Pt[n * sp + j], Ct[n * sp + i], v1);
+    // forward: layer k maps X[k] to X[k + 1] = relu(.), the last layer to dz = sigmoid(z) - y in D0
+    for (int k = 0; k < L; ++k) {
+      const float *xin = X + k * TB * sp, *wk = W + k * s * sp;
+      for (int o = tid; o < TB * s; o += GRAD_THREADS) {
+        const int n = o / s, j = o - n * s;
+        float v = Bv[k * s + j];
+        for (int i = 0; i < s; ++i) v = fmaf(wk[j * sp + i], xin[n * sp + i], v);
+        if (k + 1 < L) {
+          X[(k + 1) * TB * sp + n * sp + j] = fmaxf(v, 0.f);
+        } else {
+          float dz = 0.f;
+          if (n < rows) {
+            const float y = (float)a.Y[(base + n) * s + j];
+            dz = 1.0f / (1.0f + expf(-v)) - y;
+            loss += fmaxf(v, 0.f) - v * y + log1pf(expf(-fabsf(v)));
+          }
+          D0[n * sp + j] = dz;
         }
-        acc1[k] = v1; acc2[k] = v2;
       }
+      __syncthreads();
     }
-    if (tid < s) {
-      for (int n = 0; n < TB; ++n) { gb2 += Zt[n * sp + tid]; gb1 += Pt[n * sp + tid]; }
+    // backward: dW_k += delta_k^T X[k], db_k += sum delta_k, delta_{k-1} = (delta_k W_k) [X[k] > 0]
+    float *dcur = D0, *dnxt = D1;
+#pragma unroll
+    for (int kk = 0; kk < MAX_LAYERS; ++kk) {
+      const int k = L - 1 - kk;
+      if (k < 0) break;
+      const float *xin = X + k * TB * sp, *wk = W + k * s * sp;
+#pragma unroll
+      for (int q = 0; q < MAX_OWN; ++q) {
+        const int e = tid + q * GRAD_THREADS;
+        if (e < s * s) {
+          const int j = e / s, i = e - j * s;
+          float v = acc[kk][q];
+          for (int n = 0; n < TB; ++n) v = fmaf(dcur[n * sp + j], xin[n * sp + i], v);
+          acc[kk][q] = v;
+        }
+      }
+      if (tid < s) {
+        float v = gb[kk];
+        for (int n = 0; n < TB; ++n) v += dcur[n * sp + tid];
+        gb[kk] = v;
+      }
+      if (k > 0) {
+        for (int o = tid; o < TB * s; o += GRAD_THREADS) {
+          const int n = o / s, i = o - n * s;
+          float v = 0.f;
+          for (int j = 0; j < s; ++j) v = fmaf(dcur[n * sp + j], wk[j * sp + i], v);
+          dnxt[n * sp + i] = xin[n * sp + i] > 0.f ? v : 0.f;
+        }
+      }
+      __syncthreads();
+      float *t = dcur; dcur = dnxt; dnxt = t;
     }
   }
 
   float *out = a.gpart + (int64_t)blockIdx.x * (P + 1);
 #pragma unroll
-  for (int k = 0; k < MAX_OWN; ++k) {
-    const int e = tid + k * GRAD_THREADS;
-    if (e < s * s) { out[e] = acc1[k]; out[s * s + s + e] = acc2[k]; }
+  for (int kk = 0; kk < MAX_LAYERS; ++kk) {       // acc[kk] belongs to layer L - 1 - kk
+    const int k = L - 1 - kk;
+    if (k < 0) break;
+#pragma unroll
+    for (int q = 0; q < MAX_OWN; ++q) {
+      const int e = tid + q * GRAD_THREADS;
+      if (e < s * s) out[k * per + e] = acc[kk][q];
+    }
+    if (tid < s) out[k * per + s * s + tid] = gb[kk];
   }
-  if (tid < s) { out[s * s + tid] = gb1; out[2 * s * s + s + tid] = gb2; }
   for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xffffffffu, loss, o);
   if ((tid & 31) == 0) red[tid >> 5] = loss;
   __syncthreads();
@@ -299,22 +319,17 @@ __global__ void __launch_bounds__(ADAM_THREADS) filter_adamw_kernel(AdamArgs a) 
 
 }  // namespace
 
-size_t filter_grad_smem(int s) { return sizeof(float) * (size_t)(2 * s * (s + 1) + 2 * s + 4 * TB * (s + 1)); }
+size_t filter_grad_smem(int s, int L) { return sizeof(float) * (size_t)(L * s * (s + 1) + L * s + (L + 2) * TB * (s + 1)); }
 constexpr size_t WG_SMEM = sizeof(float) * (32 * WG_ROW + 3 * WG_WARPS * 32 + WG_WARPS * (2 * 1024 + 64));
 
-cudaError_t launch_filter_update(cudaStream_t st, const float *C, const uint8_t *Y, int64_t n0, int64_t n, int s,
+cudaError_t launch_filter_update(cudaStream_t st, const float *C, const uint8_t *Y, int64_t n0, int64_t n, int s, int n_layers,
                                  float *theta, float *m, float *v, float *gpart, int grid, const FilterTrainHyper &h,
                                  double bc1, double bc2, float *loss_out) {
-  static bool attr = false;
-  if (!attr) {
-    cudaError_t e = cudaFuncSetAttribute(filter_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)filter_grad_smem(MAX_S));
-    if (e != cudaSuccess) return e;
-    attr = true;
-  }
-  GradArgs g{C, Y, n0, n, s, theta, gpart};
+  if (n_layers < 1 || n_layers > MAX_LAYERS || s < 1 || s > MAX_S) return cudaErrorInvalidValue;
+  GradArgs g{C, Y, n0, n, s, n_layers, theta, gpart};
   int blocks;
   cudaError_t e;
-  if (s <= 32) {
+  if (s <= 32 && n_layers == 2) {
     static bool attr_w = false;
     if (!attr_w) {
       e = cudaFuncSetAttribute(filter_grad_warp_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)WG_SMEM);
@@ -325,13 +340,19 @@ cudaError_t launch_filter_update(cudaStream_t st, const float *C, const uint8_t 
     blocks = (int)(want < grid ? want : grid);
     e = launch_kernel(filter_grad_warp_kernel, dim3(blocks), dim3(WG_WARPS * 32), WG_SMEM, st, g);
   } else {
+    static bool attr = false;
+    if (!attr) {
+      e = cudaFuncSetAttribute(filter_grad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)filter_grad_smem(MAX_S, MAX_LAYERS));
+      if (e != cudaSuccess) return e;
+      attr = true;
+    }
     const int64_t n_tiles = (n + TB - 1) / TB;
     blocks = (int)(n_tiles < grid ? n_tiles : grid);
-    e = launch_kernel(filter_grad_kernel, dim3(blocks), dim3(GRAD_THREADS), filter_grad_smem(s), st, g);
+    e = launch_kernel(filter_grad_kernel, dim3(blocks), dim3(GRAD_THREADS), filter_grad_smem(s, n_layers), st, g);
   }
   if (e != cudaSuccess) return e;
   AdamArgs a{};
-  a.gpart = gpart; a.n_blocks = blocks; a.P = 2 * (s * s + s);
+  a.gpart = gpart; a.n_blocks = blocks; a.P = n_layers * (s * s + s);
   a.inv_count = (float)(1.0 / ((double)n * s));
   a.lr = h.lr; a.beta1 = h.beta1; a.beta2 = h.beta2; a.eps = h.eps; a.weight_decay = h.weight_decay;
   a.bc1 = (float)bc1; a.bc2 = (float)bc2;

@@ -125,3 +125,25 @@ def test_egp_collection_then_training_end_to_end():
     for i in range(B):
         assert steps2[i] == ref2[i].steps and np.array_equal(toks2[i], ref2[i].response)
     dec2.close()
+
+
+@pytest.mark.parametrize("depth,s,n,batch", [(1, 32, 300, 0), (4, 32, 500, 128), (3, 16, 77, 0), (4, 64, 200, 0), (2, 64, 333, 100)])
+def test_depth_variant_training_matches_the_oracle(depth, s, n, batch):
+    """Section 4.4's one- and four-layer filters (and three): the tiled kernel's backpropagation through
+    the layers against the oracle's, ragged tiles and batches included; depth 2 at s = 64 runs the same
+    kernel as the two-layer entry point."""
+    C, Y = _data(s, n, seed=depth * 100 + s)
+    rng = np.random.default_rng(depth)
+    layers0 = [((rng.normal(size=(s, s)) / np.sqrt(s)).astype(np.float32), (0.1 * rng.normal(size=s)).astype(np.float32))
+               for _ in range(depth)]
+    epochs = 120 if batch == 0 else 40
+    want, want_l = orc.train_filter_layers(layers0, C.astype(np.float64), Y.astype(np.float64), epochs, lr=5e-3, batch_size=batch)
+    got, losses = _b().filter_train_layers(layers0, C, Y, epochs, lr=5e-3, batch_size=batch)
+    assert len(losses) == len(want_l) and np.abs(losses - want_l).max() < 2e-4
+    for (w, b), (ww, wb) in zip(got, want):
+        assert np.abs(w - ww).max() < 2e-3 and np.abs(b - wb).max() < 2e-3
+    assert losses[-1] < losses[0]
+    b_ = _b()
+    with pytest.raises(b_.L2pdError) as e:
+        b_.filter_train_layers(layers0 * 5, C, Y, 1)          # more than four layers
+    assert e.value.status == -1
