@@ -60,6 +60,7 @@ GEMM_SHAPES = [
     (32, 12288, 4096, 0),       # the QKV projection of a 32-row step, automatic plan
     (256, 2048, 1032, 1002240), # alternate k-blocks on a pair of SMs (one 256-row slab), K tail
     (200, 12288, 4096, 0),      # QKV at 200 rows, automatic plan
+    (64, 8192, 320, 1001032),   # alternate k-blocks with several units per CTA (the accumulators are reused unit after unit)
 ]
 
 
@@ -108,7 +109,8 @@ def test_gemm_bf16_residual(M, N, K, tile_n):
                                           (512, 1408, 512, 202160), (300, 2048, 256, 202256),
                                           (512, 1408, 512, 202176), (200, 336, 192, 1176), (130, 1408, 128, 2144),
                                           (512, 24576, 256, 0), (32, 1408, 4096, 1000176), (90, 336, 192, 1000064),
-                                          (32, 12288, 4096, 0), (256, 1408, 4096, 1002176), (256, 12288, 4096, 0)])
+                                          (32, 12288, 4096, 0), (256, 1408, 4096, 1002176), (256, 12288, 4096, 0),
+                                          (32, 8192, 192, 1001064)])
 def test_gemm_bf16_swiglu(M, F, K, tile_n):
     b = _b()
     A = _bf16(3, 0, (M, K), 1.0)
