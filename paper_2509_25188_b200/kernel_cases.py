@@ -41,6 +41,8 @@ def main():
     ap.add_argument("--vocab", type=int, default=126464)
     ap.add_argument("--heads", type=int, default=32)
     ap.add_argument("--layers", type=int, default=2, help="step: number of layers")
+    ap.add_argument("--kv-cache", type=int, default=0, help="step: 0 = every step runs all --rows positions; 1 / 2 = prefix / dual "
+                    "cache: the timed steps are in-block steps of the first block (at most 31 of them in all)")
     ap.add_argument("--impl", type=int, default=0, help="attn: 0 = tcgen05 kernel, 1 = mma.sync kernel")
     ap.add_argument("--ring", type=int, default=0, help="number of weight buffers to rotate through (0 = enough to exceed L2)")
     a = ap.parse_args()
@@ -65,11 +67,18 @@ def main():
              "final_norm": torch.full((d,), wl.spread_gain(shape), device=dev),
              "layers": [{"wqkv": rnd(3 * d, d), "wo": rnd(d, d), "w_gate": rnd(F, d), "w_up": rnd(F, d),
                          "w_down": rnd(d, F), "norm1": ones, "norm2": ones} for _ in range(a.layers)]}
-        dec = b.Decoder(shape, w, wl.make_filter(32, 0.96, seed=0), block_len=32, max_batch=1, max_seq=T)
+        dec = b.Decoder(shape, w, wl.make_filter(32, 0.96, seed=0), block_len=32, max_batch=1, max_seq=T,
+                        kv_cache=a.kv_cache, use_filter=a.kv_cache == 0)
         prompts = torch.from_numpy(wl.make_prompts(1, T // 2, shape, seed=1)).to(dev)
+        if a.kv_cache:
+            # one commit per step: the first block has 31 steps that read the store
+            assert a.warmup + 2 * a.iters <= 31, "at most 31 in-block steps"
+            dec.state_reset_device(prompts, T - T // 2)
+            dec.denoise_step(outputs=False)
 
         def run(i):
-            dec.state_reset_device(prompts, T - T // 2)
+            if not a.kv_cache:
+                dec.state_reset_device(prompts, T - T // 2)
             dec.denoise_step(outputs=False)
         per_layer = 2.0 * T * (4 * d * d + 3 * d * F) + 4.0 * T * T * d
         flops, byts = a.layers * per_layer + 2.0 * 32 * d * V, 2.0 * (a.layers * (4 * d * d + 3 * d * F) + V * d)
