@@ -271,13 +271,35 @@ enum {
   L2PD_K_LM_HEAD = 9,     /* LM head + confidence/argmax reduction */
   L2PD_K_DECIDE = 10,     /* filter, threshold, commit, EoTP */
   L2PD_K_OTHER = 11,
-  L2PD_K_COUNT = 12
+  L2PD_K_CHAIN = 12,      /* chained launch: O projection, RMSNorm, gate/up, down, next layer's RMSNorm and QKV */
+  L2PD_K_COUNT = 13
 };
 /* Selects kinds (bit k = kind k) whose launches are bracketed by CUDA events on the step's
  * stream from now on, and clears the accumulated totals; mask 0 turns timing off. */
 l2pd_status l2pd_profile_enable(l2pd_ctx *ctx, uint32_t kind_mask);
 /* Accumulated device time (ms) and launch count of one kind since the last enable. */
 l2pd_status l2pd_profile_read(const l2pd_ctx *ctx, int32_t kind, double *ms_total, int64_t *launches);
+
+/*
+ * Chained launches.  When every projection of a step runs on SM pairs with two row slabs per unit (a few
+ * hundred to a few thousand rows, bf16, rotation fused into the QKV projection), the step runs, per layer, the
+ * attention kernel and ONE persistent launch that holds the output projection, the RMSNorm before the MLP, the
+ * gate/up and down projections and the next layer's RMSNorm and QKV projection; the results are bit-identical to
+ * the one-launch-per-projection form.  l2pd_set_chain(ctx, 1) selects the chained form, 0 (the state after
+ * l2pd_init) one launch per projection; it may be called between steps.  Measured at 512 rows the two forms
+ * take the same time within a few percent (programmatic dependent launch already hides the launch and the
+ * ring fill of a projection behind the one before it), hence the default.
+ * l2pd_chain_trace_enable(ctx, 1) makes every chained launch of the following steps record, per phase and CTA,
+ * the nanosecond timer at which the CTA opened the phase, had its first and its last accumulator ready (for an
+ * RMSNorm phase both equal the opening) and finished the phase; l2pd_chain_trace_read copies the last step's
+ * records to HOST memory as [launch][phase slot][opened, first ready, last ready, finished][CTA] uint64 (phase
+ * slots beyond a launch's phases hold stale values) and returns their count (call with h_out = NULL to size
+ * the buffer; -1 on a CUDA error); it synchronises the device.  (0) frees the record buffer.
+ */
+l2pd_status l2pd_set_chain(l2pd_ctx *ctx, int32_t enable);
+l2pd_status l2pd_chain_trace_enable(l2pd_ctx *ctx, int32_t enable);
+int64_t l2pd_chain_trace_read(l2pd_ctx *ctx, uint64_t *h_out, int64_t capacity, int32_t *launches, int32_t *phases,
+                              int32_t *ctas);
 
 /* Device time of the most recent step in milliseconds (CUDA events on the step's stream),
  * or a negative value if no step has run. */

@@ -63,11 +63,12 @@ EXPORTS = ["l2pd_init", "l2pd_state_reset", "l2pd_denoise_step", "l2pd_decode", 
            "l2pd_state_tokens", "l2pd_state_masked", "l2pd_set_unmask_rule", "l2pd_set_filter", "l2pd_set_collect", "l2pd_collect_count", "l2pd_filter_train", "l2pd_filter_train_layers", "l2pd_set_capture", "l2pd_last_step_rows",
            "l2pd_launch_count", "l2pd_last_step_ms", "l2pd_profile_enable", "l2pd_profile_read", "l2pd_last_error", "l2pd_destroy",
            "l2pd_gemm_bf16", "l2pd_gemm_bf16_residual", "l2pd_gemm_bf16_swiglu", "l2pd_lm_head_bf16",
-           "l2pd_lm_head_scratch_elems", "l2pd_attention_bf16", "l2pd_lm_head_bf16_static"]
+           "l2pd_lm_head_scratch_elems", "l2pd_attention_bf16", "l2pd_lm_head_bf16_static",
+           "l2pd_set_chain", "l2pd_chain_trace_enable", "l2pd_chain_trace_read"]
 
 
 KINDS = ["embed", "gemm_qkv", "rope", "attention", "gemm_o", "rmsnorm", "gemm_gate_up", "gemm_down",
-         "final_norm", "lm_head", "decide", "other"]
+         "final_norm", "lm_head", "decide", "other", "gemm_chain"]
 
 
 def _load() -> C.CDLL:
@@ -112,6 +113,10 @@ def _load() -> C.CDLL:
     lib.l2pd_lm_head_scratch_elems.restype = i64
     lib.l2pd_lm_head_bf16_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, i32]
     lib.l2pd_attention_bf16.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, i64, i32, i32]
+    lib.l2pd_set_chain.argtypes = [vp, i32]
+    lib.l2pd_chain_trace_enable.argtypes = [vp, i32]
+    lib.l2pd_chain_trace_read.argtypes = [vp, vp, i64, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
+    lib.l2pd_chain_trace_read.restype = i64
     return lib
 
 
@@ -315,6 +320,26 @@ class Decoder:
     @property
     def collect_count(self) -> int:
         return int(lib.l2pd_collect_count(self.ctx))
+
+    # ---- chained launches ------------------------------------------------------------------------
+    def set_chain(self, enable: bool):
+        """False: one launch per projection; True (the default): one persistent launch per layer where the shapes allow."""
+        _check(lib.l2pd_set_chain(self.ctx, int(bool(enable))), self.ctx)
+
+    def chain_trace_enable(self, enable: bool = True):
+        _check(lib.l2pd_chain_trace_enable(self.ctx, int(bool(enable))), self.ctx)
+
+    def chain_trace(self) -> Optional[np.ndarray]:
+        """Stamps of the last step's chained launches, uint64 [launch, phase slot, 4 (opened, first / last accumulator ready, finished), CTA] in ns."""
+        nl, nph, nc = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+        n = lib.l2pd_chain_trace_read(self.ctx, None, 0, C.byref(nl), C.byref(nph), C.byref(nc))
+        if n <= 0:
+            return None
+        out = np.zeros(n, np.uint64)
+        got = lib.l2pd_chain_trace_read(self.ctx, out.ctypes.data, n, C.byref(nl), C.byref(nph), C.byref(nc))
+        if got != n:
+            raise L2pdError(-4, "chain trace read failed")
+        return out.reshape(nl.value, nph.value, 4, nc.value)
 
     # ---- state and instrumentation -------------------------------------------------------------
     @property

@@ -79,11 +79,29 @@ struct l2pd_ctx {
   TmaDesc ta_n, ta_att, ta_h, ta_nf, ta_q, t_kstore, t_vstore;
   // output maps of the four projections (staged epilogue stores); re-encoded when rows or tile width change
   TmaDesc tc_qkv, tc_o, tc_h, tc_down;
+  // the same for each projection's last, narrower column tile (chained launches stage every tile); tail width, 0 = none
+  TmaDesc tct_qkv, tct_o, tct_h, tct_down;
+  int tail_qkv = 0, tail_o = 0, tail_h = 0, tail_down = 0;
   int tc_rows = -1, tcw_qkv = 0, tcw_o = 0, tcw_h = 0, tcw_down = 0;   // tile width encoded (0 = none, -w = not usable for w)
   std::vector<TmaDesc> tb_qkv, tb_o, tb_gate, tb_up, tb_down;
   TmaDesc tb_lm;
   GemmPlan pl_qkv{}, pl_o{}, pl_gu{}, pl_down{};
   int box_qkv = 0, box_o = 0, box_gu = 0, box_down = 0, tn_lm = 0;
+
+  // several projections per launch (gemm_chain.cu): on when every projection of the step runs on SM pairs with
+  // two row slabs per unit and K slices store partial sums
+  bool chain_on = false;             // l2pd_set_chain
+  int chain_clusters = 0;            // CTA pairs that can be resident at once (0: kernel not usable here)
+  unsigned int *d_chain_bar = nullptr;
+  unsigned int chain_bar_base = 0;   // host copy of the counter's value
+  // one table per chained launch of a step (first QKV, then one per layer), device-resident, rebuilt when the step's
+  // row count (hence tiling and output maps) changes
+  uint8_t *d_chain_tabs = nullptr, *h_chain_tabs = nullptr;
+  std::vector<ChainTableInfo> chain_info;
+  int chain_tab_rows = -1;
+  unsigned long long *d_chain_trace = nullptr;   // l2pd_chain_trace_enable: [launch][phase][4][CTA] stamps of the last step
+  int64_t chain_trace_cap = 0;
+  int chain_trace_launches = 0, chain_trace_phases = 0, chain_trace_ctas = 0;
 
   // debug capture
   float *cap = nullptr;
@@ -111,6 +129,11 @@ bool pdl_enabled() {
 }  // namespace l2pd
 
 namespace {
+
+constexpr int CHAIN_TILE_N = 176;       // widest tile of a step that chains projections
+constexpr int CHAIN_MAX_ROWS = 1536;    // steps of more rows run one launch per projection (the launch is then a small part)
+constexpr int CHAIN_TRACE_STAMPS = 4;   // stamps per phase and CTA
+constexpr int CHAIN_TRACE_PHASES = 6;   // phases a chained launch can hold (slots per launch in the trace)
 
 l2pd_status set_err(l2pd_ctx *c, l2pd_status s, const char *fmt, ...) {
   if (c) {
@@ -201,8 +224,8 @@ l2pd_status run_gemm_simt(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const 
 
 int64_t round_up(int64_t a, int64_t b);
 
-l2pd_status run_gemm_tc(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const TmaDesc *a, const TmaDesc *b,
-                        const TmaDesc *b2, const TmaDesc *cm, void *out, int M, int N, int K, const GemmPlan &pl) {
+GemmArgs make_gemm_args(l2pd_ctx *c, int epi, const TmaDesc *a, const TmaDesc *b, const TmaDesc *b2, const TmaDesc *cm,
+                        void *out, int M, int N, int K, const GemmPlan &pl) {
   GemmArgs g{};
   if (epi == EPI_RESIDUAL && c->ksum && effective_k_splits(K, pl.k_splits) > 1) { g.part = c->ksum; g.part_rows = (int)round_up(M, 512); }
   g.epi = epi; g.a = a; g.b = b; g.b2 = b2; g.c = cm; g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.out = out;
@@ -212,6 +235,12 @@ l2pd_status run_gemm_tc(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const Tm
     g.rope_cols = 2 * c->cfg.n_heads * c->cfg.head_dim; g.rope_dh = c->cfg.head_dim;
     g.cs_table = c->cs_table_t; g.cs_stride = c->cfg.max_seq; g.row_pos = c->d_row_pos;
   }
+  return g;
+}
+
+l2pd_status run_gemm_tc(l2pd_ctx *c, cudaStream_t s, int kind, int epi, const TmaDesc *a, const TmaDesc *b,
+                        const TmaDesc *b2, const TmaDesc *cm, void *out, int M, int N, int K, const GemmPlan &pl) {
+  const GemmArgs g = make_gemm_args(c, epi, a, b, b2, cm, out, M, N, K, pl);
   CKLK(kind, launch_gemm_tcgen05(s, g, c->num_sms));
   return L2PD_OK;
 }
@@ -227,17 +256,20 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
   if (tc) {
     // the tiling follows the row count of this step; weight tensor maps are re-encoded when the
     // box (rows of the weight tile one CTA loads) changes
-    c->pl_qkv = plan_gemm(EPI_STORE, T_rows, 3 * hd, d, c->num_sms, 0);
+    // contexts that can chain the projections of a layer into one launch keep every tile at most CHAIN_TILE_N wide:
+    // the chained kernel has one ring for all of them, and that width leaves it five stages
+    const int max_tn = (c->chain_clusters > 0 && T_rows > 256 && T_rows <= CHAIN_MAX_ROWS && T_rows <= c->ksum_rows) ? CHAIN_TILE_N : 256;
+    c->pl_qkv = plan_gemm(EPI_STORE, T_rows, 3 * hd, d, c->num_sms, 0, 4, max_tn);
     int box = c->pl_qkv.tile_n / c->pl_qkv.cta_group;
     if (box != c->box_qkv) { l2pd_status r = encode_weight_maps(c, c->tb_qkv, c->wqkv, 3 * hd, d, box); if (r) return r; c->box_qkv = box; }
     const int max_ks = (c->ksum == nullptr || T_rows <= c->ksum_rows) ? 4 : 1;   // K slices need their partial-sum area
-    c->pl_o = plan_gemm(EPI_RESIDUAL, T_rows, d, hd, c->num_sms, 0, max_ks);
+    c->pl_o = plan_gemm(EPI_RESIDUAL, T_rows, d, hd, c->num_sms, 0, max_ks, max_tn);
     box = c->pl_o.tile_n / c->pl_o.cta_group;
     if (box != c->box_o) { l2pd_status r = encode_weight_maps(c, c->tb_o, c->wo, d, hd, box); if (r) return r; c->box_o = box; }
-    c->pl_down = plan_gemm(EPI_RESIDUAL, T_rows, d, F, c->num_sms, 0, max_ks);
+    c->pl_down = plan_gemm(EPI_RESIDUAL, T_rows, d, F, c->num_sms, 0, max_ks, max_tn);
     box = c->pl_down.tile_n / c->pl_down.cta_group;
     if (box != c->box_down) { l2pd_status r = encode_weight_maps(c, c->tb_down, c->w_down, d, F, box); if (r) return r; c->box_down = box; }
-    c->pl_gu = plan_gemm(EPI_SWIGLU, T_rows, F, d, c->num_sms, 0);
+    c->pl_gu = plan_gemm(EPI_SWIGLU, T_rows, F, d, c->num_sms, 0, 4, max_tn);
     box = c->pl_gu.tile_n / 2;
     if (box != c->box_gu) {
       l2pd_status r = encode_weight_maps(c, c->tb_gate, c->w_gate, F, d, box); if (r) return r;
@@ -270,6 +302,17 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     r = out_map_x(c->tc_o, c->tcw_o, ks_o, c->pl_o.tile_n); if (r) return r;
     r = out_map(c->tc_h, c->tcw_h, c->h, false, F, c->pl_gu.tile_n / 2); if (r) return r;
     r = out_map_x(c->tc_down, c->tcw_down, ks_d, c->pl_down.tile_n); if (r) return r;
+    if (c->tc_rows != T_rows && c->chain_clusters > 0 && T_rows <= CHAIN_MAX_ROWS) {
+      // maps of the last, narrower column tiles (-1: a tail the staged epilogue cannot take; the step then does not chain)
+      auto tail_map = [&](TmaDesc &m, int &tail, void *ptr, bool fp32, int64_t rows, int64_t N, int w, int mult = 16) {
+        tail = (int)(N % w);
+        if (tail && ((tail % mult) || make_tma_out_tail(&m, ptr, fp32, rows, N, tail) != L2PD_OK)) tail = -1;
+      };
+      tail_map(c->tct_qkv, c->tail_qkv, c->qkv, false, T_rows, 3 * hd, c->pl_qkv.tile_n);
+      tail_map(c->tct_o, c->tail_o, ks_o > 1 ? (void *)c->ksum : (void *)c->x, true, ks_o > 1 ? ks_o * mpad : T_rows, d, c->pl_o.tile_n);
+      tail_map(c->tct_h, c->tail_h, c->h, false, T_rows, F, c->pl_gu.tile_n / 2, 8);   // SwiGLU drains 16 columns at a time: any multiple of 8
+      tail_map(c->tct_down, c->tail_down, ks_d > 1 ? (void *)c->ksum : (void *)c->x, true, ks_d > 1 ? ks_d * mpad : T_rows, d, c->pl_down.tile_n);
+    }
     c->tc_rows = T_rows;
   }
 
@@ -278,7 +321,91 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
                               c->norm1[0], f.rms_eps, c->x, n, T_rows, d));
   if (c->cap) CK(cudaMemcpyAsync(c->cap, c->x, (size_t)T_rows * d * 4, cudaMemcpyDeviceToDevice, s));
 
-  for (int l = 0; l < f.n_layers; ++l) {
+  // The chained form of the layer loop: QKV of layer 0 alone, then per layer the attention kernel and ONE launch that
+  // runs O, RMSNorm, gate/up, down and (but for the last layer) the next layer's RMSNorm and QKV.
+  bool chain = false;
+  if (tc && c->chain_on && c->chain_clusters > 0 && c->ksum && !c->cap && f.n_layers > 0 && T_rows <= c->ksum_rows &&
+      T_rows <= CHAIN_MAX_ROWS && c->fuse_rope) {
+    auto two_slab_pair = [](const GemmPlan &p) { return p.cta_group == 2 && p.slabs == 2 && !p.k_interleave; };
+    chain = two_slab_pair(c->pl_qkv) && two_slab_pair(c->pl_o) && two_slab_pair(c->pl_gu) && two_slab_pair(c->pl_down) &&
+            c->tcw_qkv > 0 && c->tcw_o > 0 && c->tcw_h > 0 && c->tcw_down > 0 &&
+            c->tail_qkv >= 0 && c->tail_o >= 0 && c->tail_h >= 0 && c->tail_down >= 0;
+  }
+  // the projections of layer l as steps of a chained launch (with the maps of their tail tiles)
+  auto chain_gemm = [&](int which, int l) {
+    ChainStep st{};
+    switch (which) {
+      case 0: st.g = make_gemm_args(c, EPI_QKV_ROPE, &c->ta_n, &c->tb_qkv[l], nullptr, &c->tc_qkv, qkv, T_rows, 3 * hd, d, c->pl_qkv);
+              st.g.c_tail = c->tail_qkv > 0 ? &c->tct_qkv : nullptr; st.g.tail_cols = c->tail_qkv; break;
+      case 1: st.g = make_gemm_args(c, EPI_RESIDUAL, &c->ta_att, &c->tb_o[l], nullptr, &c->tc_o, c->x, T_rows, d, hd, c->pl_o);
+              st.g.c_tail = c->tail_o > 0 ? &c->tct_o : nullptr; st.g.tail_cols = c->tail_o; break;
+      case 2: st.g = make_gemm_args(c, EPI_SWIGLU, &c->ta_n, &c->tb_gate[l], &c->tb_up[l], &c->tc_h, hbuf, T_rows, F, d, c->pl_gu);
+              st.g.c_tail = c->tail_h > 0 ? &c->tct_h : nullptr; st.g.tail_cols = c->tail_h; break;
+      default: st.g = make_gemm_args(c, EPI_RESIDUAL, &c->ta_h, &c->tb_down[l], nullptr, &c->tc_down, c->x, T_rows, d, F, c->pl_down);
+              st.g.c_tail = c->tail_down > 0 ? &c->tct_down : nullptr; st.g.tail_cols = c->tail_down; break;
+    }
+    return st;
+  };
+  if (chain)
+    for (int i = 0; i < 4; ++i) chain = chain && chain_step_supported(chain_gemm(i, 0));
+  if (chain) {
+    const int ks_o = effective_k_splits(hd, c->pl_o.k_splits), ks_d = effective_k_splits(F, c->pl_down.k_splits);
+    const int64_t ks_stride = (int64_t)round_up(T_rows, 512) * d;
+    const int n_ctas = 2 * c->chain_clusters;
+    const size_t tab_bytes = chain_table_bytes();
+    if (c->chain_tab_rows != T_rows) {
+      // the tables of this row count: launch 0 = QKV of layer 0; launch l + 1 = O, RMSNorm, gate/up, down of layer l and,
+      // but for the last layer, RMSNorm and QKV of layer l + 1
+      auto norm_step = [&](const float *gain, int n_part) {
+        ChainStep st{};
+        st.is_norm = 1;
+        st.nm.x = c->x; st.nm.gain = gain; st.nm.eps = f.rms_eps; st.nm.n = (bf16 *)n; st.nm.rows = T_rows; st.nm.d = d;
+        st.nm.part = c->ksum; st.nm.n_part = n_part > 1 ? n_part : 0; st.nm.part_stride = ks_stride;
+        return st;
+      };
+      c->chain_tab_rows = -1;
+      c->chain_info.assign(f.n_layers + 1, ChainTableInfo{});
+      for (int L = 0; L <= f.n_layers; ++L) {
+        ChainStep st[6] = {};
+        int k = 0;
+        if (L == 0) {
+          st[k++] = chain_gemm(0, 0);
+        } else {
+          const int l = L - 1;
+          st[k++] = chain_gemm(1, l);
+          st[k++] = norm_step(c->norm2[l], ks_o);
+          st[k++] = chain_gemm(2, l);
+          st[k++] = chain_gemm(3, l);
+          if (l + 1 < f.n_layers) {
+            st[k++] = norm_step(c->norm1[l + 1], ks_d);
+            st[k++] = chain_gemm(0, l + 1);
+          }
+        }
+        cudaError_t e = chain_build_table(st, k, c->d_chain_bar, c->d_status, c->h_chain_tabs + (size_t)L * tab_bytes, &c->chain_info[L]);
+        if (e != cudaSuccess) return set_err(c, L2PD_ERR_CUDA, "chained launch table %d: %s", L, cudaGetErrorString(e));
+      }
+      CK(cudaMemcpyAsync(c->d_chain_tabs, c->h_chain_tabs, (size_t)(f.n_layers + 1) * tab_bytes, cudaMemcpyHostToDevice, s));
+      c->chain_tab_rows = T_rows;
+    }
+    auto launch_chain = [&](int L) -> l2pd_status {
+      unsigned long long *tr = nullptr;
+      if (c->d_chain_trace && (int64_t)(L + 1) * CHAIN_TRACE_PHASES * CHAIN_TRACE_STAMPS * n_ctas <= c->chain_trace_cap)
+        tr = c->d_chain_trace + (int64_t)L * CHAIN_TRACE_PHASES * CHAIN_TRACE_STAMPS * n_ctas;
+      CKLK(L2PD_K_CHAIN, launch_gemm_chain(s, c->d_chain_tabs + (size_t)L * tab_bytes, c->chain_info[L], c->chain_clusters, &c->chain_bar_base, tr));
+      return L2PD_OK;
+    };
+    { l2pd_status r = launch_chain(0); if (r) return r; }
+    for (int l = 0; l < f.n_layers; ++l) {
+      CKLK(L2PD_K_ATTENTION, launch_attention_tc(s, c->tq_packed, c->tk_packed, c->tv_packed, c->d_meta, (bf16 *)att, hd, 0, 0, 1,
+                                n_slots, max_q_rows, H, c->d_status));
+      l2pd_status r = launch_chain(l + 1);
+      if (r) return r;
+    }
+    if (ks_d > 1) CKLK(L2PD_K_OTHER, launch_add_partials(s, c->x, c->ksum, ks_d, ks_stride, T_rows, d));
+    c->chain_trace_launches = f.n_layers + 1; c->chain_trace_phases = CHAIN_TRACE_PHASES; c->chain_trace_ctas = n_ctas;
+  }
+
+  for (int l = 0; l < f.n_layers && !chain; ++l) {
     T *kc = (T *)c->kc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
     T *vc = (T *)c->vc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
     l2pd_status r;
@@ -400,6 +527,8 @@ void free_all(l2pd_ctx *c) {
   cudaFree(c->kc); cudaFree(c->vc); cudaFree(c->part); cudaFree(c->logits_f32);
   for (void *w : c->wqkv_perm) cudaFree(w);
   cudaFree(c->d_row_pos); cudaFree(c->cs_table_t); cudaFree(c->ksum);
+  cudaFree(c->d_chain_bar); cudaFree(c->d_chain_trace); cudaFree(c->d_chain_tabs);
+  if (c->h_chain_tabs) cudaFreeHost(c->h_chain_tabs);
   cudaFree(c->d_meta); cudaFree(c->d_row_slot); cudaFree(c->d_summary); cudaFree(c->d_status); cudaFree(c->cs_table);
   if (c->h_meta) cudaFreeHost(c->h_meta);
   if (c->h_summary) cudaFreeHost(c->h_summary);
@@ -509,6 +638,14 @@ l2pd_status l2pd_init(const l2pd_config *cfg, const l2pd_weights *w, int device,
     c->ksum_rows = round_up(mr < 4096 ? mr : 4096, 512);   // a slice's area covers whole 512-row units
     A(dev_alloc(c, &c->ksum, 4 * c->ksum_rows * d));
   }
+  if (f.dtype == L2PD_BF16 && c->ksum && !c->force_simt) {
+    c->chain_clusters = chain_max_clusters(c->num_sms);
+    if (c->chain_clusters > 0) {
+      A(dev_alloc(c, &c->d_chain_bar, (int64_t)1));
+      A(dev_alloc(c, &c->d_chain_tabs, (int64_t)(f.n_layers + 1) * (int64_t)chain_table_bytes()));
+      if (r == L2PD_OK && cudaMallocHost((void **)&c->h_chain_tabs, (size_t)(f.n_layers + 1) * chain_table_bytes()) != cudaSuccess) r = L2PD_ERR_OOM;
+    }
+  }
   A(dev_alloc(c, &c->d_summary, (int64_t)f.max_batch));
   A(dev_alloc(c, &c->d_status, (int64_t)1));
   A(dev_alloc(c, &c->cs_table, (int64_t)f.max_seq * (f.head_dim / 2)));
@@ -518,6 +655,7 @@ l2pd_status l2pd_init(const l2pd_config *cfg, const l2pd_weights *w, int device,
       cudaMallocHost((void **)&c->h_status, sizeof(int32_t)) != cudaSuccess)
     return fail(L2PD_ERR_OOM);
   if (cudaMemset(c->d_status, 0, 4) != cudaSuccess) return fail(L2PD_ERR_CUDA);
+  if (c->d_chain_bar && cudaMemset(c->d_chain_bar, 0, 4) != cudaSuccess) return fail(L2PD_ERR_CUDA);
   // the activation buffers back TMA boxes that reach past the live rows: start them defined
   if (cudaMemset(c->n, 0, mr * d * es) != cudaSuccess || cudaMemset(c->att, 0, mr * hd * es) != cudaSuccess ||
       cudaMemset(c->h, 0, mr * F * es) != cudaSuccess || cudaMemset(c->nf, 0, c->max_lm_rows * d * es) != cudaSuccess ||
@@ -655,6 +793,7 @@ l2pd_status l2pd_denoise_step(l2pd_ctx *c, void *stream, const l2pd_step_out *ou
   if (*c->h_status != DEV_OK) {
     const int code = *c->h_status;
     cudaMemsetAsync(c->d_status, 0, 4, s);
+    if (c->d_chain_bar) { cudaMemsetAsync(c->d_chain_bar, 0, 4, s); c->chain_bar_base = 0; }   // the meeting counter stopped short
     return set_err(c, L2PD_ERR_TIMEOUT, "a bounded device wait ran out (role %d)", code);
   }
   c->total_steps++;
@@ -824,6 +963,44 @@ l2pd_status l2pd_profile_read(const l2pd_ctx *c, int32_t kind, double *ms_total,
   return L2PD_OK;
 }
 const char *l2pd_last_error(const l2pd_ctx *c);
+
+l2pd_status l2pd_set_chain(l2pd_ctx *c, int32_t enable) {
+  if (!c) return L2PD_ERR_ARG;
+  c->chain_on = enable != 0;
+  return L2PD_OK;
+}
+
+l2pd_status l2pd_chain_trace_enable(l2pd_ctx *c, int32_t enable) {
+  if (!c) return L2PD_ERR_ARG;
+  CK(cudaSetDevice(c->device));
+  if (!enable) {
+    CK(cudaDeviceSynchronize());
+    cudaFree(c->d_chain_trace);
+    c->d_chain_trace = nullptr; c->chain_trace_cap = 0; c->chain_trace_launches = 0;
+    return L2PD_OK;
+  }
+  if (c->chain_clusters <= 0) return set_err(c, L2PD_ERR_STATE, "this context does not run chained launches");
+  if (!c->d_chain_trace) {
+    const int64_t cap = (int64_t)(c->cfg.n_layers + 1) * CHAIN_TRACE_PHASES * CHAIN_TRACE_STAMPS * (2 * c->chain_clusters);
+    CK(cudaMalloc((void **)&c->d_chain_trace, (size_t)cap * 8));
+    CK(cudaMemset(c->d_chain_trace, 0, (size_t)cap * 8));
+    c->chain_trace_cap = cap;
+  }
+  c->chain_trace_launches = 0;
+  return L2PD_OK;
+}
+
+int64_t l2pd_chain_trace_read(l2pd_ctx *c, uint64_t *h_out, int64_t capacity, int32_t *launches, int32_t *phases, int32_t *ctas) {
+  if (!c || !c->d_chain_trace) return 0;
+  if (launches) *launches = c->chain_trace_launches;
+  if (phases) *phases = c->chain_trace_phases;
+  if (ctas) *ctas = c->chain_trace_ctas;
+  const int64_t n = (int64_t)c->chain_trace_launches * c->chain_trace_phases * CHAIN_TRACE_STAMPS * c->chain_trace_ctas;
+  if (!h_out || capacity < n || n == 0) return n;
+  if (cudaSetDevice(c->device) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(h_out, c->d_chain_trace, (size_t)n * 8, cudaMemcpyDeviceToHost) != cudaSuccess) return -1;
+  return n;
+}
 
 void l2pd_destroy(l2pd_ctx *c) {
   if (!c) return;

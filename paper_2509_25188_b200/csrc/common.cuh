@@ -158,6 +158,8 @@ l2pd_status make_tma_2d_bf16_strided(TmaDesc *out, const void *ptr, int64_t rows
 // Output of a GEMM as a 3-D tensor [rows][N / tile_w][tile_w] (bf16, or fp32 for the residual stream) with a
 // box of 32 rows x 128 bytes, for the epilogue's staged stores; tile_w = the output columns one tile covers.
 l2pd_status make_tma_out_3d(TmaDesc *out, void *ptr, bool fp32, int64_t rows, int64_t N, int tile_w);
+// The same for the columns [N - tail_w, N) alone, as one tile of width tail_w (rows are N elements apart).
+l2pd_status make_tma_out_tail(TmaDesc *out, void *ptr, bool fp32, int64_t rows, int64_t N, int tail_w);
 int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile);
 // How one GEMM is laid over the SMs: CTAs per tile (1, or 2 = a cta_group::2 pair on a 256-row tile),
 // tile width, K slices (residual epilogue only: slices add into X with vector reductions), and row
@@ -168,12 +170,15 @@ int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile);
 // k_interleave = 1 (single CTA, one slab, few rows): the two MMA-issuing threads take alternate k-blocks of the
 // unit into two accumulators that the epilogue adds — halves the K loop where instruction issue bounds it
 struct GemmPlan { int cta_group, tile_n, k_splits, slabs, k_interleave; };
-GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, int max_k_splits = 4);
+// max_tile_n caps the tile width (a kernel that chains several projections keeps one ring geometry for all of them)
+GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, int max_k_splits = 4, int max_tile_n = 256);
 int effective_k_splits(int K, int k_splits);   // what the launcher makes of a requested K split
 struct GemmArgs {
   int epi;                 // EPI_STORE, EPI_RESIDUAL, EPI_SWIGLU, or EPI_LMHEAD
   const TmaDesc *a, *b, *b2;
   const TmaDesc *c;        // output map from make_tma_out_3d (rows = M, tile_w matching tile_n), or null: direct stores
+  const TmaDesc *c_tail;   // optional (chained launches): map of the row's last, narrower tile alone, from make_tma_out_tail
+  int tail_cols;           // its output columns (a multiple of 16)
   int M, N, K, tile_n;
   int cta_group, k_splits; // 0 / 1 = single CTA, no split
   int slabs;               // 0 / 1 = one row slab per unit, 2 = two
@@ -194,6 +199,29 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
 cudaError_t launch_merge_partials(cudaStream_t st, const float *part_m, const float *part_s,
                                   const int32_t *part_i, int n_tiles, int rows_padded, int R,
                                   int32_t *pred, float *conf);
+
+// gemm_chain.cu : several projections (cta_group 2, two row slabs per unit) and the RMSNorms between them in one
+// persistent launch; the phases run in the order given, the CTAs meeting at a counter in global memory between them.
+struct ChainNorm {        // x += part[0] + part[1] + ... (slice s at part + s * part_stride, in that order), n = RMSNorm(x)
+  float *x; const float *gain; float eps; bf16 *n; int rows, d;
+  const float *part; int n_part; int64_t part_stride;
+};
+struct ChainStep { int is_norm; GemmArgs g; ChainNorm nm; };
+// CTA pairs of the chain kernel that can be resident at once on the current device (0: the kernel cannot run)
+int chain_max_clusters(int num_sms);
+bool chain_step_supported(const ChainStep &s);
+// A launch runs from a table in device memory: chain_build_table fills the host image (chain_table_bytes() bytes,
+// 128-byte aligned) for up to 6 steps holding at most 4 projections, the first step being a projection; the caller
+// copies it to the device once and reuses it for every launch of the same steps.  bar: device counter, zero before
+// its first use, shared by all tables of a stream; status: device status word.
+struct ChainTableInfo { int n_phases, n_stages; size_t smem_bytes; };
+size_t chain_table_bytes();
+cudaError_t chain_build_table(const ChainStep *steps, int n_steps, unsigned int *bar, int32_t *status, void *h_table,
+                              ChainTableInfo *info);
+// *bar_base: host copy of the counter's value before this launch, advanced here.  trace: optional device array
+// [n_phases][4][2 * n_clusters] of nanosecond stamps (per CTA: phase opened, first and last accumulator ready, phase finished).
+cudaError_t launch_gemm_chain(cudaStream_t st, const void *d_table, const ChainTableInfo &info, int n_clusters,
+                              unsigned int *bar_base, unsigned long long *trace);
 
 // attention.cu
 cudaError_t launch_attention_bf16(cudaStream_t st, const bf16 *q, const bf16 *kc, const bf16 *vc,

@@ -29,378 +29,14 @@
 #include <stdio.h>
 
 #include "common.cuh"
+#include "gemm_device.cuh"
 #include "ptx.cuh"
 
 namespace l2pd {
 
+using namespace gemm_dev;
+
 namespace {
-
-constexpr int TILE_M = 128;
-constexpr int TILE_K = 64;                       // 64 bf16 = 128 bytes = one swizzle row
-constexpr int A_STAGE_BYTES = TILE_M * TILE_K * 2;
-constexpr int MAX_STAGES = 8;
-constexpr int TMEM_COLS = 512;
-constexpr int ACC_COLS = 256;                    // columns per accumulator buffer
-constexpr int SMEM_BUDGET = 227 * 1024;
-
-struct KParams {
-  int M, N, K, tile_n, n_stages, b_stage_bytes;
-  int slabs, a_stage_bytes;         // row slabs (of 128 * CG rows) one unit covers: 1, or 2 = accumulators not double-buffered
-  int m_tiles, n_tiles, k_splits;   // m_tiles counts row tiles of 128 * CG * slabs rows
-  int group_m;                      // row tiles per raster group (see the unit order in gemm_body)
-  void *out;
-  const float *bias;
-  float *part_m, *part_s;
-  int32_t *part_i;
-  int rows_padded;
-  float *logits;
-  int32_t *status;
-  int out_tma;          // 1: the epilogue may stage its output in shared memory and store it through tmC
-  int out_full_tiles;   // column tiles that lie wholly inside the row (the others use direct stores)
-  int gate;             // 1: every unit's epilogue is staged; the producer keeps off the staging area meanwhile
-  float *part; int part_rows;      // EPI_RESIDUAL with K slices: slice s stores its partial sums at part[s * part_rows + row][N]
-  int rope_cols, rope_dh, cs_stride;   // EPI_QKV_ROPE, see GemmArgs
-  const float2 *cs_table;
-  const int32_t *row_pos;
-  int kil;   // 1: the unit's k-blocks alternate between the two MMA issuers (accumulators 0 and 1, added in the epilogue)
-};
-
-__device__ __forceinline__ void fail(int32_t *status, int code) {
-  if (status) atomicCAS(status, 0, code);
-}
-
-// silu(g) * u with the fast exponential and division (a few ulp, far below the bf16 rounding of the result)
-__device__ __forceinline__ float silu_mul(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
-
-// Emitters: what the epilogue does with 16 consecutive accumulator columns of one row.
-// `valid` = columns left in the row from the first of the 16 (the row length is a multiple of 8).
-__device__ __forceinline__ void emit_store16(bf16 *dst, const uint32_t *v, int valid) {   // 16 fp32 -> 16 bf16, 32 bytes
-#pragma unroll
-  for (int hseg = 0; hseg < 2; ++hseg) {
-    if (hseg * 8 >= valid) break;
-    uint4 pk;
-    uint32_t *pw = reinterpret_cast<uint32_t *>(&pk);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(v[hseg * 8 + 2 * i]), __uint_as_float(v[hseg * 8 + 2 * i + 1]));
-      pw[i] = *reinterpret_cast<uint32_t *>(&t);
-    }
-    *reinterpret_cast<uint4 *>(dst + hseg * 8) = pk;
-  }
-}
-// mode 0: x += acc (read-modify-write), 1: atomic x += acc, 2: plain store (a K slice's partial sums)
-__device__ __forceinline__ void emit_residual16(float *px, const uint32_t *v, int mode, int valid) {
-#pragma unroll
-  for (int g = 0; g < 4; ++g) {
-    if (g * 4 >= valid) break;
-    if (mode == 2) {
-      *reinterpret_cast<float4 *>(px + 4 * g) = make_float4(__uint_as_float(v[4 * g + 0]), __uint_as_float(v[4 * g + 1]),
-                                                            __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3]));
-    } else if (mode == 1) {
-      ptx::red_add_v4(px + 4 * g, __uint_as_float(v[4 * g + 0]), __uint_as_float(v[4 * g + 1]),
-                      __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3]));
-    } else {
-      float4 x = *reinterpret_cast<float4 *>(px + 4 * g);
-      x.x += __uint_as_float(v[4 * g + 0]);
-      x.y += __uint_as_float(v[4 * g + 1]);
-      x.z += __uint_as_float(v[4 * g + 2]);
-      x.w += __uint_as_float(v[4 * g + 3]);
-      *reinterpret_cast<float4 *>(px + 4 * g) = x;
-    }
-  }
-}
-__device__ __forceinline__ void emit_swiglu16(bf16 *dst, const uint32_t *g, const uint32_t *u, int valid) {
-#pragma unroll
-  for (int hseg = 0; hseg < 2; ++hseg) {
-    if (hseg * 8 >= valid) break;
-    uint4 pk;
-    uint32_t *pw = reinterpret_cast<uint32_t *>(&pk);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float g0 = __uint_as_float(g[hseg * 8 + 2 * i]), g1 = __uint_as_float(g[hseg * 8 + 2 * i + 1]);
-      const float u0 = __uint_as_float(u[hseg * 8 + 2 * i]), u1 = __uint_as_float(u[hseg * 8 + 2 * i + 1]);
-      __nv_bfloat162 t = __floats2bfloat162_rn(silu_mul(g0, u0), silu_mul(g1, u1));
-      pw[i] = *reinterpret_cast<uint32_t *>(&t);
-    }
-    *reinterpret_cast<uint4 *>(dst + hseg * 8) = pk;
-  }
-}
-
-// Rotary embedding on 32 (or 16) consecutive accumulator columns of one row, starting at the even column col0:
-// the pair (x1, x2) = columns (2t, 2t + 1) becomes (x1 cos - x2 sin, x2 cos + x1 sin), the angle being that of
-// pair index ((column % dh) / 2) at position pos.  Columns from rope_cols on (the v part) are left alone.
-__device__ __forceinline__ void rope_pairs(const KParams &p, uint32_t *v, int col0, int ncols, int pos) {
-  if (col0 >= p.rope_cols) return;               // a chunk of v columns (warp-uniform)
-  // the table is laid out [pair][position]: the 32 rows of a warp are consecutive positions, so a load is one line.
-  // All 16 angles are fetched before any is used.
-  const float2 *cs = p.cs_table + pos;
-  const int mask = p.rope_dh - 1;
-  float2 a[16];
-#pragma unroll
-  for (int t = 0; t < 16; ++t) a[t] = __ldg(cs + (int64_t)(((col0 + 2 * t) & mask) >> 1) * p.cs_stride);
-#pragma unroll
-  for (int t = 0; t < 16; ++t) {
-    if (2 * t < ncols && col0 + 2 * t < p.rope_cols) {
-      const float x1 = __uint_as_float(v[2 * t]), x2 = __uint_as_float(v[2 * t + 1]);
-      v[2 * t] = __float_as_uint(x1 * a[t].x - x2 * a[t].y);
-      v[2 * t + 1] = __float_as_uint(x2 * a[t].x + x1 * a[t].y);
-    }
-  }
-}
-
-// Drains one 128-row x tile_n accumulator from tensor memory (this warp's 32 lanes) and applies the
-// epilogue with per-thread stores (a thread owns one row).  The loads run one step ahead of the
-// arithmetic and stores: while chunk c is converted and written, chunk c + 1 is in flight
-// (tcgen05.wait::ld covers every load issued so far).
-// K slices of the residual epilogue either add into X (`res_mode` 1) or store their partial sums to
-// `res_base`, the slice's own [rows][N] area (`res_mode` 2), for a later fixed-order sum.
-template <int EPI>
-// two_acc: the unit's sum is spread over two accumulators (ACC_COLS columns apart), added here.
-__device__ __forceinline__ void drain_tile(const KParams &p, uint32_t taddr, int row, int nt, int res_mode, float *res_base,
-                                           bool two_acc = false) {
-  const bool row_ok = row < p.M;
-  const int half_n = p.tile_n >> 1;
-  if (EPI == EPI_STORE || EPI == EPI_RESIDUAL || EPI == EPI_QKV_ROPE) {
-    const int pos = (EPI == EPI_QKV_ROPE && row_ok) ? p.row_pos[row] : 0;
-    // 32 columns per step (tile_n is a multiple of 16: the last step may hold 16)
-    const int n0 = nt * p.tile_n, n = p.tile_n;
-    uint32_t va[32], vb[32];
-    auto load = [&](uint32_t *v, int c) {
-      if (n - c >= 32) ptx::tmem_ld_x32(taddr + c, v);
-      else ptx::tmem_ld_x16(taddr + c, v);
-    };
-    auto emit = [&](uint32_t *v, int c) {
-      if (!row_ok) return;
-      if (EPI == EPI_QKV_ROPE) rope_pairs(p, v, n0 + c, min(32, n - c), pos);
-#pragma unroll
-      for (int h16 = 0; h16 < 2; ++h16) {
-        const int col = n0 + c + 16 * h16;
-        if (c + 16 * h16 < n && col < p.N) {
-          if (EPI != EPI_RESIDUAL) emit_store16(reinterpret_cast<bf16 *>(p.out) + (int64_t)row * p.N + col, v + 16 * h16, p.N - col);
-          else emit_residual16(res_base + (int64_t)row * p.N + col, v + 16 * h16, res_mode, p.N - col);
-        }
-      }
-    };
-    if (two_acc) {
-      for (int c = 0; c < n; c += 32) {
-        load(va, c);
-        if (n - c >= 32) ptx::tmem_ld_x32(taddr + ACC_COLS + c, vb);
-        else ptx::tmem_ld_x16(taddr + ACC_COLS + c, vb);
-        ptx::tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 32; ++i) va[i] = __float_as_uint(__uint_as_float(va[i]) + __uint_as_float(vb[i]));
-        emit(va, c);
-      }
-      return;
-    }
-    load(va, 0);
-    for (int c = 0; c < n; c += 64) {
-      ptx::tmem_ld_wait();
-      if (c + 32 < n) load(vb, c + 32);
-      emit(va, c);
-      if (c + 32 >= n) break;
-      ptx::tmem_ld_wait();
-      if (c + 64 < n) load(va, c + 64);
-      emit(vb, c + 32);
-    }
-  } else if (EPI == EPI_SWIGLU) {
-    bf16 *H = reinterpret_cast<bf16 *>(p.out);
-    const int n0 = nt * half_n;
-    uint32_t ga[16], ua[16], gb[16], ub[16];
-    auto load = [&](uint32_t *g, uint32_t *u, int c) {
-      ptx::tmem_ld_x16(taddr + c, g);
-      ptx::tmem_ld_x16(taddr + half_n + c, u);
-    };
-    auto emit = [&](const uint32_t *g, const uint32_t *u, int c) {
-      if (row_ok && n0 + c < p.N) emit_swiglu16(H + (int64_t)row * p.N + n0 + c, g, u, min(p.N - n0 - c, half_n - c));
-    };
-    if (two_acc) {
-      for (int c = 0; c < half_n; c += 16) {
-        load(ga, ua, c);
-        ptx::tmem_ld_x16(taddr + ACC_COLS + c, gb);
-        ptx::tmem_ld_x16(taddr + ACC_COLS + half_n + c, ub);
-        ptx::tmem_ld_wait();
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          ga[i] = __float_as_uint(__uint_as_float(ga[i]) + __uint_as_float(gb[i]));
-          ua[i] = __float_as_uint(__uint_as_float(ua[i]) + __uint_as_float(ub[i]));
-        }
-        emit(ga, ua, c);
-      }
-      return;
-    }
-    load(ga, ua, 0);
-    for (int c = 0; c < half_n; c += 32) {
-      ptx::tmem_ld_wait();
-      if (c + 16 < half_n) load(gb, ub, c + 16);
-      emit(ga, ua, c);
-      if (c + 16 >= half_n) break;
-      ptx::tmem_ld_wait();
-      if (c + 32 < half_n) load(ga, ua, c + 32);
-      emit(gb, ub, c + 16);
-    }
-  } else {  // EPI_LMHEAD
-    uint32_t v[16];
-    const float L2E = 1.4426950408889634f;
-    const int n0 = nt * p.tile_n;
-    float m_run = -INFINITY, s_run = 0.f;
-    int i_run = 0x7fffffff;
-    for (int c = 0; c < p.tile_n; c += 16) {
-      ptx::tmem_ld_x16(taddr + c, v);
-      ptx::tmem_ld_wait();
-      if (row_ok && n0 + c < p.N) {
-        float f[16];
-        float cm = -INFINITY;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) {
-          const int col = n0 + c + i;
-          float val = __uint_as_float(v[i]);
-          if (col < p.N) { if (p.bias) val += __ldg(p.bias + col); }
-          else val = -INFINITY;
-          f[i] = val;
-          cm = fmaxf(cm, val);
-        }
-        if (p.logits) {
-#pragma unroll
-          for (int i = 0; i < 16; ++i)
-            if (n0 + c + i < p.N) p.logits[(int64_t)row * p.N + n0 + c + i] = f[i];
-        }
-        if (cm > m_run) {
-          s_run *= exp2f((m_run - cm) * L2E);
-          m_run = cm;
-          int ci = 0;
-#pragma unroll
-          for (int i = 15; i >= 0; --i) if (f[i] == cm) ci = i;   // lowest index holding the max
-          i_run = n0 + c + ci;
-        }
-        float add = 0.f;
-#pragma unroll
-        for (int i = 0; i < 16; ++i) add += exp2f((f[i] - m_run) * L2E);
-        s_run += add;
-      }
-    }
-    if (row_ok) {
-      const int64_t o = (int64_t)nt * p.rows_padded + row;
-      p.part_m[o] = m_run;
-      p.part_s[o] = s_run;
-      p.part_i[o] = i_run;
-    }
-  }
-}
-
-// The same through shared memory and TMA: a thread owns one accumulator row, so direct stores touch
-// 32 different lines per instruction; instead each warp lays 128 bytes of 32 rows into a swizzled
-// staging tile (4 KB) and one thread hands it to the TMA unit, which writes whole lines (bf16
-// outputs) or adds them into X in L2 (fp32 residual).  The output tensor map is 3-D
-// [rows][column tile][column in tile], so a box that runs past the tile's width is clipped there,
-// and rows beyond M are clipped by the map's row count.
-// The warp's STAGE_BUFS staging tiles lie over the A operands of the ring's last two stages and are
-// used in turn.  That memory is idle during a CTA's last unit; for earlier units (two-slab units,
-// whose drain is not overlapped anyway) the producer refills those two stages only after the
-// epilogue warps have reported the staging area free.
-constexpr int STAGE_BUFS = 2;
-template <int EPI>
-__device__ __forceinline__ void drain_tile_staged(const KParams &p, const CUtensorMap *tmC, uint32_t taddr, int row0,
-                                                  int nt, uint32_t stage0, int lane, bool res_store) {
-  const int half_n = p.tile_n >> 1;
-  const uint32_t sw = (uint32_t)(lane & 7);
-  int n_flush = 0;                       // staging tiles handed over so far; the current one is n_flush % STAGE_BUFS
-  uint32_t stage = stage0;
-  auto chunk_addr = [&](int ch) { return stage + lane * 128 + (((uint32_t)ch ^ sw) << 4); };
-  auto st16 = [&](uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-  };
-  auto flush = [&](int c0) {   // hand the staged 32 x 128-byte tile to the TMA unit
-    ptx::fence_proxy_async();
-    __syncwarp();
-    if (lane == 0) {
-      if (EPI == EPI_RESIDUAL && !res_store) ptx::tma_reduce_add_3d(tmC, stage, c0, nt, row0);
-      else ptx::tma_store_3d(tmC, stage, c0, nt, row0);
-      ptx::bulk_commit();
-    }
-    ++n_flush;
-  };
-  auto reuse = [&]() {         // pick the next staging tile; the flush that used it STAGE_BUFS turns ago has read it
-    stage = stage0 + (uint32_t)(n_flush % STAGE_BUFS) * 4096u;
-    if (n_flush >= STAGE_BUFS) {
-      if (lane == 0) ptx::bulk_wait_read_n<STAGE_BUFS - 1>();
-      __syncwarp();
-    }
-  };
-  auto pack2 = [](uint32_t a, uint32_t b) {
-    __nv_bfloat162 t = __floats2bfloat162_rn(__uint_as_float(a), __uint_as_float(b));
-    return *reinterpret_cast<uint32_t *>(&t);
-  };
-  if (EPI == EPI_STORE || EPI == EPI_RESIDUAL || EPI == EPI_QKV_ROPE) {
-    const int n = p.tile_n;
-    const int pos = (EPI == EPI_QKV_ROPE && row0 + lane < p.M) ? p.row_pos[row0 + lane] : 0;
-    uint32_t va[32], vb[32];
-    auto load = [&](uint32_t *v, int c) {
-      if (n - c >= 32) ptx::tmem_ld_x32(taddr + c, v);
-      else ptx::tmem_ld_x16(taddr + c, v);
-    };
-    auto emit = [&](uint32_t *v, int c) {   // 32 columns starting at c (the upper 16 may lie beyond the tile)
-      if (EPI == EPI_QKV_ROPE) rope_pairs(p, v, nt * n + c, min(32, n - c), pos);
-      if (EPI == EPI_RESIDUAL) {
-        reuse();
-#pragma unroll
-        for (int ch = 0; ch < 8; ++ch) st16(chunk_addr(ch), v[4 * ch], v[4 * ch + 1], v[4 * ch + 2], v[4 * ch + 3]);
-        flush(c);
-      } else {
-        const int hb = (c >> 5) & 1;              // which 64-byte half of the 128-byte staging row
-        if (hb == 0) reuse();
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch)
-          st16(chunk_addr(hb * 4 + ch), pack2(v[8 * ch], v[8 * ch + 1]), pack2(v[8 * ch + 2], v[8 * ch + 3]),
-               pack2(v[8 * ch + 4], v[8 * ch + 5]), pack2(v[8 * ch + 6], v[8 * ch + 7]));
-        if (hb == 1 || c + 32 >= n) flush(c & ~63);
-      }
-    };
-    load(va, 0);
-    for (int c = 0; c < n; c += 64) {
-      ptx::tmem_ld_wait();
-      if (c + 32 < n) load(vb, c + 32);
-      emit(va, c);
-      if (c + 32 >= n) break;
-      ptx::tmem_ld_wait();
-      if (c + 64 < n) load(va, c + 64);
-      emit(vb, c + 32);
-    }
-  } else {   // EPI_SWIGLU: 16 gate + 16 up columns give 16 outputs = 32 bytes of the staging row
-    uint32_t ga[16], ua[16], gb[16], ub[16];
-    auto load = [&](uint32_t *g, uint32_t *u, int c) {
-      ptx::tmem_ld_x16(taddr + c, g);
-      ptx::tmem_ld_x16(taddr + half_n + c, u);
-    };
-    auto emit = [&](const uint32_t *g, const uint32_t *u, int c) {
-      const int qb = (c >> 4) & 3;                // which 32-byte quarter of the staging row
-      if (qb == 0) reuse();
-#pragma unroll
-      for (int hseg = 0; hseg < 2; ++hseg) {
-        uint32_t pw[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const float g0 = __uint_as_float(g[hseg * 8 + 2 * i]), g1 = __uint_as_float(g[hseg * 8 + 2 * i + 1]);
-          const float u0 = __uint_as_float(u[hseg * 8 + 2 * i]), u1 = __uint_as_float(u[hseg * 8 + 2 * i + 1]);
-          __nv_bfloat162 t = __floats2bfloat162_rn(silu_mul(g0, u0), silu_mul(g1, u1));
-          pw[i] = *reinterpret_cast<uint32_t *>(&t);
-        }
-        st16(chunk_addr(qb * 2 + hseg), pw[0], pw[1], pw[2], pw[3]);
-      }
-      if (qb == 3 || c + 16 >= half_n) flush(c & ~63);
-    };
-    load(ga, ua, 0);
-    for (int c = 0; c < half_n; c += 32) {
-      ptx::tmem_ld_wait();
-      if (c + 16 < half_n) load(gb, ub, c + 16);
-      emit(ga, ua, c);
-      if (c + 16 >= half_n) break;
-      ptx::tmem_ld_wait();
-      if (c + 32 < half_n) load(ga, ua, c + 32);
-      emit(gb, ub, c + 16);
-    }
-  }
-}
 
 // CG = 1: one CTA per 128 x tile_n output tile.
 // CG = 2: a cluster of two CTAs per 256 x tile_n tile (cta_group::2).  CTA r loads A rows
@@ -807,6 +443,23 @@ l2pd_status make_tma_out_3d(TmaDesc *out, void *ptr, bool fp32, int64_t rows, in
   return r == CUDA_SUCCESS ? L2PD_OK : L2PD_ERR_CUDA;
 }
 
+l2pd_status make_tma_out_tail(TmaDesc *out, void *ptr, bool fp32, int64_t rows, int64_t N, int tail_w) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return L2PD_ERR_CUDA;
+  const int es = fp32 ? 4 : 2;
+  if (tail_w < 1 || tail_w >= N || ((tail_w * es) % 16) || ((N * es) % 16) || rows < 1) return L2PD_ERR_SHAPE;
+  uint8_t *base = reinterpret_cast<uint8_t *>(ptr) + (N - tail_w) * es;
+  if (reinterpret_cast<uintptr_t>(base) & 15) return L2PD_ERR_SHAPE;
+  cuuint64_t dims[3] = {(cuuint64_t)tail_w, 1, (cuuint64_t)rows};
+  cuuint64_t strides[2] = {(cuuint64_t)N * es, (cuuint64_t)N * es};
+  cuuint32_t box[3] = {(cuuint32_t)(128 / es), 1, 32};
+  cuuint32_t estr[3] = {1, 1, 1};
+  CUresult r = fn(&out->map, fp32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, base, dims,
+                  strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                  CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? L2PD_OK : L2PD_ERR_CUDA;
+}
+
 // Modelled cycles of one GEMM for a tile width / K split / slab count.  Per 64-deep k-block a CTA
 // needs the largest of: the tensor pipe's 2 * tile_n cycles per slab; the ~620 cycles one thread
 // takes to issue its four MMAs and the stage hand-over; the bytes it must take in at INGEST bytes
@@ -830,7 +483,7 @@ static double plan_cost(int M, int N, int K, int num_sms, int cg, int slabs, int
   return waves * (kb * per_kb + 6000.0 + exposed) + (slabs == 2 ? 0.0 : 0.7 * drain);
 }
 
-GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, int max_k_splits) {
+GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, int max_k_splits, int max_tile_n) {
   GemmPlan best{1, 256, 1, 1, 0};
   double best_cost = 1e300;
   const bool swiglu = epi == EPI_SWIGLU;
@@ -842,6 +495,7 @@ GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, 
       if (slabs == 2 && (cg == 1 || epi == EPI_LMHEAD || M <= TILE_M * cg)) continue;
       for (int tn = 256; tn >= 64; tn -= step) {
         if (force_tile_n && tn != force_tile_n) continue;
+        if (!force_tile_n && tn > max_tile_n) continue;
         const int unit_n = swiglu ? tn / 2 : tn;
         const int max_ks = (epi == EPI_RESIDUAL) ? (max_k_splits < 4 ? max_k_splits : 4) : 1;
         for (int ks = 1; ks <= max_ks; ++ks) {
@@ -871,29 +525,38 @@ int effective_k_splits(int K, int k_splits) {
   return ks;
 }
 
-cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms) {
+// Fills the kernel's parameter block for one GEMM.  stages / b_stage_bytes = 0: the deepest ring the shared
+// memory holds for this tile; otherwise the given ring geometry (a kernel that runs several GEMMs keeps one ring).
+cudaError_t fill_kparams(const GemmArgs &g, int stages, int b_stage_bytes, KParams &p) {
   const int cg = g.cta_group == 2 ? 2 : 1;
   if (g.k_splits > 1 && g.epi != EPI_RESIDUAL) return cudaErrorInvalidValue;
   const int ks = effective_k_splits(g.K, g.k_splits);
-  KParams p;
   p.M = g.M; p.N = g.N; p.K = g.K; p.tile_n = g.tile_n;
-  p.b_stage_bytes = g.tile_n * 128 / cg;
+  p.b_stage_bytes = b_stage_bytes > 0 ? b_stage_bytes : g.tile_n * 128 / cg;
+  if (p.b_stage_bytes < g.tile_n * 128 / cg) return cudaErrorInvalidValue;
   p.slabs = g.slabs == 2 ? 2 : 1;
   if (p.slabs == 2 && g.epi == EPI_LMHEAD) return cudaErrorInvalidValue;
   p.a_stage_bytes = p.slabs * A_STAGE_BYTES;
   const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
-  int stages = (SMEM_BUDGET - 2048) / stage_bytes;
-  if (stages > MAX_STAGES) stages = MAX_STAGES;
-  if (g.k_interleave) stages &= ~1;   // alternate k-blocks <-> alternate stages
-  if (stages < 2) return cudaErrorInvalidValue;
+  if (stages <= 0) {
+    stages = (SMEM_BUDGET - 2048) / stage_bytes;
+    if (stages > MAX_STAGES) stages = MAX_STAGES;
+    if (g.k_interleave) stages &= ~1;   // alternate k-blocks <-> alternate stages
+  }
+  if (stages < 2 || stages > MAX_STAGES || (size_t)stages * stage_bytes + 2048 > (size_t)SMEM_BUDGET) return cudaErrorInvalidValue;
   p.n_stages = stages;
   p.m_tiles = ceil_div(g.M, TILE_M * cg * p.slabs);
   const int n_per_tile = (g.epi == EPI_SWIGLU) ? g.tile_n / 2 : g.tile_n;
   // staged output: needs the output map and a staging area (the A part of the ring's last two stages)
   p.kil = g.k_interleave ? 1 : 0;
-  if (p.kil && (p.slabs != 1 || g.epi == EPI_LMHEAD)) return cudaErrorInvalidValue;
+  if (p.kil && (p.slabs != 1 || g.epi == EPI_LMHEAD || (stages & 1))) return cudaErrorInvalidValue;
   p.out_tma = (g.c != nullptr && g.epi != EPI_LMHEAD && stages >= 3 && !p.kil) ? 1 : 0;   // (the two-accumulator sum lives in the direct-store drain)
   p.out_full_tiles = p.out_tma ? g.N / n_per_tile : 0;
+  p.out_tail_cols = 0;
+  if (p.out_tma && g.c_tail && g.tail_cols > 0) {
+    if (g.tail_cols != g.N - p.out_full_tiles * n_per_tile || (g.tail_cols % (g.epi == EPI_SWIGLU ? 8 : 16))) return cudaErrorInvalidValue;
+    p.out_tail_cols = g.tail_cols;
+  }
   p.gate = (p.out_tma && p.slabs == 2 && stages >= 4) ? 1 : 0;
   p.n_tiles = ceil_div(g.N, n_per_tile);
   p.k_splits = ks;
@@ -908,6 +571,17 @@ cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms)
   p.rope_cols = g.rope_cols; p.rope_dh = g.rope_dh; p.cs_stride = g.cs_stride; p.cs_table = g.cs_table; p.row_pos = g.row_pos;
   if (g.epi == EPI_QKV_ROPE && (!g.cs_table || !g.row_pos || g.rope_dh < 2 || (g.rope_dh & (g.rope_dh - 1)) || (g.rope_cols % g.rope_dh)))
     return cudaErrorInvalidValue;
+  return cudaSuccess;
+}
+
+cudaError_t launch_gemm_tcgen05(cudaStream_t st, const GemmArgs &g, int num_sms) {
+  const int cg = g.cta_group == 2 ? 2 : 1;
+  KParams p;
+  {
+    cudaError_t e0 = fill_kparams(g, 0, 0, p);
+    if (e0 != cudaSuccess) return e0;
+  }
+  const int ks = p.k_splits, stages = p.n_stages, stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
   const int units = p.m_tiles * p.n_tiles * ks;
   if (units <= 0) return cudaSuccess;
   const int groups = num_sms / cg;
