@@ -1,13 +1,16 @@
 #!/usr/bin/env python
-"""Benchmark of the Learn2PD denoising step on B200.
+"""Benchmark of the Learn2PD denoising step and decode on B200.
 
   python bench.py --gpus N --steps K --warmup W            (this implementation)
   python bench.py --impl reference --steps K --warmup W    (the CPU oracle, timed as it stands)
 
-Workload (N = 1 and every replica at N > 1): one denoising step of the LLaDA-8B-shaped
-model — batch 1, 256 prompt tokens + 256 masked positions, block 32 — i.e. the state set-up of
-Algorithm 2 followed by M(X), the confidence head, the filter, the threshold and EoTP.
-A "step" of the timed loop is exactly that, repeated K times on the same seeded prompt.
+Timed step (N = 1 and every replica at N > 1): one denoising step of the LLaDA-8B-shaped model — batch 1, 256
+prompt tokens + 256 masked positions, block 32 — i.e. the state set-up of Algorithm 2 followed by M(X), the
+confidence head, the filter, the threshold and EoTP.  A "step" of the timed loop is exactly that, repeated K times
+on the same seeded prompt; `ms_per_step` is its time.  `value` (generated tokens per second) is measured on the full
+Learn2PD decode of the same model and prompt shape (256 + 256, EoT logit biased so that EoTP fires): tokens up to
+and including [EoT] over the decode's device time, summed over ranks.
+With --gpus N > 1 and no launcher environment the script starts its N ranks itself (one per GPU, NCCL).
 Prints ONE JSON line (rank 0).
 """
 from __future__ import annotations
@@ -33,10 +36,10 @@ WORKLOAD = "C1"
 SHAPE = wl.LLADA_8B
 DEC = wl.DECODES[WORKLOAD]
 METRIC, UNIT = "generated_tokens_per_s", "tokens/s"
-# DRAM bytes (read + write) of one gate/up launch at T = 512: dram__bytes_read.sum + dram__bytes_write.sum of
-# the ncu capture summarised in profiles/gemm_pair_T512_layer_shapes.md (209.0 MB + 4.2 MB)
-GATE_UP_DRAM_BYTES_PER_LAUNCH = 213.2e6
+EOT_BIAS = 14.0          # the seeded constant added to the [EoT] logit in the decode workloads
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# DRAM bytes of one gate/up launch at 512 rows, from the ncu capture summarised under profiles/ (null when absent)
+TRAFFIC_FILE = os.path.join(ROOT, "profiles", "gate_up_T512_dram_traffic.txt")
 
 
 def peaks():
@@ -47,8 +50,19 @@ def peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
-def step_work(shape, T, Lk, R):
-    """Algorithmic FLOPs and bytes of one denoising step over T rows, keys Lk per query, R LM-head rows."""
+def measured_traffic():
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, or None."""
+    try:
+        for line in open(TRAFFIC_FILE):
+            if line.startswith("bytes_per_launch"):
+                return float(line.split("=")[1].split("#")[0])
+    except OSError:
+        pass
+    return None
+
+
+def step_work(shape, T, Lk, R, kv_read_bytes=0.0):
+    """Algorithmic FLOPs and bytes of one denoising step over T rows, Lk keys per query, R LM-head rows."""
     d, F, V, NL = shape.d_model, shape.d_ff, shape.vocab, shape.n_layers
     hd = shape.n_heads * shape.head_dim
     gemm = 2.0 * T * NL * (d * 3 * hd + hd * d + 3 * d * F)
@@ -56,91 +70,102 @@ def step_work(shape, T, Lk, R):
     head = 2.0 * R * d * V
     w_bytes = 2.0 * (NL * (d * 3 * hd + hd * d + 3 * d * F) + V * d)
     act_bytes = 44.0 * T * d * NL
-    return {"flops": gemm + attn + head, "gemm_flops": gemm, "attn_flops": attn, "head_flops": head,
-            "weight_bytes": w_bytes, "act_bytes": act_bytes}
+    return {"flops": gemm + attn + head, "weight_bytes": w_bytes, "act_bytes": act_bytes, "kv_bytes": kv_read_bytes}
 
 
-# ------------------------------------------------------------------------------------------------
-# CPU oracle leg (shared by cpu_baseline and --impl reference)
-
-class OracleSample:
-    """Times the oracle on a bounded sample of the step: the embedding, `n_sample` of the model's
-    layers and the LM head + decision on the block's rows; the layer time is scaled to full depth."""
-
-    def __init__(self, n_sample=4, budget_s=None, calls=1):
-        if budget_s is not None:   # about 2 s per layer and 1 s for the head on 8 cores
-            n_sample = int(min(4, max(1, (budget_s / max(calls, 1) - 1.0) // 2)))
-        from oracle import l2pd_oracle as orc
-        self.orc = orc
-        self.n_sample = n_sample
-        shape = wl.thin(SHAPE, n_sample)
-        w = wl.make_weights(shape, seed=0, final_norm_gain=wl.spread_gain(SHAPE), threads=os.cpu_count() or 8)
-        self.model = orc.Model(n_layers=n_sample, d_model=shape.d_model, n_heads=shape.n_heads, head_dim=shape.head_dim,
-                               d_ff=shape.d_ff, vocab=shape.vocab, rms_eps=shape.rms_eps, rope_theta=shape.rope_theta,
-                               mask_id=shape.mask_id, eot_id=shape.eot_id, weights=w)
-        self.filt = wl.make_filter(DEC.block_len, DEC.tau, seed=0)
-        self.prompt = wl.make_prompts(1, DEC.prompt_len, SHAPE, seed=1)[0]
-        self.cfg = orc.DecodeConfig(block_len=DEC.block_len, tau=DEC.tau)
-
-    def one(self):
-        """Returns (extrapolated seconds for a full-depth step, tokens the sample's step committed)."""
-        orc = self.orc
-        st = orc.init_state(self.model, self.prompt, DEC.gen_len)
-        t0 = time.perf_counter()
-        w = self.model.weights
-        x = orc.widen(w["tok_emb"][st.tokens[: st.L_eff]])
-        pos = np.arange(st.L_eff)
-        t1 = time.perf_counter()
-        for layer in w["layers"]:
-            x = orc.layer_forward(self.model, layer, x, pos)
-        t2 = time.perf_counter()
-        S_b = st.P
-        logits = orc.lm_head_logits(self.model, x[S_b: S_b + DEC.block_len])
-        pred, conf, gap = orc.confidence_head(logits)
-        rec = orc.decide(self.model, self.filt, st, self.cfg, pred, conf)
-        t3 = time.perf_counter()
-        full = (t1 - t0) + (t2 - t1) * SHAPE.n_layers / self.n_sample + (t3 - t2)
-        return full, int(rec.unmask.sum()), (t3 - t0)
-
-
-def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
-        return
-    import threadpoolctl
-    cores = max(i["num_threads"] for i in threadpoolctl.threadpool_info() or [{"num_threads": os.cpu_count()}])
-    smp = OracleSample(budget_s=150.0, calls=args.steps + args.warmup)
-    for _ in range(args.warmup):
-        smp.one()
-    times, toks, raw = [], 0, 0.0
-    for _ in range(args.steps):
-        t, n, r = smp.one()
-        times.append(t)
-        toks += n
-        raw += r
-    total = sum(times)
-    value = toks / total
-    sample = ("embedding + %d of %d layers + LM head/decision on %d rows at T=%d, layer time scaled x%d; "
-              "tokens = commits of the sample's own step" % (smp.n_sample, SHAPE.n_layers, DEC.block_len,
-                                                            DEC.prompt_len + DEC.gen_len, SHAPE.n_layers // smp.n_sample))
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": config_dict(), "gpu_launches": 0,
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
-                             "measured_s_per_sample": raw / args.steps},
-            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
-    print(json.dumps(line))
+def roofline_ms(work, pk):
+    """The slower of FLOPs at the bf16 peak and bytes at the HBM peak, for the burst and the sustained bf16 figure."""
+    t_bytes = (work["weight_bytes"] + work["act_bytes"] + work.get("kv_bytes", 0.0)) / (pk["hbm_gbs"] * 1e9)
+    t_burst = max(work["flops"] / (pk["bf16_tflops"] * 1e12), t_bytes)
+    t_sust = max(work["flops"] / (pk["bf16_tflops_sustained"] * 1e12), t_bytes)
+    bound = "tensor" if work["flops"] / (pk["bf16_tflops"] * 1e12) >= t_bytes else "hbm"
+    return 1e3 * t_burst, 1e3 * t_sust, 1e3 * t_bytes, bound
 
 
 def config_dict():
     return {"workload": "%s: one denoising step, LLaDA-8B-shaped model (32 layers, d 4096, 32 heads x 128, "
-                        "SwiGLU 12288, vocab 126464), batch 1, prompt %d + %d masked, block %d, filter + EoTP"
+                        "SwiGLU 12288, vocab 126464), batch 1, prompt %d + %d masked, block %d, filter + EoTP "
+                        "(ms_per_step); value = generated tokens/s of the full decode of the same shape (C2)"
                         % (WORKLOAD, DEC.prompt_len, DEC.gen_len, DEC.block_len),
             "tokens_per_step_rows": DEC.prompt_len + DEC.gen_len, "block_len": DEC.block_len, "tau": DEC.tau,
+            "eot_bias": EOT_BIAS,
             "l2": "inputs larger than L2: every step streams 15 GB of weights",
             "weights": "N(0, 0.02^2) bf16, drawn on the device with torch's generator, seed 0",
             "parallelism": "replicas"}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline and --impl reference): whole steps of the full-depth model, measured
+
+class OracleStep:
+    """The oracle as it stands, one call = one whole denoising step of the 32-layer model (embedding, every layer over
+    the sequence's rows, LM head on the block's rows, confidence head, decision).  fresh(): the C1 step (state set-up,
+    then the first step); next(): the following step of the same decode (the C2 workload, EoT logit biased)."""
+
+    def __init__(self, eot_bias=None):
+        from oracle import l2pd_oracle as orc
+        self.orc = orc
+        t0 = time.perf_counter()
+        w = wl.make_weights(SHAPE, seed=0, final_norm_gain=wl.spread_gain(SHAPE), threads=os.cpu_count() or 8)
+        self.setup_s = time.perf_counter() - t0
+        self.model = orc.Model(n_layers=SHAPE.n_layers, d_model=SHAPE.d_model, n_heads=SHAPE.n_heads, head_dim=SHAPE.head_dim,
+                               d_ff=SHAPE.d_ff, vocab=SHAPE.vocab, rms_eps=SHAPE.rms_eps, rope_theta=SHAPE.rope_theta,
+                               mask_id=SHAPE.mask_id, eot_id=SHAPE.eot_id, weights=w,
+                               lm_head_bias=None if eot_bias is None else wl.make_eot_bias(SHAPE, eot_bias))
+        self.filt = wl.make_filter(DEC.block_len, DEC.tau, seed=0)
+        self.prompt = wl.make_prompts(1, DEC.prompt_len, SHAPE, seed=1)[0]
+        self.cfg = orc.DecodeConfig(block_len=DEC.block_len, tau=DEC.tau)
+        self.st = None
+
+    def fresh(self):
+        self.st = self.orc.init_state(self.model, self.prompt, DEC.gen_len)
+        return self.next()
+
+    def next(self):
+        """Returns (seconds, positions the step committed)."""
+        t0 = time.perf_counter()
+        rec = self.orc.denoise_step(self.model, self.filt, self.st, self.cfg)
+        return time.perf_counter() - t0, int(rec.unmask.sum())
+
+
+def oracle_cores():
+    import threadpoolctl
+    return max(i["num_threads"] for i in threadpoolctl.threadpool_info() or [{"num_threads": os.cpu_count()}])
+
+
+def run_reference(args):
+    """The oracle on a bounded sample of the decode workload `value` is quoted on: the first steps of the C2 decode of
+    sequence 0 (whole 32-layer steps, measured one by one), as many of the K asked as fit the time budget or until the
+    first block is fully unmasked; value = positions those steps committed / their time."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    smp = OracleStep(eot_bias=EOT_BIAS)
+    cores = oracle_cores()
+    budget_s = 150.0                     # a step is ~30 s on 16 cores
+    times, toks = [], 0
+    t, n = smp.fresh()
+    times.append(t)
+    toks += n
+    while (len(times) < args.steps and not smp.st.done and smp.st.cur_block == 0
+           and sum(times) + 1.2 * max(times) < budget_s):
+        t, n = smp.next()
+        times.append(t)
+        toks += n
+    total = sum(times)
+    value = toks / total
+    sample = ("the first %d denoising steps of the C2 decode of sequence 0 (of %d asked), each a whole step of the 32-layer model "
+              "measured directly (~%.0f s each; no warm-up step: a step is tens of seconds; weights drawn in %.0f s beforehand); "
+              "they committed %d of the first block's %d positions; value = those tokens / their time"
+              % (len(times), args.steps, total / len(times), smp.setup_s, toks, DEC.block_len))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": len(times), "steps_requested": args.steps, "warmup": 0, "warmup_requested": args.warmup,
+            "ms_per_step": 1e3 * total / len(times),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": config_dict(), "gpu_launches": 0,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
 
 
 # ------------------------------------------------------------------------------------------------
@@ -175,7 +200,7 @@ class ClockSampler:
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.Q,
-                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                       "--format=csv,noheader,nounits", "-lms", "50"], stdout=self.f,
                                       stderr=subprocess.DEVNULL)
         except Exception:
             self.p = None
@@ -204,10 +229,20 @@ class ClockSampler:
         return out
 
 
+def traced_decode(dec, d_prompts, G):
+    """The decode as state set-up + step loop, with each step's device time and row count (for per-step rooflines)."""
+    dec.state_reset_device(d_prompts, G)
+    rec = []
+    while dec.num_active > 0:
+        h = dec.denoise_step_host()
+        rec.append((dec.last_step_ms, dec.last_step_rows, h["l_eff"].copy(), h["done"].copy()))
+    return rec
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from paper_2509_25188_b200 import binding
+    from paper_2509_25188_b200 import binding, replicas
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -235,20 +270,19 @@ def run_ours(args):
         dec.state_reset_device(d_prompts, G)
         return dec.denoise_step_host()
 
-    for _ in range(max(args.warmup, 3)):
+    warm = max(args.warmup, 3)
+    for _ in range(warm):
         one_resident()
 
-    # ---- timed region 1: inputs resident in HBM
+    # ---- timed region 1: K denoising steps, inputs resident in HBM
     sampler = ClockSampler(local) if rank == 0 else None
     dec.profile_enable(["gemm_gate_up"])
     launches0 = dec.launch_count
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    tokens = 0
     barrier()
     ev0.record()
     for _ in range(args.steps):
-        h = one_resident()
-        tokens += int((s - h["masks_left"]).sum())
+        one_resident()
     ev1.record()
     barrier()
     ms = ev0.elapsed_time(ev1)
@@ -256,13 +290,12 @@ def run_ours(args):
     prof = dec.profile_read()
     dec.profile_enable([])
 
-    # ---- timed region 2: host buffers in, host results out, through the same calls
+    # ---- timed region 2: the same steps end to end — host prompt in, host results out, every step
     dev_in = torch.empty_like(d_prompts)
     o_conf = torch.empty(B, s, device=dev)
     o_pred = torch.empty(B, s, dtype=torch.int32, device=dev)
     o_un = torch.empty(B, s, dtype=torch.uint8, device=dev)
     h_conf, h_pred, h_un = (torch.empty_like(t, device="cpu").pin_memory() for t in (o_conf, o_pred, o_un))
-    tokens_e2e = 0
     barrier()
     ev0.record()
     for _ in range(args.steps):
@@ -273,236 +306,208 @@ def run_ours(args):
         h_pred.copy_(o_pred, non_blocking=True)
         h_un.copy_(o_un, non_blocking=True)
         torch.cuda.current_stream().synchronize()
-        tokens_e2e += int(h_un.sum())
     ev1.record()
     barrier()
-    ms_e2e = ev0.elapsed_time(ev1)
-    clocks = sampler.stop() if sampler else None
+    ms_e2e_step = ev0.elapsed_time(ev1)
 
+    # ---- timed region 3: full Learn2PD decodes (C2).  Two per rank, handed out from a queue shared by the ranks
+    # (a rank that is done takes the next one), gathered over the process group at the end.
+    bias = wl.make_eot_bias(SHAPE, EOT_BIAS)
+    dec2 = binding.Decoder(SHAPE, w, filt, block_len=s, tau=DEC.tau, max_batch=B, max_seq=P + G, device=local, lm_head_bias=bias)
+    n_dec = 2 * world
+    dec_prompts = wl.make_prompts(n_dec, P, SHAPE, seed=1)            # sequence 0 = the prompt of the timed step
+    h_dec_prompts = torch.from_numpy(dec_prompts).pin_memory()
+    d_one = torch.empty(1, P, dtype=torch.int32, device=dev)
+    d_out = torch.empty(1, G, dtype=torch.int32, device=dev)
+    h_out = torch.empty(1, G, dtype=torch.int32).pin_memory()
+    d_one.copy_(h_dec_prompts[0:1])
+    dec2.decode_device(d_one, G, d_out)                                # warm-up at the decode's shapes
     if world > 1:
-        from paper_2509_25188_b200 import replicas
-        ms, (tokens, launches) = replicas.reduce_timing(ms, [tokens, launches], device=dev)
-        ms_e2e, (tokens_e2e,) = replicas.reduce_timing(ms_e2e, [tokens_e2e], device=dev)
-        tokens, tokens_e2e, launches = int(tokens), int(tokens_e2e), int(launches)
-
-    # ---- untimed: per-kernel breakdown of one step
-    breakdown = {}
-    if rank == 0:
-        dec.profile_enable(binding.KINDS)
-        for _ in range(3):
-            one_resident()
-        for k, (t_ms, n) in dec.profile_read().items():
-            breakdown[k] = {"ms_per_step": round(t_ms / 3, 4), "launches_per_step": n // 3}
-        dec.profile_enable([])
-
-    # ---- untimed extra: one full decode (state set-up, every denoising step of every block, EoTP) on the same model
-    decode_info = None
-    if rank == 0:
-        eot_bias = 14.0
-        dec2 = binding.Decoder(SHAPE, w, filt, block_len=s, tau=DEC.tau, max_batch=B, max_seq=P + G, device=local,
-                               lm_head_bias=wl.make_eot_bias(SHAPE, eot_bias))
-        d_out = torch.empty(B, G, dtype=torch.int32, device=dev)
-        dec2.decode_device(d_prompts, G, d_out)
-        torch.cuda.synchronize()
+        store = dist.distributed_c10d._get_default_store()
+    idx, toks, lens, stps = [], [], [], []
+    dec_ms = dec_ms_e2e = 0.0
+    barrier()
+    t_wall0 = time.perf_counter()
+    chunks = replicas.claim_chunks(store, n_dec) if world > 1 else iter(range(n_dec))
+    for i in chunks:
+        # end to end: the prompt comes from pinned host memory and the response goes back to it, inside the timed region
         ev0.record()
-        out_len, seq_steps, total_steps = dec2.decode_device(d_prompts, G, d_out)
+        d_one.copy_(h_dec_prompts[i:i + 1], non_blocking=True)
+        ev_in = torch.cuda.Event(enable_timing=True)
+        ev_in.record()
+        out_len, seq_steps, total_steps = dec2.decode_device(d_one, G, d_out)
+        ev_out = torch.cuda.Event(enable_timing=True)
+        ev_out.record()
+        h_out.copy_(d_out, non_blocking=True)
         ev1.record()
         torch.cuda.synchronize()
-        ms_dec = ev0.elapsed_time(ev1)
-        decode_info = {"workload": "C2: full Learn2PD decode, prompt %d + generation %d, block %d, filter + EoTP, "
-                                   "EoT logit biased by the constant %.1f" % (P, G, s, eot_bias),
-                       "steps_per_sequence": float(np.mean(seq_steps)), "steps_one_token_per_step": G,
-                       "out_len": [int(v) for v in out_len], "ms": ms_dec, "ms_per_step": ms_dec / max(total_steps, 1),
-                       "generated_tokens_per_s": float(np.sum(out_len)) / (ms_dec * 1e-3)}
-        dec2.close()
+        dec_ms += ev_in.elapsed_time(ev_out)
+        dec_ms_e2e += ev0.elapsed_time(ev1)
+        idx.append(i)
+        toks.append(h_out.numpy().copy())
+        lens.append(int(out_len[0]))
+        stps.append(int(seq_steps[0]))
+    barrier()
+    wall_ms = 1e3 * (time.perf_counter() - t_wall0)
+    toks_np = np.concatenate(toks) if toks else np.zeros((0, G), np.int32)
+    if world > 1:
+        all_toks, all_len, all_steps = replicas.gather_indexed(idx, toks_np, np.array(lens), np.array(stps), n_dec, G, device=dev)
+        dec_ms, (_,) = replicas.reduce_timing(dec_ms, [0.0], device=dev)
+        dec_ms_e2e, (_,) = replicas.reduce_timing(dec_ms_e2e, [0.0], device=dev)
+        ms, (launches,) = replicas.reduce_timing(ms, [launches], device=dev)
+        ms_e2e_step, (_,) = replicas.reduce_timing(ms_e2e_step, [0.0], device=dev)
+        launches = int(launches)
+    else:
+        all_toks, all_len, all_steps = toks_np, np.array(lens), np.array(stps)
+    clocks = sampler.stop() if sampler else None
+    gen_tokens = float(np.sum(all_len))
+    value = gen_tokens / (dec_ms * 1e-3)                 # all ranks' tokens over the slowest rank's decode time
+    value_e2e = gen_tokens / (dec_ms_e2e * 1e-3)
 
-    # ---- optional, untimed by the contract: first step (and, with the prefix cache, a cached step) of the batched workloads
-    extra = None
-    if rank == 0 and args.extra_workloads:
-        extra = {}
-        for name in ("C3", "C4"):
-            dsh = wl.DECODES[name]
-            Bx, Px, Gx = dsh.batch, dsh.prompt_len, dsh.gen_len
-            decx = binding.Decoder(SHAPE, w, filt, block_len=s, tau=dsh.tau, max_batch=Bx, max_seq=Px + Gx, device=local,
-                                   kv_cache=dsh.kv_cache)
-            px = torch.from_numpy(wl.make_prompts(Bx, Px, SHAPE, seed=100)).to(dev)
-
-            def first_step():
-                decx.state_reset_device(px, Gx)
-                decx.denoise_step_host()
-                return decx.last_step_ms
-            for _ in range(2):
-                first_step()
-            t_first = statistics.median(first_step() for _ in range(5))
-            Tx = Bx * (Px + Gx)
-            wk = step_work(SHAPE, Tx, Px + Gx, Bx * s)
-            t_roof = 1e3 * max(wk["flops"] / (pk["bf16_tflops_sustained"] * 1e12),
-                               (wk["weight_bytes"] + wk["act_bytes"]) / (pk["hbm_gbs"] * 1e9))
-            rec = {"rows": Tx, "first_step_ms": t_first, "first_step_roofline_ms": t_roof, "frac": t_roof / t_first,
-                   "tflops": wk["flops"] / (t_first * 1e-3) / 1e12}
-            if dsh.kv_cache:
-                decx.state_reset_device(px, Gx)
-                decx.denoise_step_host()
-                times = []
-                for _ in range(3):
-                    if decx.num_active == 0:
-                        break
-                    decx.denoise_step_host()
-                    times.append((decx.last_step_ms, decx.last_step_rows))
-                if times:
-                    rec["cached_step_ms"], rec["cached_step_rows"] = times[-1]
-            extra[name] = rec
-            decx.close()
-        # dual cache (Section 4.3): in-block steps run the block's s rows per sequence against the stored keys and
-        # values of every other position; with so few rows the step streams the weights once and is HBM-bound
-        for name, dsh in (("C2_dual_cache", wl.DECODES["C2"]), ("C4_dual_cache", wl.DECODES["C4"])):
-            Bx, Px, Gx = dsh.batch, dsh.prompt_len, dsh.gen_len
-            decx = binding.Decoder(SHAPE, w, None, block_len=s, tau=dsh.tau, max_batch=Bx, max_seq=Px + Gx, device=local,
-                                   kv_cache=2, use_filter=False)      # one commit per step: s - 1 stored-key steps per block
-            px = torch.from_numpy(wl.make_prompts(Bx, Px, SHAPE, seed=100)).to(dev)
-            decx.state_reset_device(px, Gx)
-            decx.denoise_step_host()
-            t_first = decx.last_step_ms
-            for _ in range(3):
-                decx.denoise_step_host()
-            times = []
-            for _ in range(12):
-                decx.denoise_step_host()
-                times.append(decx.last_step_ms)
-            rows = decx.last_step_rows
-            t_in = statistics.median(times)
-            wk = step_work(SHAPE, rows, Px + Gx, Bx * s)
-            kv_bytes = 2.0 * 2 * SHAPE.n_layers * Bx * (Px + Gx) * SHAPE.n_heads * SHAPE.head_dim   # stored K and V read once
-            t_roof = 1e3 * max(wk["flops"] / (pk["bf16_tflops_sustained"] * 1e12),
-                               (wk["weight_bytes"] + wk["act_bytes"] + kv_bytes) / (pk["hbm_gbs"] * 1e9))
-            extra[name] = {"rows": rows, "first_step_ms": t_first, "in_block_step_ms": t_in, "in_block_roofline_ms": t_roof,
-                           "frac": t_roof / t_in, "bound": "hbm",
-                           "achieved_gbs": (wk["weight_bytes"] + wk["act_bytes"] + kv_bytes) / (t_in * 1e-3) / 1e9,
-                           "rows_per_s": rows / (t_in * 1e-3)}
-            decx.close()
-
-        # long generation (the setting of Section 4.3's EoTP study: generation length 1024, block 32): one sequence, the
-        # EoT logit biased so that the answer ends early; the same decode with and without EoTP
-        Pl, Gl, bias_l = 1024, 1024, 14.0
-        pl_ = torch.from_numpy(wl.make_prompts(1, Pl, SHAPE, seed=7)).to(dev)
-        out_l = torch.empty(1, Gl, dtype=torch.int32, device=dev)
-        rec = {"prompt_len": Pl, "gen_len": Gl, "eot_bias": bias_l}
-        for tag, eotp in (("eotp", True), ("no_eotp", False)):
-            decl = binding.Decoder(SHAPE, w, filt, block_len=s, tau=DEC.tau, max_batch=1, max_seq=Pl + Gl, device=local,
-                                   use_eotp=eotp, lm_head_bias=wl.make_eot_bias(SHAPE, bias_l))
-            decl.state_reset_device(pl_, Gl)
-            decl.denoise_step_host()                       # warm-up at this shape
-            ev0.record()
-            ol, st_l, tot_l = decl.decode_device(pl_, Gl, out_l)
-            ev1.record()
-            torch.cuda.synchronize()
-            first_eot = (out_l[0] == SHAPE.eot_id).nonzero()
-            rec[tag] = {"ms": ev0.elapsed_time(ev1), "steps": int(tot_l), "out_len": int(ol[0]),
-                        "first_eot": int(first_eot[0]) if len(first_eot) else -1}
-            decl.close()
-        rec["speedup_from_eotp"] = rec["no_eotp"]["ms"] / rec["eotp"]["ms"]
-        extra["long_generation"] = rec
-
-        # threshold sweep (Section 4.4 studies tau = 0.9 ... 0.99) and the comparison policies on the C2 decode: steps and
-        # generated tokens per second of one sequence with the same synthetic model, filter and EoT bias
-        sweep = {}
-        d_out2 = torch.empty(B, G, dtype=torch.int32, device=dev)
-        for tag, kw, rule in [("tau_0.90", {"tau": 0.90}, None), ("tau_0.96", {"tau": 0.96}, None), ("tau_0.99", {"tau": 0.99}, None),
-                              ("confidence_0.9", {"tau": DEC.tau}, ("confidence", 0.9)),
-                              ("one_token_per_step", {"tau": DEC.tau}, ("confidence", 1.0))]:
-            decs = binding.Decoder(SHAPE, w, filt, block_len=s, max_batch=B, max_seq=P + G, device=local,
-                                   lm_head_bias=wl.make_eot_bias(SHAPE, 14.0), **kw)
-            if rule:
-                decs.set_unmask_rule(rule[0], conf_threshold=rule[1])
-            decs.state_reset_device(d_prompts, G)
-            decs.denoise_step_host()
-            ev0.record()
-            ol, st_s, tot_s = decs.decode_device(d_prompts, G, d_out2)
-            ev1.record()
-            torch.cuda.synchronize()
-            ms_s = ev0.elapsed_time(ev1)
-            sweep[tag] = {"steps": int(tot_s), "out_len": int(ol[0]), "ms": ms_s,
-                          "generated_tokens_per_s": float(np.sum(ol)) / (ms_s * 1e-3)}
-            decs.close()
-        base_steps = sweep["one_token_per_step"]["steps"]
-        for v in sweep.values():
-            v["steps_vs_one_token_per_step"] = base_steps / max(v["steps"], 1)
-        extra["policy_sweep_C2"] = sweep
-
-        # filter training at the paper's scale (Section 4.1: 2,640 prompts, 5,000 epochs, lr 0.001): synthetic samples,
-        # one per decoding step of a 32-step-per-prompt EGP run; the whole of stage 2 on the device
-        n_samp = 2640 * 32
-        rng = np.random.default_rng(0)
-        c_s = rng.uniform(0.0, 1.0, size=(n_samp, s)).astype(np.float32)
-        y_s = (c_s + 0.15 * rng.normal(size=(n_samp, s)) > 0.6).astype(np.uint8)
-        tc_s, ty_s = torch.from_numpy(c_s).to(dev), torch.from_numpy(y_s).to(dev)
-        binding.filter_train(filt, tc_s, ty_s, 20)
-        ev0.record()
-        _, tr_losses = binding.filter_train(filt, tc_s, ty_s, 5000)
-        ev1.record()
-        torch.cuda.synchronize()
-        ms_tr = ev0.elapsed_time(ev1)
-        fl_epoch = 10.0 * n_samp * s * s        # two products forward, three backward, 2 flops per multiply-add
-        extra["filter_training"] = {"samples": n_samp, "block_len": s, "epochs": 5000, "batch": "full", "ms": ms_tr,
-                                    "us_per_epoch": 1e3 * ms_tr / 5000, "gflops": fl_epoch * 5000 / (ms_tr * 1e-3) / 1e9,
-                                    "loss_first": float(tr_losses[0]), "loss_last": float(tr_losses[-1])}
-
+    line = None
     if rank == 0:
         T, R = B * (P + G), B * s
         work = step_work(SHAPE, T, P + G, R)
-        t_flops = work["flops"] / (pk["bf16_tflops_sustained"] * 1e12)
-        t_bytes = (work["weight_bytes"] + work["act_bytes"]) / (pk["hbm_gbs"] * 1e9)
-        t_roof_ms = 1e3 * max(t_flops, t_bytes)
+        t_burst, t_sust, t_bytes, bound = roofline_ms(work, pk)
         ms_step = ms / args.steps
         gu_ms, gu_n = prof.get("gemm_gate_up", (0.0, 0))
         gu_flops = 2.0 * T * SHAPE.d_model * 2 * SHAPE.d_ff
         achieved = gu_flops / (gu_ms / gu_n * 1e-3) / 1e12 if gu_n else None
         line = {
-            "metric": METRIC, "value": tokens / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": config_dict(),
-            "clocks": clocks,
-            "e2e": {"value": tokens_e2e / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e / args.steps,
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+            "data": "synthetic", "config": config_dict(), "clocks": clocks,
+            "e2e": {"value": value_e2e, "unit": UNIT, "ms_per_step": ms_e2e_step / args.steps,
+                    "what": "decodes with the prompt copied from pinned host memory and the response copied back inside the timed "
+                            "region (value); ms_per_step: the timed step with its prompt copied in and conf / pred / unmask copied out",
                     "h2d_bytes_per_step": int(h_prompts.numel() * 4),
                     "d2h_bytes_per_step": int(h_conf.numel() * 4 + h_pred.numel() * 4 + h_un.numel() + 6 * 4 * B + 4)},
             "gpu_launches": int(launches),
-            "tokens_per_step": tokens / (args.steps * world),
             "roofline": {"kernel": "gemm_tcgen05_pair_kernel<EPI_SWIGLU> (gate/up projection + SwiGLU)", "bound": "tensor",
-                         "achieved": achieved, "peak": pk["bf16_tflops_sustained"], "unit": "TFLOP/s",
-                         "frac": (achieved / pk["bf16_tflops_sustained"]) if achieved else None,
-                         "peak_source": pk_src + " (sustained bf16, kernel timed inside a long step)",
+                         "achieved": achieved, "peak": pk["bf16_tflops"], "unit": "TFLOP/s",
+                         "frac": (achieved / pk["bf16_tflops"]) if achieved else None,
+                         "peak_source": pk_src + " (burst bf16)",
+                         "frac_sustained": (achieved / pk["bf16_tflops_sustained"]) if achieved else None,
                          "flops_per_launch": gu_flops, "avg_launch_ms": gu_ms / gu_n if gu_n else None,
-                         "traffic": GATE_UP_DRAM_BYTES_PER_LAUNCH,
+                         "traffic": measured_traffic(),
                          "algorithmic_bytes": 2.0 * (2 * SHAPE.d_ff * SHAPE.d_model + T * SHAPE.d_model + T * SHAPE.d_ff)},
             "step_roofline": {"flops": work["flops"], "weight_bytes": work["weight_bytes"], "act_bytes": work["act_bytes"],
-                              "t_flops_ms": 1e3 * t_flops, "t_bytes_ms": 1e3 * t_bytes, "t_roof_ms": t_roof_ms,
-                              "frac": t_roof_ms / ms_step,
-                              # the same against the burst bf16 figure (a GEMM timed alone for a moment; a whole step runs
-                              # under the power cap, which is what the sustained figure measures)
-                              "t_roof_burst_ms": 1e3 * max(work["flops"] / (pk["bf16_tflops"] * 1e12), t_bytes),
-                              "frac_burst": 1e3 * max(work["flops"] / (pk["bf16_tflops"] * 1e12), t_bytes) / ms_step,
+                              "bound": bound, "t_bytes_ms": t_bytes, "t_roof_ms": t_burst, "frac": t_burst / ms_step,
+                              "t_roof_sustained_ms": t_sust, "frac_sustained": t_sust / ms_step,
+                              "note": "frac: against the burst bf16 figure (the target's denominator); frac_sustained: against the "
+                                      "seconds-long figure under the power cap",
                               "peaks": pk, "peak_source": pk_src},
-            "breakdown": breakdown,
-            "decode": decode_info,
+            "decode": {"workload": "C2: full Learn2PD decode, prompt %d + generation %d, block %d, filter + EoTP, EoT logit biased "
+                                   "by the constant %.1f; %d sequences (2 per rank, taken from a shared queue)" % (P, G, s, EOT_BIAS, n_dec),
+                       "sequences": n_dec, "out_len": [int(v) for v in all_len], "steps_per_sequence": float(np.mean(all_steps)),
+                       "steps_one_token_per_step": G, "device_ms_slowest_rank": dec_ms, "wall_ms": wall_ms,
+                       "generated_tokens_per_s": value},
         }
-        if extra is not None:
-            line["extra_workloads"] = extra
-        if world == 1 and not args.no_cpu_baseline:
-            import threadpoolctl
-            smp = OracleSample()
-            cores = max(i["num_threads"] for i in threadpoolctl.threadpool_info() or [{"num_threads": os.cpu_count()}])
-            smp.one()
-            full_s, n_tok, raw = smp.one()
-            line["cpu_baseline"] = {
-                "value": (tokens / (args.steps * world)) / full_s, "unit": UNIT, "cores": cores, "kind": "oracle",
-                "ms_per_step": 1e3 * full_s,
-                "sample": "embedding + %d of %d layers + LM head/decision on %d rows at T=%d (%.1f s measured), layer "
-                          "time scaled x%d; tokens per step taken from the GPU run of the same workload"
-                          % (smp.n_sample, SHAPE.n_layers, s, T, raw, SHAPE.n_layers // smp.n_sample)}
-        print(json.dumps(line))
+
+    # ---- untimed, rank 0: per-kernel breakdown of the step; per-step rooflines of a decode; the other configurations
+    if rank == 0:
+        dec.profile_enable(binding.KINDS)
+        for _ in range(3):
+            one_resident()
+        line["breakdown"] = {k: {"ms_per_step": round(t_ms / 3, 4), "launches_per_step": n // 3}
+                             for k, (t_ms, n) in dec.profile_read().items()}
+        dec.profile_enable([])
+
+        # the decode of sequence 0 step by step: each step's roofline from its actual row count (T = L_eff keys = rows here)
+        d_one.copy_(h_dec_prompts[0:1])
+        rec = traced_decode(dec2, d_one, G)
+        t_meas = sum(r[0] for r in rec)
+        roofs = [roofline_ms(step_work(SHAPE, rows, rows, s), pk) for (_, rows, _, _) in rec]
+        line["decode"]["per_step"] = {
+            "steps": len(rec), "rows_first_last": [rec[0][1], rec[-1][1]], "ms_total": t_meas,
+            "roofline_ms_total": sum(r[0] for r in roofs), "frac_time_weighted": sum(r[0] for r in roofs) / t_meas,
+            "frac_time_weighted_sustained": sum(r[1] for r in roofs) / t_meas,
+            "note": "sum over the decode's steps of each step's roofline (from its own T = L_q = L_k and R = 32) / sum of their device times"}
+    dec2.close()
     dec.close()
+
+    if rank == 0 and not args.no_other_configs:
+        line["other_configs"] = other_configs(binding, torch, w, filt, pk, dev, local)
+
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            del w
+            torch.cuda.empty_cache()
+            smp = OracleStep()
+            t_step, n_tok = smp.fresh()
+            line["cpu_baseline"] = {
+                "value": n_tok / t_step, "unit": UNIT, "cores": oracle_cores(), "kind": "oracle", "ms_per_step": 1e3 * t_step,
+                "sample": "one whole denoising step of the C1 workload (32 layers, 512 rows, LM head on 32 rows, decision) measured "
+                          "directly: %.1f s; tokens = the %d positions that step committed; compare ms_per_step with ms_per_step"
+                          % (t_step, n_tok)}
+        print(json.dumps(line))
     if world > 1:
+        dist.barrier()
         dist.destroy_process_group()
+
+
+def other_configs(binding, torch, w, filt, pk, dev, local):
+    """First / cached steps of the batched configurations and the dual cache's in-block step, each with its roofline
+    (burst and sustained bf16 figure).  Bounded: a few steps per configuration."""
+    s = DEC.block_len
+    out = {}
+
+    def frac(work, t_ms):
+        t_burst, t_sust, _, bound = roofline_ms(work, pk)
+        return {"ms": t_ms, "roofline_ms": t_burst, "frac": t_burst / t_ms, "roofline_sustained_ms": t_sust,
+                "frac_sustained": t_sust / t_ms, "bound": bound}
+
+    for name in ("C3", "C4"):
+        dsh = wl.DECODES[name]
+        Bx, Px, Gx = dsh.batch, dsh.prompt_len, dsh.gen_len
+        decx = binding.Decoder(SHAPE, w, filt, block_len=s, tau=dsh.tau, max_batch=Bx, max_seq=Px + Gx, device=local,
+                               kv_cache=dsh.kv_cache)
+        px = torch.from_numpy(wl.make_prompts(Bx, Px, SHAPE, seed=100)).to(dev)
+
+        def first_step():
+            decx.state_reset_device(px, Gx)
+            decx.denoise_step_host()
+            return decx.last_step_ms
+        first_step()
+        t_first = statistics.median(first_step() for _ in range(3))
+        Tx = Bx * (Px + Gx)
+        rec = {"rows": Tx, "first_step": frac(step_work(SHAPE, Tx, Px + Gx, Bx * s), t_first)}
+        if dsh.kv_cache:
+            decx.state_reset_device(px, Gx)
+            decx.denoise_step_host()
+            times = []
+            for _ in range(3):
+                if decx.num_active == 0:
+                    break
+                decx.denoise_step_host()
+                times.append((decx.last_step_ms, decx.last_step_rows))
+            if times:
+                t_c, rows_c = times[-1]
+                kv = 2.0 * 2 * SHAPE.n_layers * Bx * Px * SHAPE.n_heads * SHAPE.head_dim     # stored K and V of the prefix, read once
+                rec["cached_step"] = dict(rows=rows_c, **frac(step_work(SHAPE, rows_c, Px + Gx, Bx * s, kv), t_c))
+        out[name] = rec
+        decx.close()
+    # dual cache (Section 4.3): in-block steps run the block's s rows per sequence against the stored keys and values
+    for name, dsh in (("C2_dual_cache", wl.DECODES["C2"]), ("C4_dual_cache", wl.DECODES["C4"])):
+        Bx, Px, Gx = dsh.batch, dsh.prompt_len, dsh.gen_len
+        decx = binding.Decoder(SHAPE, w, None, block_len=s, tau=dsh.tau, max_batch=Bx, max_seq=Px + Gx, device=local,
+                               kv_cache=2, use_filter=False)      # one commit per step: s - 1 stored-key steps per block
+        px = torch.from_numpy(wl.make_prompts(Bx, Px, SHAPE, seed=100)).to(dev)
+        decx.state_reset_device(px, Gx)
+        decx.denoise_step_host()
+        t_first = decx.last_step_ms
+        for _ in range(3):
+            decx.denoise_step_host()
+        times = []
+        for _ in range(10):
+            decx.denoise_step_host()
+            times.append(decx.last_step_ms)
+        rows = decx.last_step_rows
+        kv = 2.0 * 2 * SHAPE.n_layers * Bx * (Px + Gx) * SHAPE.n_heads * SHAPE.head_dim
+        out[name] = dict(rows=rows, first_step_ms=t_first,
+                         in_block_step=frac(step_work(SHAPE, rows, Px + Gx, Bx * s, kv), statistics.median(times)))
+        decx.close()
+    return out
 
 
 def main():
@@ -512,19 +517,17 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
-    ap.add_argument("--extra-workloads", action="store_true",
-                    help="also time the first step of the batched workloads (C3: 16 x 1024 rows; C4: 8 x 2048 rows with the "
-                         "prefix cache, plus a cached step) and the in-block step of the dual cache at the C2 and C4 shapes; "
-                         "reported under extra_workloads, outside the contract's numbers")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the steps of the batched configurations (C3, C4) and of the dual cache")
     args = ap.parse_args()
     if args.impl == "reference":
-        if args.steps == 30:
-            args.steps = 3
-        if args.warmup == 5:
-            args.warmup = 1
         run_reference(args)
-    else:
-        run_ours(args)
+        return
+    from paper_2509_25188_b200 import replicas
+    if args.gpus > 1 and not replicas.launcher_env_present():
+        # no launcher started us: start the N ranks ourselves, one per GPU
+        sys.exit(replicas.spawn_local_ranks(args.gpus, os.path.abspath(__file__), sys.argv[1:]))
+    run_ours(args)
 
 
 if __name__ == "__main__":

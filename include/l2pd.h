@@ -5,20 +5,18 @@
  * traps the device: each call returns an l2pd_status, and l2pd_last_error() gives
  * a human-readable reason for the last failure on that context.
  *
- * The computation is the inference procedure of "Learning to Parallel:
- * Accelerating Diffusion LLMs via Learnable Parallel Decoding" (Algorithm 2, with
- * the end-of-text break of Algorithm 3 in the appendix "Update Inference
- * Algorithm"):
- *
- *   X <- concat(prompt, [MASK]^G)
- *   for each block b of s generation positions, left to right:
- *     while the block still has masked positions:
- *        conf, pre = M(X)                       (one "denoising step")
- *        p = sigmoid(f_theta(conf))             (Section 3.2)
- *        for masked j with p_j > tau:  X[P + b*s + j] <- pre_j, j leaves the mask set
- *        EoTP: once an [EoT] token is committed, positions after it are dropped
- *              from the next step's input (Section 3.3)
- *     stop after a block that contains [EoT]
+ * The computation is the inference procedure of the Learn2PD paper (Algorithm 2, with the
+ * end-of-text stop of Algorithm 3).  In this library's terms:
+ *   state   a token row per sequence (prompt, then G generation positions that start as the mask
+ *           token), the set of still-masked generation positions, the current block, and the
+ *           effective length L_eff;
+ *   step    one evaluation of the mask predictor M on every unfinished sequence, giving a
+ *           prediction and a confidence for each position of the sequence's current block (Eq. 3-4),
+ *           followed by the decision: the filter f_theta turns the block's confidences into
+ *           probabilities (Section 3.2), masked positions whose probability exceeds tau are
+ *           committed in place, and a block whose masks are all gone hands over to the next;
+ *   cut     End-of-Text Prediction (Section 3.3): once an [EoT] token is committed, the positions
+ *           after it leave the next step's input, and no block after that one is decoded.
  *
  * M is a LLaDA-style bidirectional transformer: token embedding, n_layers pre-norm
  * blocks (RMSNorm, fused QKV projection, rotary embedding on q and k with
@@ -301,6 +299,13 @@ l2pd_status l2pd_chain_trace_enable(l2pd_ctx *ctx, int32_t enable);
 int64_t l2pd_chain_trace_read(l2pd_ctx *ctx, uint64_t *h_out, int64_t capacity, int32_t *launches, int32_t *phases,
                               int32_t *ctas);
 
+/*
+ * Test hook for the error path: writes `code` into the context's device status word, as a kernel whose bounded
+ * wait ran out would (no kernel is made to wait).  The next l2pd_denoise_step then returns L2PD_ERR_TIMEOUT and
+ * clears the word; the context stays usable.  code = 0 clears it.
+ */
+l2pd_status l2pd_debug_set_device_status(l2pd_ctx *ctx, void *stream, int32_t code);
+
 /* Device time of the most recent step in milliseconds (CUDA events on the step's stream),
  * or a negative value if no step has run. */
 float l2pd_last_step_ms(const l2pd_ctx *ctx);
@@ -379,6 +384,18 @@ l2pd_status l2pd_attention_bf16(void *stream, const void *q, const void *k, cons
                                 void *out, int32_t Tq, int32_t Tk, int32_t H, int32_t dh,
                                 int64_t q_stride, int64_t kv_stride, int64_t out_stride,
                                 int32_t impl, int32_t check);
+
+/*
+ * Environment switches (read once, at l2pd_init or at the first call that uses them; diagnostics and
+ * comparisons only — the defaults are the product):
+ *   L2PD_FORCE_SIMT=1       bf16 configurations run their GEMMs and attention on the CUDA-core cross-check kernels
+ *   L2PD_ATTN_WARP=1        head size 128 keeps the warp-level (mma.sync) attention kernel instead of tcgen05
+ *   L2PD_NO_ROPE_FUSION=1   rotary embedding as a separate kernel instead of the QKV epilogue
+ *   L2PD_NO_PDL=1           kernels launched without programmatic dependent launch
+ *   L2PD_ATOMIC_KSPLIT=1    K slices of the O / down projections add into x in completion order (not
+ *                           bit-reproducible) instead of storing partial sums that are added in slice order
+ *   L2PD_DIRECT_STORES=1    stand-alone GEMM calls use per-thread stores in the epilogue instead of staged TMA stores
+ */
 
 #ifdef __cplusplus
 }

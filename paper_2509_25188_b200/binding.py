@@ -64,7 +64,7 @@ EXPORTS = ["l2pd_init", "l2pd_state_reset", "l2pd_denoise_step", "l2pd_decode", 
            "l2pd_launch_count", "l2pd_last_step_ms", "l2pd_profile_enable", "l2pd_profile_read", "l2pd_last_error", "l2pd_destroy",
            "l2pd_gemm_bf16", "l2pd_gemm_bf16_residual", "l2pd_gemm_bf16_swiglu", "l2pd_lm_head_bf16",
            "l2pd_lm_head_scratch_elems", "l2pd_attention_bf16", "l2pd_lm_head_bf16_static",
-           "l2pd_set_chain", "l2pd_chain_trace_enable", "l2pd_chain_trace_read"]
+           "l2pd_set_chain", "l2pd_chain_trace_enable", "l2pd_chain_trace_read", "l2pd_debug_set_device_status"]
 
 
 KINDS = ["embed", "gemm_qkv", "rope", "attention", "gemm_o", "rmsnorm", "gemm_gate_up", "gemm_down",
@@ -113,6 +113,7 @@ def _load() -> C.CDLL:
     lib.l2pd_lm_head_scratch_elems.restype = i64
     lib.l2pd_lm_head_bf16_static.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, i32]
     lib.l2pd_attention_bf16.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i64, i64, i64, i32, i32]
+    lib.l2pd_debug_set_device_status.argtypes = [vp, vp, i32]
     lib.l2pd_set_chain.argtypes = [vp, i32]
     lib.l2pd_chain_trace_enable.argtypes = [vp, i32]
     lib.l2pd_chain_trace_read.argtypes = [vp, vp, i64, C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]
@@ -320,6 +321,10 @@ class Decoder:
     @property
     def collect_count(self) -> int:
         return int(lib.l2pd_collect_count(self.ctx))
+
+    def debug_set_device_status(self, code: int):
+        """Test hook: presets the device status word (what a kernel's exhausted bounded wait would leave)."""
+        _check(lib.l2pd_debug_set_device_status(self.ctx, _stream(), int(code)), self.ctx)
 
     # ---- chained launches ------------------------------------------------------------------------
     def set_chain(self, enable: bool):

@@ -7,6 +7,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -463,7 +464,7 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
   float *part_m, *part_s;
   int32_t *part_i;
   if (tc) {
-    int tn = pick_tile_n(R, V, c->num_sms, 16, 256);
+    int tn = lm_head_tile_n(R, V, d, c->num_sms);
     if (tn != c->tn_lm) {
       l2pd_status r = make_tma_2d_bf16(&c->tb_lm, c->lm_head, V, d, tn);
       if (r) return set_err(c, r, "tensor map encode failed for the LM head");
@@ -511,8 +512,7 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
   a.n_filter_layers = c->n_filter_layers;
   for (int k = 0; k < 4; ++k) { a.fw[k] = c->flt_w[k]; a.fb[k] = c->flt_b[k]; }
   if (c->n_filter_layers > 0) a.use_filter = 1;
-  if (c->collect_c) {
-    if (c->collect_n + n_slots > c->collect_cap) return set_err(c, L2PD_ERR_SHAPE, "sample sink full (%lld of %lld)", (long long)c->collect_n, (long long)c->collect_cap);
+  if (c->collect_c) {   // (capacity was checked before the step's first launch)
     a.collect_c = c->collect_c; a.collect_y = c->collect_y; a.collect_base = c->collect_n;
     c->collect_n += n_slots;
   }
@@ -568,6 +568,17 @@ l2pd_status validate(const l2pd_config *f, const l2pd_weights *w, std::string *w
 }
 
 }  // namespace
+
+// what failed in the calling thread's last stand-alone call (l2pd_last_error(NULL))
+static thread_local char g_standalone_err[160] = "";
+namespace l2pd {
+void set_standalone_error(const char *fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_standalone_err, sizeof(g_standalone_err), fmt, ap);
+  va_end(ap);
+}
+}  // namespace l2pd
 
 extern "C" {
 
@@ -779,6 +790,8 @@ l2pd_status l2pd_denoise_step(l2pd_ctx *c, void *stream, const l2pd_step_out *ou
     if (L > max_kv) max_kv = L;
   }
   c->last_rows = T_rows;
+  if (c->collect_c && c->collect_n + n_slots > c->collect_cap)   // a full sink: nothing is launched, nothing appended
+    return set_err(c, L2PD_ERR_SHAPE, "sample sink full (%lld of %lld)", (long long)c->collect_n, (long long)c->collect_cap);
   CK(cudaEventRecord(c->ev0, s));
   CK(cudaMemcpyAsync(c->d_meta, c->h_meta, sizeof(SeqMeta) * n_slots, cudaMemcpyHostToDevice, s));
   l2pd_status r = (f.dtype == L2PD_BF16) ? forward_and_decide<bf16>(c, s, n_slots, T_rows, max_q, max_kv, out)
@@ -964,6 +977,14 @@ l2pd_status l2pd_profile_read(const l2pd_ctx *c, int32_t kind, double *ms_total,
 }
 const char *l2pd_last_error(const l2pd_ctx *c);
 
+l2pd_status l2pd_debug_set_device_status(l2pd_ctx *c, void *stream, int32_t code) {
+  if (!c) return L2PD_ERR_ARG;
+  CK(cudaSetDevice(c->device));
+  CK(cudaMemcpyAsync(c->d_status, &code, 4, cudaMemcpyHostToDevice, (cudaStream_t)stream));
+  CK(cudaStreamSynchronize((cudaStream_t)stream));
+  return L2PD_OK;
+}
+
 l2pd_status l2pd_set_chain(l2pd_ctx *c, int32_t enable) {
   if (!c) return L2PD_ERR_ARG;
   c->chain_on = enable != 0;
@@ -1012,8 +1033,6 @@ void l2pd_destroy(l2pd_ctx *c) {
 
 // ---- stand-alone kernels --------------------------------------------------------------------------------
 
-// what failed in the calling thread's last stand-alone call (l2pd_last_error(NULL))
-static thread_local char g_standalone_err[160] = "";
 static l2pd_status standalone_cuda_error(const char *where, cudaError_t e) {
   snprintf(g_standalone_err, sizeof(g_standalone_err), "%s: %s", where, cudaGetErrorString(e));
   return L2PD_ERR_CUDA;
@@ -1021,8 +1040,10 @@ static l2pd_status standalone_cuda_error(const char *where, cudaError_t e) {
 
 static int32_t *standalone_status() {
   static int32_t *p[64] = {};
+  static std::mutex mu;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
   if (!p[dev]) {
     if (cudaMalloc((void **)&p[dev], 4) != cudaSuccess) return nullptr;
     cudaMemset(p[dev], 0, 4);
@@ -1122,7 +1143,7 @@ l2pd_status l2pd_lm_head_bf16(void *stream, const void *A, const void *W, const 
   if (!A || !W || !d_scratch || !d_pred || !d_conf) return L2PD_ERR_ARG;
   if (R < 1 || V < 2 || K < 8 || (K % 8)) return L2PD_ERR_SHAPE;
   const int sms = device_sms();
-  const int tile_n = pick_tile_n(R, V, sms, 16, 256);
+  const int tile_n = lm_head_tile_n(R, V, K, sms);
   int32_t *status = standalone_status();
   if (!status) return L2PD_ERR_CUDA;
   TmaDesc ta, tb;

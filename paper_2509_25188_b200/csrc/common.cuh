@@ -160,7 +160,9 @@ l2pd_status make_tma_2d_bf16_strided(TmaDesc *out, const void *ptr, int64_t rows
 l2pd_status make_tma_out_3d(TmaDesc *out, void *ptr, bool fp32, int64_t rows, int64_t N, int tile_w);
 // The same for the columns [N - tail_w, N) alone, as one tile of width tail_w (rows are N elements apart).
 l2pd_status make_tma_out_tail(TmaDesc *out, void *ptr, bool fp32, int64_t rows, int64_t N, int tail_w);
-int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile);
+int lm_head_tile_n(int R, int V, int K, int num_sms);   // tile width of the LM-head GEMM (single CTAs)
+// what failed in the calling thread's last context-free call: reported by l2pd_last_error(NULL) (api.cu)
+void set_standalone_error(const char *fmt, ...);
 // How one GEMM is laid over the SMs: CTAs per tile (1, or 2 = a cta_group::2 pair on a 256-row tile),
 // tile width, K slices (residual epilogue only: slices add into X with vector reductions), and row
 // slabs per unit (2 = a unit covers two 128 * cta_group row slabs against one load of the weight

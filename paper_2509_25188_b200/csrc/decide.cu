@@ -30,7 +30,7 @@ __global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
   __shared__ int s_masked[MAX_S];
   __shared__ int s_unmask[MAX_S];
   __shared__ int s_commit[MAX_S];
-  __shared__ int s_any, s_e, s_left;
+  __shared__ int s_any, s_forced, s_e, s_left;
 
   grid_dep_launch();
   grid_dep_wait();
@@ -47,12 +47,26 @@ __global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
     int ix = 0x7fffffff;
     if (j < m.n_blk_rows) {
       int r = slot * s + j;
-      for (int t = lane; t < a.n_tiles; t += 32) {
-        float tm = a.part_m[(int64_t)t * a.rows_padded + r];
-        float ts = a.part_s[(int64_t)t * a.rows_padded + r];
-        int ti = a.part_i[(int64_t)t * a.rows_padded + r];
-        if (tm > mx) { sum = sum * expf(mx - tm) + ts; mx = tm; ix = ti; }
-        else { sum += ts * expf(tm - mx); if (tm == mx && ti < ix) ix = ti; }
+      // eight records per lane are requested before the first is folded in (the fold order is unchanged)
+      constexpr int U = 8;
+      for (int t0 = lane; t0 < a.n_tiles; t0 += 32 * U) {
+        float tm[U], ts[U];
+        int ti[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          const int t = t0 + 32 * u;
+          const bool in = t < a.n_tiles;
+          const int64_t o = (int64_t)(in ? t : t0) * a.rows_padded + r;
+          tm[u] = in ? a.part_m[o] : -INFINITY;
+          ts[u] = in ? a.part_s[o] : 0.f;
+          ti[u] = in ? a.part_i[o] : 0x7fffffff;
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          if (t0 + 32 * u >= a.n_tiles) break;
+          if (tm[u] > mx) { sum = sum * expf(mx - tm[u]) + ts[u]; mx = tm[u]; ix = ti[u]; }
+          else { sum += ts[u] * expf(tm[u] - mx); if (tm[u] == mx && ti[u] < ix) ix = ti[u]; }
+        }
       }
       for (int o = 16; o > 0; o >>= 1) {
         float om = __shfl_xor_sync(0xffffffffu, mx, o);
@@ -75,7 +89,7 @@ __global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
     s_masked[j] = a.masked[(int64_t)seq * a.G + g0 + j];
     s_unmask[j] = 0;
   }
-  if (threadIdx.x == 0) { s_any = 0; s_e = 0x7fffffff; s_left = 0; }
+  if (threadIdx.x == 0) { s_any = 0; s_forced = 0; s_e = 0x7fffffff; s_left = 0; }
   __syncthreads();
 
   // ---- filter ----------------------------------------------------------------------------------
@@ -131,21 +145,20 @@ __global__ void __launch_bounds__(1024) decide_kernel(DecideArgs a) {
     if (s_masked[j] && pass) { s_unmask[j] = 1; s_any = 1; }
   }
   __syncthreads();
-  int forced = 0;
-  if (!s_any) {
-    if (threadIdx.x == 0) {
-      int best = -1;
-      float bc = -1.f;
-      for (int j = 0; j < s; ++j)
-        if (s_masked[j] && s_conf[j] > bc) { bc = s_conf[j]; best = j; }
-      if (best >= 0) {
-        s_unmask[best] = 1; s_any = 2;
-        if (a.rule == 2) s_commit[best] = a.ref[(int64_t)seq * a.G + g0 + best];
-      }
+  // Nothing passed: thread 0 commits the most confident masked position.  s_any is not written after the barrier
+  // above, and every thread takes the barrier below, so all warps run the same number of barriers whatever they read.
+  if (threadIdx.x == 0 && s_any == 0) {
+    int best = -1;
+    float bc = -1.f;
+    for (int j = 0; j < s; ++j)
+      if (s_masked[j] && s_conf[j] > bc) { bc = s_conf[j]; best = j; }
+    if (best >= 0) {
+      s_unmask[best] = 1; s_forced = 1;
+      if (a.rule == 2) s_commit[best] = a.ref[(int64_t)seq * a.G + g0 + best];
     }
-    __syncthreads();
-    forced = (s_any == 2);
   }
+  __syncthreads();
+  const int forced = s_forced;
 
   // ---- commit in place ----------------------------------------------------------------------------
   if (threadIdx.x < s) {

@@ -18,6 +18,34 @@ __device__ __forceinline__ float block_sum(float v, float *red) {
   return t;
 }
 
+template <typename T> struct Vec8;
+template <> struct Vec8<bf16> {
+  uint4 raw;
+  __device__ __forceinline__ void load(const bf16 *p) { raw = *reinterpret_cast<const uint4 *>(p); }
+  __device__ __forceinline__ void store(bf16 *p) const { *reinterpret_cast<uint4 *>(p) = raw; }
+  __device__ __forceinline__ float get(int i) const {
+    const __nv_bfloat16 *h = reinterpret_cast<const __nv_bfloat16 *>(&raw);
+    return __bfloat162float(h[i]);
+  }
+  __device__ __forceinline__ void set(int i, float f) {
+    __nv_bfloat16 *h = reinterpret_cast<__nv_bfloat16 *>(&raw);
+    h[i] = __float2bfloat16_rn(f);
+  }
+};
+template <> struct Vec8<float> {
+  float4 a, b;
+  __device__ __forceinline__ void load(const float *p) {
+    a = *reinterpret_cast<const float4 *>(p);
+    b = *reinterpret_cast<const float4 *>(p + 4);
+  }
+  __device__ __forceinline__ void store(float *p) const {
+    *reinterpret_cast<float4 *>(p) = a;
+    *reinterpret_cast<float4 *>(p + 4) = b;
+  }
+  __device__ __forceinline__ float get(int i) const { return reinterpret_cast<const float *>(&a)[i]; }
+  __device__ __forceinline__ void set(int i, float f) { reinterpret_cast<float *>(&a)[i] = f; }
+};
+
 // x[row,:] = emb[token,:];  n[row,:] = x * g / sqrt(mean(x^2) + eps)
 template <typename T>
 __global__ void embed_rmsnorm_kernel(const int32_t *tokens, int64_t tok_stride, const SeqMeta *meta,
@@ -32,7 +60,34 @@ __global__ void embed_rmsnorm_kernel(const int32_t *tokens, int64_t tok_stride, 
   int tok = tokens[(int64_t)m.seq * tok_stride + pos];
   const T *e = emb + (int64_t)tok * d;
   float *xr = x + (int64_t)row * d;
+  T *nr = n + (int64_t)row * d;
   float ss = 0.f;
+  if ((d & 7) == 0) {
+    // 8 elements per access (16 bytes of bf16 / 32 of fp32); per thread the sum runs over its chunks in order and
+    // over the 8 elements of a chunk in order
+    const int d8 = d >> 3;
+    for (int c = threadIdx.x; c < d8; c += blockDim.x) {
+      Vec8<T> v;
+      v.load(e + 8 * c);
+      float f[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) { f[i] = v.get(i); ss += f[i] * f[i]; }
+      *reinterpret_cast<float4 *>(xr + 8 * c) = make_float4(f[0], f[1], f[2], f[3]);
+      *reinterpret_cast<float4 *>(xr + 8 * c + 4) = make_float4(f[4], f[5], f[6], f[7]);
+    }
+    const float tot = block_sum(ss, red);
+    const float inv = 1.0f / sqrtf(tot / (float)d + eps);
+    for (int c = threadIdx.x; c < d8; c += blockDim.x) {
+      Vec8<T> v, o;
+      v.load(e + 8 * c);
+      const float4 g0 = *reinterpret_cast<const float4 *>(gain + 8 * c), g1 = *reinterpret_cast<const float4 *>(gain + 8 * c + 4);
+      const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+#pragma unroll
+      for (int i = 0; i < 8; ++i) o.set(i, v.get(i) * g[i] * inv);
+      o.store(nr + 8 * c);
+    }
+    return;
+  }
   for (int i = threadIdx.x; i < d; i += blockDim.x) {
     float v = to_f32(e[i]);
     xr[i] = v;
@@ -40,7 +95,6 @@ __global__ void embed_rmsnorm_kernel(const int32_t *tokens, int64_t tok_stride, 
   }
   float tot = block_sum(ss, red);
   float inv = 1.0f / sqrtf(tot / (float)d + eps);
-  T *nr = n + (int64_t)row * d;
   for (int i = threadIdx.x; i < d; i += blockDim.x)
     nr[i] = from_f32<T>(to_f32(e[i]) * gain[i] * inv);
 }
@@ -126,34 +180,6 @@ __global__ void __launch_bounds__(256) add_partials_kernel(float *x, const float
     reinterpret_cast<float4 *>(x)[i] = w;
   }
 }
-
-template <typename T> struct Vec8;
-template <> struct Vec8<bf16> {
-  uint4 raw;
-  __device__ __forceinline__ void load(const bf16 *p) { raw = *reinterpret_cast<const uint4 *>(p); }
-  __device__ __forceinline__ void store(bf16 *p) const { *reinterpret_cast<uint4 *>(p) = raw; }
-  __device__ __forceinline__ float get(int i) const {
-    const __nv_bfloat16 *h = reinterpret_cast<const __nv_bfloat16 *>(&raw);
-    return __bfloat162float(h[i]);
-  }
-  __device__ __forceinline__ void set(int i, float f) {
-    __nv_bfloat16 *h = reinterpret_cast<__nv_bfloat16 *>(&raw);
-    h[i] = __float2bfloat16_rn(f);
-  }
-};
-template <> struct Vec8<float> {
-  float4 a, b;
-  __device__ __forceinline__ void load(const float *p) {
-    a = *reinterpret_cast<const float4 *>(p);
-    b = *reinterpret_cast<const float4 *>(p + 4);
-  }
-  __device__ __forceinline__ void store(float *p) const {
-    *reinterpret_cast<float4 *>(p) = a;
-    *reinterpret_cast<float4 *>(p + 4) = b;
-  }
-  __device__ __forceinline__ float get(int i) const { return reinterpret_cast<const float *>(&a)[i]; }
-  __device__ __forceinline__ void set(int i, float f) { reinterpret_cast<float *>(&a)[i] = f; }
-};
 
 // Rotates q and k (pair (i, i+dh/2) by the tabulated angle of the row's position) and writes
 // q to the packed query buffer and k, v to the key/value store at [sequence, position].
@@ -259,6 +285,35 @@ __global__ void final_norm_gather_kernel(const float *x, const SeqMeta *meta, co
   int row = m.row0 + (m.blk_start - m.pos0) + j;
   const float *xr = x + (int64_t)row * d;
   float ss = 0.f;
+  if ((d & 3) == 0) {
+    // four elements per access; the row stays in registers between the two passes when it fits
+    const int d4 = d >> 2;
+    const float4 *x4 = reinterpret_cast<const float4 *>(xr), *g4 = reinterpret_cast<const float4 *>(gain);
+    constexpr int CACHE = 4;
+    float4 v[CACHE];
+#pragma unroll
+    for (int k = 0; k < CACHE; ++k) {
+      const int i = threadIdx.x + k * blockDim.x;
+      v[k] = i < d4 ? x4[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+      ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+    }
+    for (int i = threadIdx.x + CACHE * blockDim.x; i < d4; i += blockDim.x) {
+      const float4 w = x4[i];
+      ss += w.x * w.x + w.y * w.y + w.z * w.z + w.w * w.w;
+    }
+    const float tot = block_sum(ss, red);
+    const float inv = 1.0f / sqrtf(tot / (float)d + eps);
+#pragma unroll
+    for (int k = 0; k < CACHE; ++k) {
+      const int i = threadIdx.x + k * blockDim.x;
+      if (i < d4) { const float4 g = g4[i]; store4(out + 4 * i, v[k].x * g.x * inv, v[k].y * g.y * inv, v[k].z * g.z * inv, v[k].w * g.w * inv); }
+    }
+    for (int i = threadIdx.x + CACHE * blockDim.x; i < d4; i += blockDim.x) {
+      const float4 w = x4[i], g = g4[i];
+      store4(out + 4 * i, w.x * g.x * inv, w.y * g.y * inv, w.z * g.z * inv, w.w * g.w * inv);
+    }
+    return;
+  }
   for (int i = threadIdx.x; i < d; i += blockDim.x) { float v = xr[i]; ss += v * v; }
   float tot = block_sum(ss, red);
   float inv = 1.0f / sqrtf(tot / (float)d + eps);

@@ -512,10 +512,7 @@ GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, 
   return best;
 }
 
-int pick_tile_n(int M, int N, int num_sms, int multiple, int max_tile) {
-  (void)multiple; (void)max_tile;
-  return plan_gemm(EPI_LMHEAD, M, N, 4096, num_sms, 0).tile_n;
-}
+int lm_head_tile_n(int R, int V, int K, int num_sms) { return plan_gemm(EPI_LMHEAD, R, V, K, num_sms, 0).tile_n; }
 
 int effective_k_splits(int K, int k_splits) {
   // every K slice must hold at least one k-block (an empty slice would add an unwritten accumulator)

@@ -13,7 +13,7 @@ constexpr int64_t STATIC_SCRATCH_ELEMS = 3ll * STATIC_MAX_TILES * STATIC_MAX_ROW
 
 // Resident on every GPU that loads the library, from load until the process exits.
 static __device__ __align__(256) float g_lm_scratch[STATIC_SCRATCH_ELEMS];
-static __device__ __align__(256) int32_t g_lm_status[64];
+static __device__ __align__(256) int32_t g_lm_status[1];   // one word per device image
 
 // In host code the names above are host-side handles, not device addresses: the addresses the
 // kernels get come from cudaGetSymbolAddress, looked up once per device with that device current.
@@ -44,38 +44,39 @@ using namespace l2pd;
 extern "C" l2pd_status l2pd_lm_head_bf16_static(void *stream, const void *A, const void *W, const float *bias,
                                                 int32_t R, int32_t V, int32_t K, int32_t *d_pred, float *d_conf,
                                                 int32_t check) {
-  if (!A || !W || !d_pred || !d_conf) return L2PD_ERR_ARG;
-  if (R < 1 || V < 2 || K < 8 || (K % 8)) return L2PD_ERR_SHAPE;
-  if (R > STATIC_MAX_ROWS || V > 64 * STATIC_MAX_TILES) return L2PD_ERR_SHAPE;   // beyond the built-in scratch
+  auto bad = [](l2pd_status st, const char *what) { set_standalone_error("l2pd_lm_head_bf16_static: %s", what); return st; };
+  if (!A || !W || !d_pred || !d_conf) return bad(L2PD_ERR_ARG, "null pointer");
+  if (R < 1 || V < 2 || K < 8 || (K % 8)) return bad(L2PD_ERR_SHAPE, "R >= 1, V >= 2, K a positive multiple of 8");
+  if (R > STATIC_MAX_ROWS || V > 64 * STATIC_MAX_TILES) return bad(L2PD_ERR_SHAPE, "beyond the built-in scratch (R <= 128, V <= 131072)");
   int dev = 0, sms = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return L2PD_ERR_CUDA;
-  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return L2PD_ERR_CUDA;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return bad(L2PD_ERR_CUDA, "no current device");
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return bad(L2PD_ERR_CUDA, "device attribute query failed");
   DevicePtrs ptr;
   l2pd_status r = device_ptrs(dev, &ptr);
-  if (r != L2PD_OK) return r;
-  const int tile_n = pick_tile_n(R, V, sms, 16, 256);
+  if (r != L2PD_OK) return bad(r, "cudaGetSymbolAddress failed for the built-in scratch");
+  const int tile_n = lm_head_tile_n(R, V, K, sms);
   const int n_tiles = ceil_div(V, tile_n);
   const int rows_padded = STATIC_MAX_ROWS;
-  if (tile_n < 64 || n_tiles > STATIC_MAX_TILES) return L2PD_ERR_SHAPE;
+  if (tile_n < 64 || n_tiles > STATIC_MAX_TILES) return bad(L2PD_ERR_SHAPE, "tile records exceed the built-in scratch");
   TmaDesc ta, tb;
   r = make_tma_2d_bf16(&ta, A, R, K, 128);
-  if (r) return r;
+  if (r) return bad(r, "tensor map of A (16-byte aligned pointer, K a multiple of 8)");
   r = make_tma_2d_bf16(&tb, W, V, K, tile_n);
-  if (r) return r;
+  if (r) return bad(r, "tensor map of W (16-byte aligned pointer, K a multiple of 8)");
   cudaStream_t s = (cudaStream_t)stream;
   // the status word must start at zero; every record the merge reads is rewritten by this call
-  if (cudaMemsetAsync(ptr.status + dev, 0, sizeof(int32_t), s) != cudaSuccess) return L2PD_ERR_CUDA;
+  if (cudaMemsetAsync(ptr.status, 0, sizeof(int32_t), s) != cudaSuccess) return bad(L2PD_ERR_CUDA, "clearing the status word failed");
   GemmArgs g{};
   g.epi = EPI_LMHEAD; g.a = &ta; g.b = &tb; g.M = R; g.N = V; g.K = K; g.tile_n = tile_n;
   g.bias = bias; g.part_m = ptr.scratch; g.part_s = ptr.scratch + (int64_t)n_tiles * rows_padded;
   g.part_i = reinterpret_cast<int32_t *>(g.part_s + (int64_t)n_tiles * rows_padded);
-  g.rows_padded = rows_padded; g.logits = nullptr; g.status = ptr.status + dev;
-  if (launch_gemm_tcgen05(s, g, sms) != cudaSuccess) return L2PD_ERR_CUDA;
+  g.rows_padded = rows_padded; g.logits = nullptr; g.status = ptr.status;
+  if (launch_gemm_tcgen05(s, g, sms) != cudaSuccess) return bad(L2PD_ERR_CUDA, "GEMM launch failed");
   if (launch_merge_partials(s, g.part_m, g.part_s, g.part_i, n_tiles, rows_padded, R, d_pred, d_conf) != cudaSuccess)
-    return L2PD_ERR_CUDA;
+    return bad(L2PD_ERR_CUDA, "merge launch failed");
   if (!check) return L2PD_OK;
   int32_t h = 0;
-  if (cudaMemcpyAsync(&h, ptr.status + dev, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return L2PD_ERR_CUDA;
-  if (cudaStreamSynchronize(s) != cudaSuccess) return L2PD_ERR_CUDA;
-  return h == DEV_OK ? L2PD_OK : L2PD_ERR_TIMEOUT;
+  if (cudaMemcpyAsync(&h, ptr.status, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess) return bad(L2PD_ERR_CUDA, "status read-back failed");
+  if (cudaStreamSynchronize(s) != cudaSuccess) return bad(L2PD_ERR_CUDA, "stream synchronisation failed");
+  return h == DEV_OK ? L2PD_OK : bad(L2PD_ERR_TIMEOUT, "a bounded device wait ran out");
 }

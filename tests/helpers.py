@@ -37,6 +37,17 @@ def identity_filter(s: int, k: float, b: float):
 # ------------------------------------------------------------------------------------------------
 # GPU-vs-oracle lockstep (used by the -m gpu tests)
 
+def conf_interval(conf, eps):
+    """Eq. 4 under a bounded logit error: conf = p_top; if every logit of the row is off by at most eps, the odds
+    p_top / (1 - p_top) change by a factor within [exp(-2 eps), exp(2 eps)] (numerator by exp(+-eps), every term of the
+    rest by exp(-+eps)), and a changed argmax stays inside the same interval.  Returns (lo, hi) per row."""
+    c = np.clip(np.asarray(conf, dtype=np.float64), 1e-300, 1.0)
+    e = np.asarray(eps, dtype=np.float64)
+    odds = c / np.maximum(1.0 - c, 1e-300)
+    lo = 1.0 / (1.0 + np.exp(2 * e) / odds)
+    hi = 1.0 / (1.0 + np.exp(-2 * e) / odds)
+    return lo, hi
+
 def _sync_oracle_state(st, m, toks, msk, l_eff, done, cur_block):
     st.tokens[:] = toks
     st.masked[:] = msk
@@ -53,7 +64,12 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
     """Runs the CUDA decoder step by step; before every step the oracle is put in the decoder's
     state (teacher forcing), then both take the step and are compared:
       logits  |gpu - orc| <= logit_rtol * max|orc row|
-      conf    |gpu - orc| <= conf_atol
+      conf    within conf_atol of the interval the row's measured logit error allows: if every logit of the row
+              moves by at most eps, the odds of the top class move by a factor in [exp(-2 eps), exp(2 eps)], i.e.
+              conf_gpu lies in [sigmoid(L - 2 eps), sigmoid(L + 2 eps)] with L = logit(conf_orc) (Eq. 4; exact, not
+              first order, and it also covers a changed argmax).  Where that interval is narrower than conf_atol
+              (peaked or flat rows, small eps) the check is conf_atol absolute.  Without logits (check_logits off)
+              it is |gpu - orc| <= conf_atol.
       pred    equal wherever the oracle's top-2 logit gap exceeds 2 * logit_rtol * max|orc row|
       unmask  equal to the oracle's wherever every |p - tau| of the block exceeds p_margin (and, on a
               forced step, the two best confidences differ by more than conf_margin, default
@@ -70,9 +86,6 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
     """
     import copy
 
-    if conf_margin is None:
-        conf_margin = 2 * conf_atol
-
     def boundary_distance(r, blk_masked, n):
         if cfg.rule == "filter":
             return np.abs(r.p - cfg.tau)[blk_masked]
@@ -86,7 +99,8 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
     dec.state_reset(prompts, G)
     states = [orc.init_state(m, p, G) for p in prompts]
     stat = dict(steps=0, rows=0, pred_checked=0, unmask_checked=0, replay_checked=0, forced=0,
-                max_logit_rel=0.0, max_conf_err=0.0, seq_steps=[0] * B, oracle_steps=0, trace=[])
+                max_logit_rel=0.0, max_logit_abs=0.0, max_conf_err=0.0, max_conf_excess=0.0, max_conf_allowed=0.0,
+                seq_steps=[0] * B, oracle_steps=0, trace=[])
     while dec.num_active > 0:
         if max_steps is not None and stat["steps"] >= max_steps:
             break
@@ -115,13 +129,28 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
                 stat["oracle_steps"] += 1
                 assert rec.block == blk and rec.n_rows == n
                 row_max = np.abs(rec.logits).max(axis=-1)
-                if check_logits:
-                    err = np.abs(out["logits"][i, :n] - rec.logits).max(axis=-1) / row_max
-                    stat["max_logit_rel"] = max(stat["max_logit_rel"], float(err.max()))
-                    assert err.max() <= logit_rtol, "logits off by %g (rel) at step %d" % (err.max(), stat["steps"])
                 cerr = np.abs(out["conf"][i, :n] - rec.conf)
                 stat["max_conf_err"] = max(stat["max_conf_err"], float(cerr.max()))
-                assert cerr.max() <= conf_atol, "confidence off by %g at step %d" % (cerr.max(), stat["steps"])
+                step_conf_margin = conf_margin
+                if check_logits:
+                    eps = np.abs(out["logits"][i, :n] - rec.logits).max(axis=-1)
+                    err = eps / row_max
+                    stat["max_logit_rel"] = max(stat["max_logit_rel"], float(err.max()))
+                    stat["max_logit_abs"] = max(stat["max_logit_abs"], float(eps.max()))
+                    assert err.max() <= logit_rtol, "logits off by %g (rel) at step %d" % (err.max(), stat["steps"])
+                    lo, hi = conf_interval(rec.conf, eps)
+                    g = out["conf"][i, :n].astype(np.float64)
+                    excess = np.maximum(np.maximum(lo - g, g - hi), 0.0)
+                    stat["max_conf_excess"] = max(stat["max_conf_excess"], float(excess.max()))
+                    stat["max_conf_allowed"] = max(stat["max_conf_allowed"], float(np.maximum(hi - rec.conf, rec.conf - lo).max()))
+                    assert excess.max() <= conf_atol, ("confidence outside what the row's logit error allows by %g at step %d"
+                                                       % (excess.max(), stat["steps"]))
+                    if step_conf_margin is None:   # two confidences are told apart only beyond twice what their rows allow
+                        step_conf_margin = 2 * (float(np.maximum(hi - rec.conf, rec.conf - lo).max()) + conf_atol)
+                else:
+                    assert cerr.max() <= conf_atol, "confidence off by %g at step %d" % (cerr.max(), stat["steps"])
+                if step_conf_margin is None:
+                    step_conf_margin = 2 * conf_atol
                 sure = rec.gap > 2 * logit_rtol * row_max
                 stat["pred_checked"] += int(sure.sum())
                 assert np.array_equal(out["pred"][i, :n][sure], rec.pred[sure])
@@ -153,7 +182,7 @@ def lockstep(dec, m, filt, cfg, prompts, G, *, logit_rtol, conf_atol, p_margin, 
                 clear = bool(sure.all())
             if rec.forced:
                 cm = np.sort(rec.conf[blk_masked[:n]])[::-1]
-                clear = clear and (len(cm) < 2 or cm[0] - cm[1] > conf_margin)
+                clear = clear and (len(cm) < 2 or cm[0] - cm[1] > step_conf_margin)
             if clear:
                 stat["unmask_checked"] += 1
                 assert np.array_equal(out["unmask"][i].astype(bool), rec.unmask), "unmask decision differs"

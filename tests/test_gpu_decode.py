@@ -258,6 +258,28 @@ def test_errors_come_back_as_status_codes():
         b.Decoder(shape, w, filt, block_len=65, max_batch=1, max_seq=96)
 
 
+def test_device_timeout_status_maps_to_an_error_and_the_context_recovers():
+    """A kernel whose bounded wait runs out leaves a code in the context's status word; the host turns it into
+    L2PD_ERR_TIMEOUT, clears it, and the context stays usable.  The word is preset through the test hook: no kernel is
+    made to wait."""
+    b = _b()
+    shape, w = _tiny()
+    d = wl.DECODES["C0"]
+    filt = wl.make_filter(d.block_len, d.tau, seed=0)
+    prompts = wl.make_prompts(1, d.prompt_len, shape, seed=1)
+    dec = _decoder(shape, w, filt)
+    want, _, steps, _ = dec.decode(prompts, d.gen_len)
+    dec.state_reset(prompts, d.gen_len)
+    dec.debug_set_device_status(2)
+    with pytest.raises(b.L2pdError) as e:
+        dec.denoise_step()
+    assert e.value.status == -5 and "role 2" in str(e.value)
+    # the word was cleared: the same context decodes again, with the same result
+    got, _, steps2, _ = dec.decode(prompts, d.gen_len)
+    assert np.array_equal(got, want) and steps2[0] == steps[0]
+    dec.close()
+
+
 # ----------------------------------------------------------------------------- bf16 tensor-core path
 
 def _bf16_shape(**kw):
@@ -280,12 +302,36 @@ def test_bf16_small_model_lockstep(spread, kv_cache):
     b = _b()
     dec = b.Decoder(shape, w, filt, block_len=s, max_batch=B, max_seq=P + G, kv_cache=kv_cache,
                     lm_head_bias=m.lm_head_bias)
-    # spread logits (std ~ 6) turn a 2e-2-relative logit error into a visible confidence error:
-    # |d conf| <= conf (1 - conf) |d logit| <= 0.25 * 2e-2 * max|logit|
-    conf_atol = 1e-3 if not spread else 0.05
-    st = lockstep(dec, m, filt, cfg, prompts, G, logit_rtol=2e-2, conf_atol=conf_atol,
+    # confidence: 1e-3 beyond what each row's measured logit error allows (helpers.conf_interval)
+    st = lockstep(dec, m, filt, cfg, prompts, G, logit_rtol=2e-2, conf_atol=1e-3,
                   p_margin=0.02 if not spread else 0.3)
+    print("bf16 small model spread=%s kv_cache=%d: max logit err rel %.2e abs %.3f, max conf err %.4f (allowed by the rows' logit "
+          "errors: %.4f, excess %.1e)" % (spread, kv_cache, st["max_logit_rel"], st["max_logit_abs"], st["max_conf_err"],
+                                         st["max_conf_allowed"], st["max_conf_excess"]))
     assert st["max_logit_rel"] < 2e-2
     assert st["replay_checked"] >= 0.9 * sum(st["seq_steps"])
     assert st["unmask_checked"] > 0
+    dec.close()
+
+
+@pytest.mark.parametrize("kv_cache", [1, 2])
+def test_bf16_six_layers_three_sequences_cached_lockstep(kv_cache):
+    """The key/value store at depth: six layers and three sequences, so that layer strides (layers 2..5) and sequence
+    strides of the store are exercised together, every step compared with the oracle run under the same caching rule;
+    an [EoT] bias cuts the sequences at different places (cached steps then run on shortened inputs)."""
+    shape = _bf16_shape(n_layers=6)
+    w = wl.make_weights(shape, seed=2, final_norm_gain=wl.spread_gain(shape))
+    s, P, G, B = 32, 72, 96, 3
+    filt = wl.make_filter(s, 0.96, seed=1)
+    prompts = wl.make_prompts(B, P, shape, seed=41)
+    m = oracle_model(shape, w, lm_head_bias=wl.make_eot_bias(shape, 6.0))
+    cfg = orc.DecodeConfig(block_len=s, kv_cache=True, dual_cache=kv_cache == 2)
+    dec = _b().Decoder(shape, w, filt, block_len=s, max_batch=B, max_seq=P + G, kv_cache=kv_cache, lm_head_bias=m.lm_head_bias)
+    st = lockstep(dec, m, filt, cfg, prompts, G, logit_rtol=2e-2, conf_atol=1e-3, p_margin=0.3)
+    cached_steps = sum(1 for t in st["trace"]) - len({int(b) for t in st["trace"] for b in np.asarray(t["block"]) if b >= 0})
+    print("six layers kv_cache=%d: %d steps (%d oracle), max logit err rel %.2e, max conf err %.4f (allowed %.4f)"
+          % (kv_cache, st["steps"], st["oracle_steps"], st["max_logit_rel"], st["max_conf_err"], st["max_conf_allowed"]))
+    assert st["oracle_steps"] == sum(st["seq_steps"]) and st["max_logit_rel"] < 2e-2
+    assert cached_steps >= 3                      # most steps read the store
+    assert st["replay_checked"] >= 0.9 * sum(st["seq_steps"])
     dec.close()

@@ -67,3 +67,24 @@ def test_two_ranks_reproduce_the_single_process_batch():
     assert np.array_equal(got[0], toks) and np.array_equal(got[1], out_len) and np.array_equal(got[2], steps)
     assert got[3] == 11.0                      # MAX over ranks
     assert got[4] == float(out_len.sum())      # SUM over ranks
+
+
+def test_spawned_ranks_pull_chunks_from_the_queue_and_gather(tmp_path):
+    """The path bench.py --gpus N takes when no launcher started it: replicas.spawn_local_ranks starts the ranks
+    (here two gloo ranks on CPU), the ranks take chunks of the batch from the shared queue until none is left
+    (over-decomposition: rank 0 is slowed down, so rank 1 ends up with more of them), and the gathered result
+    equals the single-process decode of the whole batch."""
+    sys.path.insert(0, ROOT)
+    from paper_2509_25188_b200 import replicas, workloads as wl
+    from tests.helpers import small_shape
+    B, P, G, s, chunk = 7, 6, 16, 4, 2         # four chunks (2, 2, 2, 1 sequences) for two ranks
+    out = str(tmp_path / "gathered.npz")
+    rc = replicas.spawn_local_ranks(2, os.path.join(ROOT, "tests", "multi_rank_worker.py"),
+                                    [out, str(B), str(P), str(G), str(s), str(chunk)],
+                                    extra_env={"OMP_NUM_THREADS": "2"}, timeout=600)
+    assert rc == 0
+    got = np.load(out)
+    toks, out_len, steps = _decode_share(wl.make_prompts(B, P, small_shape(), seed=7), G, s)
+    assert np.array_equal(got["toks"], toks) and np.array_equal(got["out_len"], out_len) and np.array_equal(got["steps"], steps)
+    assert int(got["world"]) == 2 and float(got["decoded"]) == B and float(got["ms"]) == 11.0
+    assert 0 < int(got["mine"]) < B            # both ranks took part

@@ -583,6 +583,66 @@ def test_dual_cache_two_layers_brute_force_and_eotp():
     assert later >= 2 and 0 <= st.eot_pos < G - 1            # cut before the end
 
 
+def test_prefix_cache_two_layers_later_steps_by_hand_with_eotp():
+    """Two layers, prefix rule: a later step of a block equals a by-hand evaluation of the rows from the
+    block start to L_eff in which the keys and values of the positions BEFORE the block are those the
+    block's first step stored, layer by layer (layer 1's equal the fresh ones, layer 2's are stale: they
+    were computed when the block was still all masks), and the keys and values of the rows from the block
+    start on are fresh.  An [EoT] bias cuts the sequence, so some later steps run on a shortened input."""
+    shape, m = _cache_models(2)
+    s, G = 4, 12
+    filt = const_filter(s, -50.0)
+    cfg = orc.DecodeConfig(block_len=s, kv_cache=True)
+    seed, bias, _ = find_eot_bias(m, shape, filt, G, cfg, 5, grid=np.arange(5.0, 120.0, 5.0))
+    m.lm_head_bias = wl.make_eot_bias(shape, bias)
+    p = wl.make_prompts(1, 5, shape, seed=seed)[0]
+    st = orc.init_state(m, p, G)
+    H, dh = m.n_heads, m.head_dim
+    layers = m.weights["layers"]
+    stored = None
+    later = shortened = stale_seen = 0
+    while not st.done:
+        first = st.cache_block != st.cur_block
+        S_b = st.P + st.cur_block * s
+        L = st.L_eff
+        n = min(s, L - S_b)
+        pos = np.arange(L)
+        x0 = orc.widen(m.weights["tok_emb"][st.tokens[:L]])
+        if first:
+            kv1, kv2 = [], []
+            x1 = orc.layer_forward(m, layers[0], x0, pos, kv_out=kv1)
+            x2 = orc.layer_forward(m, layers[1], x1, pos, kv_out=kv2)
+            stored = [(kv1[0][0][:S_b], kv1[0][1][:S_b]), (kv2[0][0][:S_b], kv2[0][1][:S_b])]
+            stored_len = L
+            want = orc.lm_head_logits(m, x2[S_b: S_b + n])
+        else:
+            later += 1
+            shortened += int(L < stored_len)
+            rows = slice(S_b, L)
+            xr = x0[rows]
+            for li, layer in enumerate(layers):
+                nn = orc.rmsnorm(xr, layer["norm1"], m.rms_eps)
+                qkv = orc.linear(nn, layer["wqkv"])
+                T = L - S_b
+                q = orc.rope(qkv[:, : H * dh].reshape(T, H, dh), pos[rows], m.rope_theta)
+                kf = orc.rope(qkv[:, H * dh: 2 * H * dh].reshape(T, H, dh), pos[rows], m.rope_theta)
+                vf = qkv[:, 2 * H * dh:].reshape(T, H, dh)
+                k_all = np.concatenate([stored[li][0], kf])
+                v_all = np.concatenate([stored[li][1], vf])
+                xo = xr + orc.linear(orc.attention(q, k_all, v_all).reshape(T, H * dh), layer["wo"])
+                nn = orc.rmsnorm(xo, layer["norm2"], m.rms_eps)
+                xr = xo + orc.linear(orc.silu(orc.linear(nn, layer["w_gate"])) * orc.linear(nn, layer["w_up"]), layer["w_down"])
+            want = orc.lm_head_logits(m, xr[:n])
+            # layer 2's stored prefix keys really are stale: they differ from what a full forward gives now
+            kv_now = []
+            orc.forward_hidden(m, st.tokens[:L], kv_out=kv_now)
+            assert np.allclose(kv_now[0][0][:S_b], stored[0][0], atol=1e-12)      # layer 1: token-only, never stale
+            stale_seen += int(np.abs(kv_now[1][0][:S_b] - stored[1][0]).max() > 1e-8)
+        rec = orc.denoise_step(m, filt, st, cfg, keep_logits=True)
+        assert rec.n_rows == n and np.allclose(rec.logits, want, atol=1e-9)
+    assert later >= 2 and stale_seen >= 1 and 0 <= st.eot_pos < G - 1
+
+
 # ----------------------------------------------------------------------------- planted mistakes
 
 def test_planted_mistakes_are_caught(monkeypatch):

@@ -5,8 +5,10 @@ owned by an arena set up at start, or is fully committed to weights and caches. 
 library keeps the LM head's per-tile reduction records in a fixed array of its own.  This test calls
 that entry point through the C ABI twice in a row, on different inputs, and checks both results
 against l2pd_lm_head_bf16 (same kernels, caller-provided scratch): predictions identical,
-confidences within the 1e-6 the kernel tests use for identical arithmetic.  It is collected last so
-that a run stopping at the first failure has already run everything else; it also passes alone.
+confidences within the 1e-6 the kernel tests use for identical arithmetic — and against the CPU
+oracle's Eq. 3-4 on the same inputs, with the checks the LM-head kernel test applies (ids where the
+top-2 logit gap is clear, confidences to 1e-3).  It is collected last so that a run stopping at the
+first failure has already run everything else; it also passes alone.
 """
 from __future__ import annotations
 
@@ -14,16 +16,22 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import l2pd_oracle as orc
 from paper_2509_25188_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
 
 
-def _case(b, seed, R, V, K, with_bias):
-    A = b.to_device(wl.make_activations(seed, 0, (R, K), 1.0, "bf16"))
-    W = b.to_device(wl.make_activations(seed, 1, (V, K), 0.3, "bf16"))
-    bias = b.to_device(wl.make_activations(seed, 2, (V,), 1.0, "fp32")) if with_bias else None
+def _host_case(seed, R, V, K, with_bias):
+    A = wl.make_activations(seed, 0, (R, K), 1.0, "bf16")
+    W = wl.make_activations(seed, 1, (V, K), 0.3, "bf16")
+    bias = wl.make_activations(seed, 2, (V,), 1.0, "fp32") if with_bias else None
     return A, W, bias
+
+
+def _case(b, seed, R, V, K, with_bias):
+    A, W, bias = _host_case(seed, R, V, K, with_bias)
+    return b.to_device(A), b.to_device(W), (b.to_device(bias) if with_bias else None)
 
 
 def test_static_scratch_entry_point_matches_twice_in_a_row():
@@ -43,6 +51,16 @@ def test_static_scratch_entry_point_matches_twice_in_a_row():
         assert np.array_equal(pred[:R].cpu().numpy(), want_pred.cpu().numpy()), "call %d" % call
         assert np.abs(conf[:R].cpu().numpy() - want_conf.cpu().numpy()).max() <= 1e-6, "call %d" % call
         assert (pred[R:] == -7).all() and (conf[R:] == -1.0).all()      # nothing written past R rows
+        # the oracle on the same bytes: Eq. 3 where the top-2 gap is clear, Eq. 4 to 1e-3
+        hA, hW, hbias = _host_case(seed, R, V, K, with_bias)
+        ref = orc.linear(orc.widen(hA), hW)
+        if with_bias:
+            ref = ref + hbias.astype(np.float64)[None, :]
+        rp, rc, gap = orc.confidence_head(ref)
+        sure = gap > 1e-3 * np.abs(ref).max()
+        assert sure.mean() > 0.5
+        assert np.array_equal(pred[:R].cpu().numpy()[sure], rp[sure]), "call %d: ids differ from the oracle" % call
+        assert np.abs(conf[:R].cpu().numpy() - rc)[sure].max() < 1e-3, "call %d: confidences differ from the oracle" % call
         if call > 0:
             assert after == before      # once the kernels are loaded, a call takes no device memory
 
