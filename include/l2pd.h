@@ -279,14 +279,18 @@ l2pd_status l2pd_profile_enable(l2pd_ctx *ctx, uint32_t kind_mask);
 l2pd_status l2pd_profile_read(const l2pd_ctx *ctx, int32_t kind, double *ms_total, int64_t *launches);
 
 /*
- * Chained launches.  When every projection of a step runs on SM pairs with two row slabs per unit (a few
- * hundred to a few thousand rows, bf16, rotation fused into the QKV projection), the step runs, per layer, the
- * attention kernel and ONE persistent launch that holds the output projection, the RMSNorm before the MLP, the
- * gate/up and down projections and the next layer's RMSNorm and QKV projection; the results are bit-identical to
- * the one-launch-per-projection form.  l2pd_set_chain(ctx, 1) selects the chained form, 0 (the state after
- * l2pd_init) one launch per projection; it may be called between steps.  Measured at 512 rows the two forms
- * take the same time within a few percent (programmatic dependent launch already hides the launch and the
- * ring fill of a projection behind the one before it), hence the default.
+ * Chained launches.  A step whose projections all run on SM pairs (bf16; up to 1536 rows) can run, per layer, the
+ * attention kernel (preceded by the rotation / scatter kernel in the key/value-cache configurations) and ONE persistent
+ * launch that holds the output projection, the RMSNorm before the MLP, the gate/up and down projections and the next
+ * layer's RMSNorm and QKV projection: the weight loads of a projection then start while the one before it is still
+ * draining, which is what the small steps of the dual cache (a few dozen rows, bound by weight streaming) gain from.
+ * l2pd_set_chain(ctx, mode): 0 (the state after l2pd_init) one launch per projection; 1 chained launches where the step's
+ * shapes allow, one launch per projection elsewhere; 2 the chained form's tiling in single launches (for comparisons:
+ * modes 1 and 2 give bit-identical results).  With more than 256 rows the tiling does not depend on the mode, and all
+ * three modes agree bit for bit; with at most 256 rows modes 1 and 2 use one 256-row slab per unit with the two
+ * MMA-issuing threads on alternate k-blocks (key/value-cache configurations only).  May be called between steps.
+ * Measured at 512 rows the chained and the single-launch form take the same time within a few percent (programmatic
+ * dependent launch already hides the launch and the ring fill of a projection behind the one before it).
  * l2pd_chain_trace_enable(ctx, 1) makes every chained launch of the following steps record, per phase and CTA,
  * the nanosecond timer at which the CTA opened the phase, had its first and its last accumulator ready (for an
  * RMSNorm phase both equal the opening) and finished the phase; l2pd_chain_trace_read copies the last step's
@@ -294,7 +298,7 @@ l2pd_status l2pd_profile_read(const l2pd_ctx *ctx, int32_t kind, double *ms_tota
  * slots beyond a launch's phases hold stale values) and returns their count (call with h_out = NULL to size
  * the buffer; -1 on a CUDA error); it synchronises the device.  (0) frees the record buffer.
  */
-l2pd_status l2pd_set_chain(l2pd_ctx *ctx, int32_t enable);
+l2pd_status l2pd_set_chain(l2pd_ctx *ctx, int32_t mode);
 l2pd_status l2pd_chain_trace_enable(l2pd_ctx *ctx, int32_t enable);
 int64_t l2pd_chain_trace_read(l2pd_ctx *ctx, uint64_t *h_out, int64_t capacity, int32_t *launches, int32_t *phases,
                               int32_t *ctas);

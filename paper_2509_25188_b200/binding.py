@@ -327,9 +327,10 @@ class Decoder:
         _check(lib.l2pd_debug_set_device_status(self.ctx, _stream(), int(code)), self.ctx)
 
     # ---- chained launches ------------------------------------------------------------------------
-    def set_chain(self, enable: bool):
-        """False: one launch per projection; True (the default): one persistent launch per layer where the shapes allow."""
-        _check(lib.l2pd_set_chain(self.ctx, int(bool(enable))), self.ctx)
+    def set_chain(self, mode):
+        """0 / False: one launch per projection (the default); 1 / True: one persistent launch per layer where the step's
+        shapes allow; 2: the chained form's tiling in single launches (bit-identical to 1, for comparisons)."""
+        _check(lib.l2pd_set_chain(self.ctx, int(mode)), self.ctx)
 
     def chain_trace_enable(self, enable: bool = True):
         _check(lib.l2pd_chain_trace_enable(self.ctx, int(bool(enable))), self.ctx)

@@ -78,6 +78,9 @@ struct l2pd_ctx {
 
   // TMA descriptors (bf16 path)
   TmaDesc ta_n, ta_att, ta_h, ta_nf, ta_q, t_kstore, t_vstore;
+  // steps of at most 128 rows load only their rows: the same maps with a box of `a_box` rows (a_box_nf for the LM head's)
+  TmaDesc ta_n_s, ta_att_s, ta_h_s, ta_nf_s;
+  int a_box = 0, a_box_nf = 0;
   // output maps of the four projections (staged epilogue stores); re-encoded when rows or tile width change
   TmaDesc tc_qkv, tc_o, tc_h, tc_down;
   // the same for each projection's last, narrower column tile (chained launches stage every tile); tail width, 0 = none
@@ -91,7 +94,7 @@ struct l2pd_ctx {
 
   // several projections per launch (gemm_chain.cu): on when every projection of the step runs on SM pairs with
   // two row slabs per unit and K slices store partial sums
-  bool chain_on = false;             // l2pd_set_chain
+  int chain_mode = 0;                // l2pd_set_chain: 0 one launch per projection, 1 chained launches, 2 the chained form's tiling in single launches
   int chain_clusters = 0;            // CTA pairs that can be resident at once (0: kernel not usable here)
   unsigned int *d_chain_bar = nullptr;
   unsigned int chain_bar_base = 0;   // host copy of the counter's value
@@ -232,6 +235,10 @@ GemmArgs make_gemm_args(l2pd_ctx *c, int epi, const TmaDesc *a, const TmaDesc *b
   g.epi = epi; g.a = a; g.b = b; g.b2 = b2; g.c = cm; g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.out = out;
   g.cta_group = pl.cta_group; g.k_splits = pl.k_splits; g.slabs = pl.slabs; g.k_interleave = pl.k_interleave;
   g.status = c->d_status;
+  if (M <= 128 && pl.slabs == 1 && c->a_box > 0 && c->a_box < 128) {   // few rows: the map of the same buffer with the small box
+    g.a = a == &c->ta_n ? &c->ta_n_s : a == &c->ta_att ? &c->ta_att_s : a == &c->ta_h ? &c->ta_h_s : a;
+    if (g.a != a) g.a_box_rows = c->a_box;
+  }
   if (epi == EPI_QKV_ROPE) {
     g.rope_cols = 2 * c->cfg.n_heads * c->cfg.head_dim; g.rope_dh = c->cfg.head_dim;
     g.cs_table = c->cs_table_t; g.cs_stride = c->cfg.max_seq; g.row_pos = c->d_row_pos;
@@ -260,17 +267,40 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     // contexts that can chain the projections of a layer into one launch keep every tile at most CHAIN_TILE_N wide:
     // the chained kernel has one ring for all of them, and that width leaves it five stages
     const int max_tn = (c->chain_clusters > 0 && T_rows > 256 && T_rows <= CHAIN_MAX_ROWS && T_rows <= c->ksum_rows) ? CHAIN_TILE_N : 256;
-    c->pl_qkv = plan_gemm(EPI_STORE, T_rows, 3 * hd, d, c->num_sms, 0, 4, max_tn);
+    // steps of at most 256 rows chain with one row slab per unit (key/value-cache configurations: the rotation is a kernel
+    // of its own there); their tiling is used only when chaining is asked for
+    const bool small_chain = c->chain_mode != 0 && c->chain_clusters > 0 && c->ksum && T_rows <= 256 && !c->fuse_rope;
+    {
+      const int abox = T_rows <= 128 ? (int)round_up(T_rows, 8) : 128;
+      if (abox != c->a_box) {
+        if (abox < 128) {
+          const int64_t mr = c->max_rows;
+          if (make_tma_2d_bf16(&c->ta_n_s, c->n, mr, d, abox) || make_tma_2d_bf16(&c->ta_att_s, c->att, mr, hd, abox) ||
+              make_tma_2d_bf16(&c->ta_h_s, c->h, mr, F, abox))
+            return set_err(c, L2PD_ERR_CUDA, "tensor map encode failed (activation box of %d rows)", abox);
+        }
+        c->a_box = abox;
+        c->chain_tab_rows = -1;
+      }
+    }
+    const int max_ks = (c->ksum == nullptr || T_rows <= c->ksum_rows) ? 4 : 1;   // K slices need their partial-sum area
+    if (small_chain) {
+      c->pl_qkv = plan_gemm_pair_one_slab(EPI_STORE, T_rows, 3 * hd, d, c->num_sms, 1, CHAIN_TILE_N);
+      c->pl_o = plan_gemm_pair_one_slab(EPI_RESIDUAL, T_rows, d, hd, c->num_sms, max_ks, CHAIN_TILE_N);
+      c->pl_down = plan_gemm_pair_one_slab(EPI_RESIDUAL, T_rows, d, F, c->num_sms, max_ks, CHAIN_TILE_N);
+      c->pl_gu = plan_gemm_pair_one_slab(EPI_SWIGLU, T_rows, F, d, c->num_sms, 1, CHAIN_TILE_N);
+    } else {
+      c->pl_qkv = plan_gemm(EPI_STORE, T_rows, 3 * hd, d, c->num_sms, 0, 4, max_tn);
+      c->pl_o = plan_gemm(EPI_RESIDUAL, T_rows, d, hd, c->num_sms, 0, max_ks, max_tn);
+      c->pl_down = plan_gemm(EPI_RESIDUAL, T_rows, d, F, c->num_sms, 0, max_ks, max_tn);
+      c->pl_gu = plan_gemm(EPI_SWIGLU, T_rows, F, d, c->num_sms, 0, 4, max_tn);
+    }
     int box = c->pl_qkv.tile_n / c->pl_qkv.cta_group;
     if (box != c->box_qkv) { l2pd_status r = encode_weight_maps(c, c->tb_qkv, c->wqkv, 3 * hd, d, box); if (r) return r; c->box_qkv = box; }
-    const int max_ks = (c->ksum == nullptr || T_rows <= c->ksum_rows) ? 4 : 1;   // K slices need their partial-sum area
-    c->pl_o = plan_gemm(EPI_RESIDUAL, T_rows, d, hd, c->num_sms, 0, max_ks, max_tn);
     box = c->pl_o.tile_n / c->pl_o.cta_group;
     if (box != c->box_o) { l2pd_status r = encode_weight_maps(c, c->tb_o, c->wo, d, hd, box); if (r) return r; c->box_o = box; }
-    c->pl_down = plan_gemm(EPI_RESIDUAL, T_rows, d, F, c->num_sms, 0, max_ks, max_tn);
     box = c->pl_down.tile_n / c->pl_down.cta_group;
     if (box != c->box_down) { l2pd_status r = encode_weight_maps(c, c->tb_down, c->w_down, d, F, box); if (r) return r; c->box_down = box; }
-    c->pl_gu = plan_gemm(EPI_SWIGLU, T_rows, F, d, c->num_sms, 0, 4, max_tn);
     box = c->pl_gu.tile_n / 2;
     if (box != c->box_gu) {
       l2pd_status r = encode_weight_maps(c, c->tb_gate, c->w_gate, F, d, box); if (r) return r;
@@ -325,10 +355,12 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
   // The chained form of the layer loop: QKV of layer 0 alone, then per layer the attention kernel and ONE launch that
   // runs O, RMSNorm, gate/up, down and (but for the last layer) the next layer's RMSNorm and QKV.
   bool chain = false;
-  if (tc && c->chain_on && c->chain_clusters > 0 && c->ksum && !c->cap && f.n_layers > 0 && T_rows <= c->ksum_rows &&
-      T_rows <= CHAIN_MAX_ROWS && c->fuse_rope) {
-    auto two_slab_pair = [](const GemmPlan &p) { return p.cta_group == 2 && p.slabs == 2 && !p.k_interleave; };
-    chain = two_slab_pair(c->pl_qkv) && two_slab_pair(c->pl_o) && two_slab_pair(c->pl_gu) && two_slab_pair(c->pl_down) &&
+  const int epi_qkv = c->fuse_rope ? EPI_QKV_ROPE : EPI_STORE;
+  if (tc && c->chain_mode == 1 && c->chain_clusters > 0 && c->ksum && !c->cap && f.n_layers > 0 && T_rows <= c->ksum_rows &&
+      T_rows <= CHAIN_MAX_ROWS && (c->fuse_rope || c->attn_tc)) {
+    // SM pairs throughout: two row slabs per unit, or one slab with the two MMA issuers on alternate k-blocks
+    auto chainable = [](const GemmPlan &p) { return p.cta_group == 2 && ((p.slabs == 2 && !p.k_interleave) || (p.slabs == 1 && p.k_interleave)); };
+    chain = chainable(c->pl_qkv) && chainable(c->pl_o) && chainable(c->pl_gu) && chainable(c->pl_down) &&
             c->tcw_qkv > 0 && c->tcw_o > 0 && c->tcw_h > 0 && c->tcw_down > 0 &&
             c->tail_qkv >= 0 && c->tail_o >= 0 && c->tail_h >= 0 && c->tail_down >= 0;
   }
@@ -336,7 +368,7 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
   auto chain_gemm = [&](int which, int l) {
     ChainStep st{};
     switch (which) {
-      case 0: st.g = make_gemm_args(c, EPI_QKV_ROPE, &c->ta_n, &c->tb_qkv[l], nullptr, &c->tc_qkv, qkv, T_rows, 3 * hd, d, c->pl_qkv);
+      case 0: st.g = make_gemm_args(c, epi_qkv, &c->ta_n, &c->tb_qkv[l], nullptr, &c->tc_qkv, qkv, T_rows, 3 * hd, d, c->pl_qkv);
               st.g.c_tail = c->tail_qkv > 0 ? &c->tct_qkv : nullptr; st.g.tail_cols = c->tail_qkv; break;
       case 1: st.g = make_gemm_args(c, EPI_RESIDUAL, &c->ta_att, &c->tb_o[l], nullptr, &c->tc_o, c->x, T_rows, d, hd, c->pl_o);
               st.g.c_tail = c->tail_o > 0 ? &c->tct_o : nullptr; st.g.tail_cols = c->tail_o; break;
@@ -397,8 +429,18 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     };
     { l2pd_status r = launch_chain(0); if (r) return r; }
     for (int l = 0; l < f.n_layers; ++l) {
-      CKLK(L2PD_K_ATTENTION, launch_attention_tc(s, c->tq_packed, c->tk_packed, c->tv_packed, c->d_meta, (bf16 *)att, hd, 0, 0, 1,
-                                n_slots, max_q_rows, H, c->d_status));
+      if (c->fuse_rope) {
+        CKLK(L2PD_K_ATTENTION, launch_attention_tc(s, c->tq_packed, c->tk_packed, c->tv_packed, c->d_meta, (bf16 *)att, hd, 0, 0, 1,
+                                  n_slots, max_q_rows, H, c->d_status));
+      } else {
+        // key/value-cache configurations: rotation + scatter into the store, then attention over the store
+        T *kc = (T *)c->kc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
+        T *vc = (T *)c->vc + (f.kv_cache_mode ? (int64_t)l * c->kv_layer_stride : 0);
+        CKLK(L2PD_K_ROPE, launch_rope_scatter<T>(s, qkv, c->d_meta, c->d_row_slot, c->cs_table, q, kc, vc, c->kv_seq_stride, T_rows, H, dh));
+        const int kv_row_base = f.kv_cache_mode ? l * f.max_batch * f.max_seq : 0;
+        CKLK(L2PD_K_ATTENTION, launch_attention_tc(s, c->ta_q, c->t_kstore, c->t_vstore, c->d_meta, (bf16 *)att, hd, f.max_seq,
+                                  kv_row_base, 0, n_slots, max_q_rows, H, c->d_status));
+      }
       l2pd_status r = launch_chain(l + 1);
       if (r) return r;
     }
@@ -473,8 +515,13 @@ l2pd_status forward_and_decide(l2pd_ctx *c, cudaStream_t s, int n_slots, int T_r
     n_tiles = ceil_div(V, tn);
     part_m = c->part; part_s = part_m + (int64_t)n_tiles * rows_padded;
     part_i = (int32_t *)(part_s + (int64_t)n_tiles * rows_padded);
+    const int nf_box = R <= 128 ? (int)round_up(R, 8) : 128;
+    if (nf_box < 128 && nf_box != c->a_box_nf) {
+      if (make_tma_2d_bf16(&c->ta_nf_s, c->nf, c->max_lm_rows, d, nf_box)) return set_err(c, L2PD_ERR_CUDA, "tensor map encode failed for the LM head's rows");
+      c->a_box_nf = nf_box;
+    }
     GemmArgs g{};
-    g.epi = EPI_LMHEAD; g.a = &c->ta_nf; g.b = &c->tb_lm; g.M = R; g.N = V; g.K = d; g.tile_n = tn;
+    g.epi = EPI_LMHEAD; g.a = nf_box < 128 ? &c->ta_nf_s : &c->ta_nf; g.a_box_rows = nf_box; g.b = &c->tb_lm; g.M = R; g.N = V; g.K = d; g.tile_n = tn;
     g.bias = c->lm_bias; g.part_m = part_m; g.part_s = part_s; g.part_i = part_i; g.rows_padded = rows_padded;
     g.logits = nullptr; g.status = c->d_status;
     float *tmp_logits = nullptr;
@@ -985,9 +1032,12 @@ l2pd_status l2pd_debug_set_device_status(l2pd_ctx *c, void *stream, int32_t code
   return L2PD_OK;
 }
 
-l2pd_status l2pd_set_chain(l2pd_ctx *c, int32_t enable) {
+l2pd_status l2pd_set_chain(l2pd_ctx *c, int32_t mode) {
   if (!c) return L2PD_ERR_ARG;
-  c->chain_on = enable != 0;
+  if (mode < 0 || mode > 2) return set_err(c, L2PD_ERR_ARG, "chain mode %d outside [0, 2]", mode);
+  c->chain_mode = mode;
+  c->tc_rows = -1;          // the tiling may change with the mode: output maps and launch tables are rebuilt
+  c->chain_tab_rows = -1;
   return L2PD_OK;
 }
 
@@ -1097,7 +1147,8 @@ static l2pd_status gemm_common(void *stream, int epi, const void *A, const void 
   if (!status) return L2PD_ERR_CUDA;
   const int box = epi == EPI_SWIGLU ? pl.tile_n / 2 : pl.tile_n / pl.cta_group;
   TmaDesc ta, tb, tb2;
-  l2pd_status r = make_tma_2d_bf16(&ta, A, M, K, 128);
+  const int a_box = (M <= 128 && pl.slabs == 1) ? (int)round_up(M, 8) : 128;   // few rows: load only those
+  l2pd_status r = make_tma_2d_bf16(&ta, A, M, K, a_box);
   if (r) return r;
   r = make_tma_2d_bf16(&tb, W, N, K, box);
   if (r) return r;
@@ -1111,7 +1162,7 @@ static l2pd_status gemm_common(void *stream, int epi, const void *A, const void 
   g.c = staged ? &tcm : nullptr;
   g.epi = epi; g.a = &ta; g.b = &tb; g.b2 = epi == EPI_SWIGLU ? &tb2 : nullptr;
   g.M = M; g.N = N; g.K = K; g.tile_n = pl.tile_n; g.cta_group = pl.cta_group; g.k_splits = pl.k_splits;
-  g.slabs = pl.slabs; g.k_interleave = pl.k_interleave;
+  g.slabs = pl.slabs; g.k_interleave = pl.k_interleave; g.a_box_rows = a_box;
   g.out = out; g.status = status;
   { cudaError_t e = launch_gemm_tcgen05((cudaStream_t)stream, g, sms); if (e != cudaSuccess) return standalone_cuda_error("GEMM launch", e); }
   return finish_standalone((cudaStream_t)stream, status, check);
@@ -1147,7 +1198,8 @@ l2pd_status l2pd_lm_head_bf16(void *stream, const void *A, const void *W, const 
   int32_t *status = standalone_status();
   if (!status) return L2PD_ERR_CUDA;
   TmaDesc ta, tb;
-  l2pd_status r = make_tma_2d_bf16(&ta, A, R, K, 128);
+  const int a_box = R <= 128 ? (int)round_up(R, 8) : 128;
+  l2pd_status r = make_tma_2d_bf16(&ta, A, R, K, a_box);
   if (r) return r;
   r = make_tma_2d_bf16(&tb, W, V, K, tile_n);
   if (r) return r;
@@ -1157,7 +1209,7 @@ l2pd_status l2pd_lm_head_bf16(void *stream, const void *A, const void *W, const 
   g.epi = EPI_LMHEAD; g.a = &ta; g.b = &tb; g.M = R; g.N = V; g.K = K; g.tile_n = tile_n;
   g.bias = bias; g.part_m = d_scratch; g.part_s = d_scratch + (int64_t)n_tiles * rows_padded;
   g.part_i = (int32_t *)(g.part_s + (int64_t)n_tiles * rows_padded); g.rows_padded = rows_padded;
-  g.logits = d_logits; g.status = status;
+  g.logits = d_logits; g.status = status; g.a_box_rows = a_box;
   cudaStream_t s = (cudaStream_t)stream;
   if (launch_gemm_tcgen05(s, g, sms) != cudaSuccess) return L2PD_ERR_CUDA;
   if (launch_merge_partials(s, g.part_m, g.part_s, g.part_i, n_tiles, rows_padded, R, d_pred, d_conf) != cudaSuccess)

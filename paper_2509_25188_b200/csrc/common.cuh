@@ -174,6 +174,7 @@ void set_standalone_error(const char *fmt, ...);
 struct GemmPlan { int cta_group, tile_n, k_splits, slabs, k_interleave; };
 // max_tile_n caps the tile width (a kernel that chains several projections keeps one ring geometry for all of them)
 GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, int max_k_splits = 4, int max_tile_n = 256);
+GemmPlan plan_gemm_pair_one_slab(int epi, int M, int N, int K, int num_sms, int max_k_splits, int max_tile_n);
 int effective_k_splits(int K, int k_splits);   // what the launcher makes of a requested K split
 struct GemmArgs {
   int epi;                 // EPI_STORE, EPI_RESIDUAL, EPI_SWIGLU, or EPI_LMHEAD
@@ -185,6 +186,7 @@ struct GemmArgs {
   int cta_group, k_splits; // 0 / 1 = single CTA, no split
   int slabs;               // 0 / 1 = one row slab per unit, 2 = two
   int k_interleave;        // see GemmPlan
+  int a_box_rows;          // 0 / 128: map `a` has a box of 128 rows; M <= 128 only: a box of that many rows (a multiple of 8, >= M)
   void *out;               // bf16 C, fp32 X, or bf16 H
   // LM head
   const float *bias; float *part_m, *part_s; int32_t *part_i; int rows_padded; float *logits;

@@ -4,8 +4,10 @@
 // launch per projection exposes, each time, the launch itself, the ring fill, the accumulator drain and the
 // wait for the slowest CTA.  This kernel keeps the CTAs (one pair of CTAs per SM pair, cta_group::2), their
 // shared-memory ring, their barriers and their tensor memory alive over a list of phases:
-//     GEMM phase   the tiles of one projection, exactly as gemm_tcgen05_pair_kernel runs them with two row
-//                  slabs per unit (same tiling, same epilogues, same K-slice partial sums);
+//     GEMM phase   the tiles of one projection, exactly as gemm_tcgen05_pair_kernel runs them (same tiling, same
+//                  epilogues, same K-slice partial sums): two 256-row slabs per unit, each with its own MMA
+//                  issuer, or — for steps of at most 256 rows — one slab whose k-blocks alternate between the two
+//                  issuers into two accumulators that the epilogue adds;
 //     NORM phase   x += the K slices' partial sums (in slice order), n = RMSNorm(x) for the next projection.
 // Between phases the CTAs meet at a counter in global memory (release add / acquire poll, bounded).  Only the
 // threads that touch what another CTA wrote wait there: the producer of the activation tiles and the
@@ -295,7 +297,7 @@ gemm_chain_kernel(const ChainLaunch cl) {
         const int epi = s_ph[ph].epi;
         const CUtensorMap *tmB = &cp.maps[s_ph[ph].map0 + 1], *tmB2 = &cp.maps[s_ph[ph].map0 + 2];
         const int half_n = p.tile_n >> 1;
-        const uint32_t tx = CG * (a_stage_bytes + (uint32_t)half_n * 128u);
+        const uint32_t tx = (1 + p.a_peer_loads) * (uint32_t)p.slabs * p.a_box_bytes + CG * (uint32_t)half_n * 128u;
         const int num_units = p.m_tiles * p.n_tiles * p.k_splits;
         const int num_kb = (p.K + TILE_K - 1) / TILE_K, kb_per = (num_kb + p.k_splits - 1) / p.k_splits;
         const CUtensorMap *mine = (epi == EPI_SWIGLU) ? (leader ? tmB : tmB2) : tmB;
@@ -319,7 +321,12 @@ gemm_chain_kernel(const ChainLaunch cl) {
       if (!ok) abort_flag = 1;
     }
   } else if (warp == 1 || warp == 2) {
-    // ------------------------------------------------------------------ MMA issuers (leader CTA): warp 1 slab 0, warp 2 slab 1
+    // ------------------------------------------------------------------ MMA issuers (leader CTA)
+    // Two slabs: warp 1 feeds slab 0, warp 2 slab 1 (separate accumulators, no ordering between the two streams).
+    // One slab: the two issuers take alternate k-blocks of the unit into two accumulators (an issuer is limited to
+    // one instruction per ~132 cycles, which alone would bound a K loop of few rows).  Either way BOTH issuers wait
+    // on every stage's `full` barrier and commit once on its `empty` barrier, so every barrier sees the same two
+    // arrivals per use whatever the phase's shape, and no issuer ever skips a barrier phase.
     const int sl = warp - 1;
     if (lane == 0 && leader) {
       uint32_t phases = 0;
@@ -332,6 +339,7 @@ gemm_chain_kernel(const ChainLaunch cl) {
         const uint32_t idesc = ptx::idesc_bf16(TILE_M * CG, (uint32_t)p.tile_n);
         const int num_units = p.m_tiles * p.n_tiles * p.k_splits;
         const int num_kb = (p.K + TILE_K - 1) / TILE_K, kb_per = (num_kb + p.k_splits - 1) / p.k_splits;
+        const bool alternate = p.slabs == 1;
         for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
           int mt, nt, ks, kb0, kb1;
           decode_unit(p, kb_per, num_kb, u, mt, nt, ks, kb0, kb1);
@@ -341,11 +349,14 @@ gemm_chain_kernel(const ChainLaunch cl) {
           for (int kb = kb0; kb < kb1; ++kb) {
             if (!wait_bar(full_bar(stage), (phases >> stage) & 1u)) { fail(g_status, DEV_TIMEOUT_MMA); ok = false; break; }
             ptx::tc_fence_after_sync();
-            const uint64_t a_desc = ptx::smem_desc_sw128(sA + stage * a_stage_bytes + sl * A_STAGE_BYTES);
-            const uint64_t b_desc = ptx::smem_desc_sw128(sB + stage * b_stage_bytes);
+            if (!alternate || ((kb - kb0) & 1) == sl) {
+              const uint64_t a_desc = ptx::smem_desc_sw128(sA + stage * a_stage_bytes + (alternate ? 0 : sl * A_STAGE_BYTES));
+              const uint64_t b_desc = ptx::smem_desc_sw128(sB + stage * b_stage_bytes);
+              const int first_kb = kb0 + (alternate ? sl : 0);       // this accumulator's first k-block
 #pragma unroll
-            for (int k = 0; k < TILE_K / 16; ++k)
-              ptx::mma_bf16_ss_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+              for (int k = 0; k < TILE_K / 16; ++k)
+                ptx::mma_bf16_ss_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb > first_kb || k > 0) ? 1u : 0u);
+            }
             ptx::mma_commit_pair(empty_bar(stage), 3);
             phases ^= 1u << stage;
             if (++stage == n_stages) stage = 0;
@@ -374,10 +385,11 @@ gemm_chain_kernel(const ChainLaunch cl) {
           if (!wait_grid(bar_target(ph - 1))) { fail(g_status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
           fence_proxy_async_all();
         }
-        for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
+        const bool loads_a = leader || p.a_peer_loads;   // few rows: the second CTA of a pair has none
+        for (int u = group; u < num_units && ok && loads_a; u += n_groups, ++lt) {
           int mt, nt, ks, kb0, kb1;
           decode_unit(p, kb_per, num_kb, u, mt, nt, ks, kb0, kb1);
-          const int m0 = mt * (TILE_M * CG * SLABS) + (int)rank * TILE_M;
+          const int m0 = mt * (TILE_M * CG * p.slabs) + (int)rank * TILE_M;
           int stage = 0;
           for (int kb = kb0; kb < kb1; ++kb) {
             // the last two stages' A parts double as the epilogue's staging area: refill them only once the
@@ -386,8 +398,7 @@ gemm_chain_kernel(const ChainLaunch cl) {
             if (!wait_bar(empty_bar(stage), ((phases >> stage) & 1u) ^ 1u)) { fail(g_status, DEV_TIMEOUT_PRODUCER); ok = false; break; }
             const uint32_t dstA = sA + stage * a_stage_bytes;
             const uint32_t lead_full = ptx::mapa(full_bar(stage), 0);
-#pragma unroll
-            for (int sl = 0; sl < SLABS; ++sl)
+            for (int sl = 0; sl < p.slabs; ++sl)
               ptx::tma_load_2d_pair_hint(dstA + sl * A_STAGE_BYTES, tmA, lead_full, kb * TILE_K, m0 + sl * TILE_M * CG, pol_a);
             phases ^= 1u << stage;
             if (++stage == n_stages) stage = 0;
@@ -425,22 +436,27 @@ gemm_chain_kernel(const ChainLaunch cl) {
         for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
           int mt, nt, ks, kb0, kb1;
           decode_unit(p, kb_per, num_kb, u, mt, nt, ks, kb0, kb1);
-          const int row0 = mt * (TILE_M * CG * SLABS) + sl * (TILE_M * CG) + (int)rank * TILE_M + q * 32;
+          const int row0 = mt * (TILE_M * CG * p.slabs) + sl * (TILE_M * CG) + (int)rank * TILE_M + q * 32;
           if (!wait_bar(tfull_bar, (uint32_t)lt & 1u)) { fail(g_status, DEV_TIMEOUT_EPILOGUE); ok = false; break; }
           ptx::tc_fence_after_sync();
           if (etid == 0) { if (u == group) stamp(ph, 1); stamp(ph, 2); }
-          const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + sl * ACC_COLS;
+          const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (p.slabs == 2 ? sl * ACC_COLS : 0);
           const bool res_store = P.epi == EPI_RESIDUAL && p.part != nullptr && p.k_splits > 1;
           const int slice_row0 = res_store ? ks * p.part_rows : 0;
           const uint32_t stage0 = sOut + (uint32_t)(warp - 4) * (4096u * STAGE_BUFS);
-          // every tile goes through the staging area and the TMA unit; the row's last, narrower tile has a map of its own
+          // every tile goes through the staging area and the TMA unit; the row's last, narrower tile has a map of its own.
+          // One-slab phases: the second group of epilogue warps has no rows (it only takes part in the hand-overs below),
+          // and the unit's sum is the two issuers' accumulators added.
           const int tail = nt < p.out_full_tiles ? 0 : p.out_tail_cols;
           const CUtensorMap *tm = tail ? tmC + 1 : tmC;
-          switch (P.epi) {
-            case EPI_QKV_ROPE: drain_tile_staged<EPI_QKV_ROPE>(p, tm, taddr, slice_row0 + row0, nt, stage0, lane, res_store, tail); break;
-            case EPI_RESIDUAL: drain_tile_staged<EPI_RESIDUAL>(p, tm, taddr, slice_row0 + row0, nt, stage0, lane, res_store, tail); break;
-            case EPI_SWIGLU: drain_tile_staged<EPI_SWIGLU>(p, tm, taddr, slice_row0 + row0, nt, stage0, lane, res_store, tail); break;
-            default: drain_tile_staged<EPI_STORE>(p, tm, taddr, slice_row0 + row0, nt, stage0, lane, res_store, tail); break;
+          const bool two_acc = p.slabs == 1;
+          if (sl < p.slabs) {
+            switch (P.epi) {
+              case EPI_QKV_ROPE: drain_tile_staged<EPI_QKV_ROPE>(p, tm, taddr, slice_row0 + row0, nt, stage0, lane, res_store, tail); break;
+              case EPI_RESIDUAL: drain_tile_staged<EPI_RESIDUAL>(p, tm, taddr, slice_row0 + row0, nt, stage0, lane, res_store, tail, two_acc); break;
+              case EPI_SWIGLU: drain_tile_staged<EPI_SWIGLU>(p, tm, taddr, slice_row0 + row0, nt, stage0, lane, res_store, tail, two_acc); break;
+              default: drain_tile_staged<EPI_STORE>(p, tm, taddr, slice_row0 + row0, nt, stage0, lane, res_store, tail, two_acc); break;
+            }
           }
           ptx::tc_fence_before_sync();
           __syncwarp();
@@ -539,8 +555,11 @@ int chain_max_clusters(int num_sms) {
 bool chain_step_supported(const ChainStep &s) {
   if (s.is_norm) return s.nm.d % 4 == 0 && (s.nm.n_part == 0 || (s.nm.n_part >= 2 && s.nm.n_part <= 4));
   const GemmArgs &g = s.g;
-  if (g.cta_group != 2 || g.slabs != 2 || g.k_interleave) return false;
+  // SM pairs; two slabs with an issuer each, or one slab with the two issuers on alternate k-blocks
+  if (g.cta_group != 2) return false;
+  if (!((g.slabs == 2 && !g.k_interleave) || (g.slabs <= 1 && g.k_interleave))) return false;
   if (g.epi != EPI_STORE && g.epi != EPI_QKV_ROPE && g.epi != EPI_RESIDUAL && g.epi != EPI_SWIGLU) return false;
+  if (g.epi == EPI_QKV_ROPE && g.slabs != 2) return false;   // the rotating epilogue does not add two accumulators
   if (g.tile_n < 32 || g.tile_n > 256 || (g.tile_n % 16)) return false;
   // a K split must leave every unit at least a ring's worth of k-blocks (the staging gate is taken once per unit)
   const int ks = effective_k_splits(g.K, g.k_splits);
@@ -591,9 +610,8 @@ cudaError_t chain_build_table(const ChainStep *steps, int n_steps, unsigned int 
       continue;
     }
     const GemmArgs &g = steps[i].g;
-    cudaError_t e = fill_kparams(g, stages, max_b, P.g);
+    cudaError_t e = fill_kparams(g, stages, max_b, P.g, true);
     if (e != cudaSuccess) return e;
-    if (!P.g.gate && P.g.out_tma) return cudaErrorInvalidValue;   // staged stores need the gated staging area
     P.g.status = status;
     P.epi = g.epi;
     if (!P.g.out_tma || (g.N % (g.epi == EPI_SWIGLU ? g.tile_n / 2 : g.tile_n) != 0 && !P.g.out_tail_cols)) return cudaErrorInvalidValue;

@@ -39,6 +39,10 @@ struct KParams {
   const float2 *cs_table;
   const int32_t *row_pos;
   int kil;   // 1: the unit's k-blocks alternate between the two MMA issuers (accumulators 0 and 1, added in the epilogue)
+  // Few rows (M <= 128, one row tile): an activation load brings only a_box_bytes = (M rounded up to 8) x 128 bytes
+  // instead of a whole 128-row tile; the MMA still reads 128 rows, the rest being whatever shared memory holds, into
+  // accumulator rows that are never stored.  a_peer_loads = 0: the second CTA of a pair has no rows and loads none.
+  int a_box_bytes, a_peer_loads;
 };
 
 __device__ __forceinline__ void fail(int32_t *status, int code) {
@@ -396,9 +400,12 @@ __device__ __forceinline__ void emit_swiglu_cols(StagedOut &o, const uint32_t (&
 
 // tail_cols > 0: the row's last, narrower column tile — only its first tail_cols output columns are drained, and tmC
 // is a map of that tile alone (tile coordinate 0, inner extent tail_cols), so boxes are clipped at the row's end.
+// two_acc: the unit's sum is spread over two accumulators ACC_COLS columns apart (two MMA issuers on alternate
+// k-blocks); they are added here, first + second, before the epilogue (not for the rotating epilogue).
 template <int EPI>
 __device__ __forceinline__ void drain_tile_staged(const KParams &p, const CUtensorMap *tmC, uint32_t taddr, int row0,
-                                                  int nt, uint32_t stage0, int lane, bool res_store, int tail_cols = 0) {
+                                                  int nt, uint32_t stage0, int lane, bool res_store, int tail_cols = 0,
+                                                  bool two_acc = false) {
   const int half_n = p.tile_n >> 1;
   StagedOut o(tmC, stage0, lane, tail_cols > 0 ? 0 : nt, row0, EPI == EPI_RESIDUAL && !res_store);
   if (EPI == EPI_QKV_ROPE) {
@@ -424,6 +431,17 @@ __device__ __forceinline__ void drain_tile_staged(const KParams &p, const CUtens
   } else if (EPI == EPI_STORE || EPI == EPI_RESIDUAL) {
     const int n = tail_cols > 0 ? tail_cols : p.tile_n;
     uint32_t va[32], vb[32];
+    if (two_acc) {
+      for (int c = 0; c < n; c += 32) {
+        tmem_load_cols(taddr + c, va, n - c);
+        tmem_load_cols(taddr + ACC_COLS + c, vb, n - c);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) va[i] = __float_as_uint(__uint_as_float(va[i]) + __uint_as_float(vb[i]));
+        emit_cols<EPI>(o, va, c, n);
+      }
+      return;
+    }
     tmem_load_cols(taddr, va, n);
     for (int c = 0; c < n; c += 64) {
       ptx::tmem_ld_wait();
@@ -437,6 +455,22 @@ __device__ __forceinline__ void drain_tile_staged(const KParams &p, const CUtens
   } else {   // EPI_SWIGLU
     const int hn = tail_cols > 0 ? tail_cols : half_n;   // output columns to drain
     uint32_t ga[16], ua[16], gb[16], ub[16];
+    if (two_acc) {
+      for (int c = 0; c < hn; c += 16) {
+        ptx::tmem_ld_x16(taddr + c, ga);
+        ptx::tmem_ld_x16(taddr + half_n + c, ua);
+        ptx::tmem_ld_x16(taddr + ACC_COLS + c, gb);
+        ptx::tmem_ld_x16(taddr + ACC_COLS + half_n + c, ub);
+        ptx::tmem_ld_wait();
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          ga[i] = __float_as_uint(__uint_as_float(ga[i]) + __uint_as_float(gb[i]));
+          ua[i] = __float_as_uint(__uint_as_float(ua[i]) + __uint_as_float(ub[i]));
+        }
+        emit_swiglu_cols(o, ga, ua, c, hn);
+      }
+      return;
+    }
     ptx::tmem_ld_x16(taddr, ga);
     ptx::tmem_ld_x16(taddr + half_n, ua);
     for (int c = 0; c < hn; c += 32) {
@@ -455,6 +489,6 @@ __device__ __forceinline__ void drain_tile_staged(const KParams &p, const CUtens
 
 // Fills the kernel's parameter block for one GEMM (gemm_tcgen05.cu).  stages / b_stage_bytes = 0: the deepest
 // ring the shared memory holds for this tile; otherwise the given ring geometry.
-cudaError_t fill_kparams(const GemmArgs &g, int stages, int b_stage_bytes, gemm_dev::KParams &p);
+cudaError_t fill_kparams(const GemmArgs &g, int stages, int b_stage_bytes, gemm_dev::KParams &p, bool chained = false);
 
 }  // namespace l2pd

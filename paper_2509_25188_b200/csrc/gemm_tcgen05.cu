@@ -128,7 +128,7 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
     if (lane == 0) {
       const uint64_t pol_w = ptx::policy_evict_first();   // weights are read once per step
       const uint32_t b_bytes = (CG == 2) ? (uint32_t)half_n * 128u : (uint32_t)p.tile_n * 128u;
-      const uint32_t tx = CG * (p.a_stage_bytes + b_bytes);
+      const uint32_t tx = (CG == 2 ? (1 + p.a_peer_loads) : 1) * (uint32_t)slabs * p.a_box_bytes + CG * b_bytes;
       auto issue_b = [&](int stage, int kb, int nt) {   // weight tile of k-block kb (and the stage's byte count)
         const uint32_t dstB = sB + stage * p.b_stage_bytes;
         if (CG == 1) {
@@ -259,7 +259,8 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
       uint32_t phases = 0;
       int lt = 0;
       bool ok = true;
-      for (int u = group; u < num_units && ok; u += n_groups, ++lt) {
+      const bool loads_a = leader || p.a_peer_loads;   // few rows: the second CTA of a pair has none
+      for (int u = group; u < num_units && ok && loads_a; u += n_groups, ++lt) {
         int mt, nt, kb0, kb1;
         decode(u, mt, nt, kb0, kb1);
         const int m0 = mt * unit_rows + (int)rank * TILE_M;
@@ -512,6 +513,24 @@ GemmPlan plan_gemm(int epi, int M, int N, int K, int num_sms, int force_tile_n, 
   return best;
 }
 
+// The plan of a step of few rows inside a chained launch: SM pairs, one 256-row slab per unit, the two MMA issuers on
+// alternate k-blocks; tile width and K slices by the same cost model.
+GemmPlan plan_gemm_pair_one_slab(int epi, int M, int N, int K, int num_sms, int max_k_splits, int max_tile_n) {
+  GemmPlan best{2, max_tile_n < 176 ? max_tile_n : 176, 1, 1, 1};
+  double best_cost = 1e300;
+  for (int tn = 256; tn >= 64; tn -= 16) {
+    if (tn > max_tile_n) continue;
+    const int unit_n = epi == EPI_SWIGLU ? tn / 2 : tn;
+    const int max_ks = (epi == EPI_RESIDUAL) ? (max_k_splits < 4 ? max_k_splits : 4) : 1;
+    for (int ks = 1; ks <= max_ks; ++ks) {
+      if (ceil_div(K, TILE_K) < 8 * ks) break;
+      const double c = plan_cost(M, N, K, num_sms, 2, 1, unit_n, tn, ks, epi == EPI_RESIDUAL, true);
+      if (c < best_cost - 1e-9) { best_cost = c; best = GemmPlan{2, tn, ks, 1, 1}; }
+    }
+  }
+  return best;
+}
+
 int lm_head_tile_n(int R, int V, int K, int num_sms) { return plan_gemm(EPI_LMHEAD, R, V, K, num_sms, 0).tile_n; }
 
 int effective_k_splits(int K, int k_splits) {
@@ -524,7 +543,7 @@ int effective_k_splits(int K, int k_splits) {
 
 // Fills the kernel's parameter block for one GEMM.  stages / b_stage_bytes = 0: the deepest ring the shared
 // memory holds for this tile; otherwise the given ring geometry (a kernel that runs several GEMMs keeps one ring).
-cudaError_t fill_kparams(const GemmArgs &g, int stages, int b_stage_bytes, KParams &p) {
+cudaError_t fill_kparams(const GemmArgs &g, int stages, int b_stage_bytes, KParams &p, bool chained) {
   const int cg = g.cta_group == 2 ? 2 : 1;
   if (g.k_splits > 1 && g.epi != EPI_RESIDUAL) return cudaErrorInvalidValue;
   const int ks = effective_k_splits(g.K, g.k_splits);
@@ -534,6 +553,13 @@ cudaError_t fill_kparams(const GemmArgs &g, int stages, int b_stage_bytes, KPara
   p.slabs = g.slabs == 2 ? 2 : 1;
   if (p.slabs == 2 && g.epi == EPI_LMHEAD) return cudaErrorInvalidValue;
   p.a_stage_bytes = p.slabs * A_STAGE_BYTES;
+  p.a_box_bytes = A_STAGE_BYTES;
+  p.a_peer_loads = 1;
+  if (g.a_box_rows > 0 && g.a_box_rows < TILE_M) {
+    if (g.M > TILE_M || p.slabs != 1 || g.a_box_rows < g.M || (g.a_box_rows % 8)) return cudaErrorInvalidValue;
+    p.a_box_bytes = g.a_box_rows * TILE_K * 2;
+  }
+  if (cg == 2 && g.M <= TILE_M) p.a_peer_loads = 0;
   const int stage_bytes = p.a_stage_bytes + p.b_stage_bytes;
   if (stages <= 0) {
     stages = (SMEM_BUDGET - 2048) / stage_bytes;
@@ -546,8 +572,10 @@ cudaError_t fill_kparams(const GemmArgs &g, int stages, int b_stage_bytes, KPara
   const int n_per_tile = (g.epi == EPI_SWIGLU) ? g.tile_n / 2 : g.tile_n;
   // staged output: needs the output map and a staging area (the A part of the ring's last two stages)
   p.kil = g.k_interleave ? 1 : 0;
-  if (p.kil && (p.slabs != 1 || g.epi == EPI_LMHEAD || (stages & 1))) return cudaErrorInvalidValue;
-  p.out_tma = (g.c != nullptr && g.epi != EPI_LMHEAD && stages >= 3 && !p.kil) ? 1 : 0;   // (the two-accumulator sum lives in the direct-store drain)
+  // single GEMM launches: alternate k-blocks <-> alternate stages (even ring), and the two-accumulator sum lives in the
+  // direct-store drain; the chained kernel's issuers see every stage and its staged drain adds the accumulators
+  if (p.kil && (p.slabs != 1 || g.epi == EPI_LMHEAD || (!chained && (stages & 1)))) return cudaErrorInvalidValue;
+  p.out_tma = (g.c != nullptr && g.epi != EPI_LMHEAD && stages >= 3 && (!p.kil || chained)) ? 1 : 0;
   p.out_full_tiles = p.out_tma ? g.N / n_per_tile : 0;
   p.out_tail_cols = 0;
   if (p.out_tma && g.c_tail && g.tail_cols > 0) {

@@ -59,7 +59,8 @@ extern "C" l2pd_status l2pd_lm_head_bf16_static(void *stream, const void *A, con
   const int rows_padded = STATIC_MAX_ROWS;
   if (tile_n < 64 || n_tiles > STATIC_MAX_TILES) return bad(L2PD_ERR_SHAPE, "tile records exceed the built-in scratch");
   TmaDesc ta, tb;
-  r = make_tma_2d_bf16(&ta, A, R, K, 128);
+  const int a_box = (R + 7) / 8 * 8;   // R <= 128: load only the rows there are
+  r = make_tma_2d_bf16(&ta, A, R, K, a_box);
   if (r) return bad(r, "tensor map of A (16-byte aligned pointer, K a multiple of 8)");
   r = make_tma_2d_bf16(&tb, W, V, K, tile_n);
   if (r) return bad(r, "tensor map of W (16-byte aligned pointer, K a multiple of 8)");
@@ -70,7 +71,7 @@ extern "C" l2pd_status l2pd_lm_head_bf16_static(void *stream, const void *A, con
   g.epi = EPI_LMHEAD; g.a = &ta; g.b = &tb; g.M = R; g.N = V; g.K = K; g.tile_n = tile_n;
   g.bias = bias; g.part_m = ptr.scratch; g.part_s = ptr.scratch + (int64_t)n_tiles * rows_padded;
   g.part_i = reinterpret_cast<int32_t *>(g.part_s + (int64_t)n_tiles * rows_padded);
-  g.rows_padded = rows_padded; g.logits = nullptr; g.status = ptr.status;
+  g.rows_padded = rows_padded; g.logits = nullptr; g.status = ptr.status; g.a_box_rows = a_box;
   if (launch_gemm_tcgen05(s, g, sms) != cudaSuccess) return bad(L2PD_ERR_CUDA, "GEMM launch failed");
   if (launch_merge_partials(s, g.part_m, g.part_s, g.part_i, n_tiles, rows_padded, R, d_pred, d_conf) != cudaSuccess)
     return bad(L2PD_ERR_CUDA, "merge launch failed");

@@ -43,6 +43,8 @@ def main():
     ap.add_argument("--layers", type=int, default=2, help="step: number of layers")
     ap.add_argument("--kv-cache", type=int, default=0, help="step: 0 = every step runs all --rows positions; 1 / 2 = prefix / dual "
                     "cache: the timed steps are in-block steps of the first block (at most 31 of them in all)")
+    ap.add_argument("--chain", type=int, default=0, help="step: 0 = one launch per projection, 1 = chained launches (one persistent "
+                    "launch per layer), 2 = the chained form's tiling in single launches")
     ap.add_argument("--impl", type=int, default=0, help="attn: 0 = tcgen05 kernel, 1 = mma.sync kernel")
     ap.add_argument("--ring", type=int, default=0, help="number of weight buffers to rotate through (0 = enough to exceed L2)")
     a = ap.parse_args()
@@ -70,6 +72,7 @@ def main():
         dec = b.Decoder(shape, w, wl.make_filter(32, 0.96, seed=0), block_len=32, max_batch=1, max_seq=T,
                         kv_cache=a.kv_cache, use_filter=a.kv_cache == 0)
         prompts = torch.from_numpy(wl.make_prompts(1, T // 2, shape, seed=1)).to(dev)
+        dec.set_chain(a.chain)
         if a.kv_cache:
             # one commit per step: the first block has 31 steps that read the store
             assert a.warmup + 2 * a.iters <= 31, "at most 31 in-block steps"

@@ -24,7 +24,7 @@ def _device_weights(shape, seed=0):
 
 
 def _steps(dec, prompts, G, n_steps, chain):
-    dec.set_chain(chain)
+    dec.set_chain(int(chain))
     dec.state_reset(prompts, G)
     outs = []
     for _ in range(n_steps):
@@ -72,6 +72,7 @@ def test_chain_trace_records_every_phase():
     dev = _device_weights(shape)
     dec = binding.Decoder(shape, dev, wl.make_filter(32, 0.96, seed=0), block_len=32, max_batch=1, max_seq=512)
     prompts = wl.make_prompts(1, 256, shape, seed=5)
+    dec.set_chain(1)
     dec.chain_trace_enable(True)
     dec.state_reset(prompts, 256)
     dec.denoise_step(outputs=False)
@@ -87,3 +88,35 @@ def test_chain_trace_records_every_phase():
         assert (np.diff(t, axis=1) >= 0).all()   # per CTA: opened <= first ready <= last ready <= finished
         done = t[:, 3].max(axis=1)
         assert (np.diff(done) > 0).all()       # phases finish in order
+
+
+@pytest.mark.parametrize("kv_cache,B,P,G", [(2, 1, 256, 256),     # dual cache: in-block steps of 32 rows
+                                            (2, 8, 96, 64),       # eight sequences: 256 rows per in-block step
+                                            (1, 2, 64, 64)])      # prefix cache: cached steps of 128 rows, then 64
+def test_chained_cached_steps_equal_single_launches(kv_cache, B, P, G):
+    """Key/value-cache configurations: steps of at most 256 rows chain with one row slab per unit and the two MMA issuers
+    on alternate k-blocks.  Mode 2 runs the same tiling as single launches: every output of every step must agree bit for
+    bit, across a block's first step (all rows) and the steps served from the store (including a block change)."""
+    import torch
+    from paper_2509_25188_b200 import binding
+    shape = wl.thin(wl.LLADA_8B, 3)
+    dev = _device_weights(shape)
+    prompts = wl.make_prompts(B, P, shape, seed=9)
+    # no filter: one commit per step, so a block has 32 steps and most of them read the store
+    dec = binding.Decoder(shape, dev, None, block_len=32, max_batch=B, max_seq=P + G, kv_cache=kv_cache, use_filter=False,
+                          lm_head_bias=wl.make_eot_bias(shape, 14.0))
+    n_steps = 36                                   # crosses into the second block
+    launches0 = dec.launch_count
+    a, tok_a = _steps(dec, prompts, G, n_steps, chain=1)
+    launches_chain = dec.launch_count - launches0
+    b, tok_b = _steps(dec, prompts, G, n_steps, chain=2)
+    launches_plain = dec.launch_count - launches0 - launches_chain
+    dec.close()
+    del dev
+    torch.cuda.empty_cache()
+    assert len(a) == len(b) >= 33
+    assert launches_chain < launches_plain - len(a) * 3 * 2          # the chained form really ran on (nearly) every step
+    for k_step, (sa, sb) in enumerate(zip(a, b)):
+        for k in ("logits", "conf", "pred", "p", "unmask", "masks_left", "l_eff", "done", "forced"):
+            assert np.array_equal(sa[k], sb[k]), "step %d: chained and single-launch steps differ in %s" % (k_step, k)
+    assert np.array_equal(tok_a, tok_b)
