@@ -316,7 +316,10 @@ __device__ __forceinline__ void gemm_body(const CUtensorMap *tmA, const CUtensor
       }
     }
     if (!ok) *abort_flag = 1;
-    if (EPI != EPI_LMHEAD && p.out_tma && lane == 0) ptx::bulk_wait_all();   // staged stores are complete before the CTA leaves
+    // The TMA unit must have READ this warp's staging tiles before the CTA's shared memory goes away; the writes themselves
+    // are part of the kernel's memory operations, which complete before the kernel does (and before anything ordered
+    // after it, programmatic dependents included, sees its results).
+    if (EPI != EPI_LMHEAD && p.out_tma && lane == 0) ptx::bulk_wait_read();
   }
 
   // ---------------------------------------------------------------------- teardown

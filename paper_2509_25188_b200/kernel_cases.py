@@ -45,6 +45,8 @@ def main():
                     "cache: the timed steps are in-block steps of the first block (at most 31 of them in all)")
     ap.add_argument("--chain", type=int, default=0, help="step: 0 = one launch per projection, 1 = chained launches (one persistent "
                     "launch per layer), 2 = the chained form's tiling in single launches")
+    ap.add_argument("--trace", action="store_true", help="step with --chain 1: also print the phases' time stamps of the last step "
+                    "(per launch and phase: when the slowest CTA opened it, had its last accumulator ready, finished it)")
     ap.add_argument("--impl", type=int, default=0, help="attn: 0 = tcgen05 kernel, 1 = mma.sync kernel")
     ap.add_argument("--ring", type=int, default=0, help="number of weight buffers to rotate through (0 = enough to exceed L2)")
     a = ap.parse_args()
@@ -157,6 +159,28 @@ def main():
     e1.record()
     torch.cuda.synchronize()
     ms_b2b = e0.elapsed_time(e1) / a.iters
+    if a.case == "step" and a.trace and a.chain == 1:
+        import numpy as np
+        dec.chain_trace_enable(True)
+        run(0)
+        tr = dec.chain_trace()
+        dec.chain_trace_enable(False)
+        if tr is not None:
+            tr = tr.astype(np.int64)
+            names = ["O", "norm2", "gate_up", "down", "norm1", "QKV"]
+            for launch in range(tr.shape[0]):
+                n = 1 if launch == 0 else (6 if launch < tr.shape[0] - 1 else 4)
+                t = tr[launch, :n]
+                t0, prev = t[0, 0].min(), t[0, 0].min()
+                row = []
+                for ph in range(n):
+                    op, r1, r2, fin = t[ph]
+                    busy = r2 > op
+                    row.append({"phase": names[ph] if launch else "QKV", "us": round((fin.max() - prev) / 1e3, 2),
+                                "main_loop_us_median": round(float(np.median((r1 - op)[busy])) / 1e3, 2) if busy.any() else 0.0,
+                                "drain_us_median": round(float(np.median((fin - r2)[busy])) / 1e3, 2) if busy.any() else 0.0})
+                    prev = fin.max()
+                print(json.dumps({"launch": launch, "total_us": round((t[n - 1, 3].max() - t0) / 1e3, 2), "phases": row}))
     print(json.dumps({"case": a.case, "rows": T, "tile_n": a.tile_n, "ms": ms, "ms_back_to_back": ms_b2b, "tflops_b2b": flops / ms_b2b / 1e9, "tflops": flops / ms / 1e9,
                       "gbs": byts / ms / 1e6, "flops": flops, "bytes": byts}))
 
