@@ -247,7 +247,8 @@ def run_ours(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
+    multi = replicas.launcher_env_present()      # started by a launcher (any world size): the process-group path runs
+    if multi:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     torch.cuda.set_device(local)
     dev = "cuda:%d" % local
@@ -262,7 +263,7 @@ def run_ours(args):
     d_prompts = h_prompts.to(dev)
 
     def barrier():
-        if world > 1:
+        if multi:
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -322,13 +323,13 @@ def run_ours(args):
     h_out = torch.empty(1, G, dtype=torch.int32).pin_memory()
     d_one.copy_(h_dec_prompts[0:1])
     dec2.decode_device(d_one, G, d_out)                                # warm-up at the decode's shapes
-    if world > 1:
+    if multi:
         store = dist.distributed_c10d._get_default_store()
     idx, toks, lens, stps = [], [], [], []
     dec_ms = dec_ms_e2e = 0.0
     barrier()
     t_wall0 = time.perf_counter()
-    chunks = replicas.claim_chunks(store, n_dec) if world > 1 else iter(range(n_dec))
+    chunks = replicas.claim_chunks(store, n_dec) if multi else iter(range(n_dec))
     for i in chunks:
         # end to end: the prompt comes from pinned host memory and the response goes back to it, inside the timed region
         ev0.record()
@@ -350,7 +351,7 @@ def run_ours(args):
     barrier()
     wall_ms = 1e3 * (time.perf_counter() - t_wall0)
     toks_np = np.concatenate(toks) if toks else np.zeros((0, G), np.int32)
-    if world > 1:
+    if multi:
         all_toks, all_len, all_steps = replicas.gather_indexed(idx, toks_np, np.array(lens), np.array(stps), n_dec, G, device=dev)
         dec_ms, (_,) = replicas.reduce_timing(dec_ms, [0.0], device=dev)
         dec_ms_e2e, (_,) = replicas.reduce_timing(dec_ms_e2e, [0.0], device=dev)
@@ -441,7 +442,7 @@ def run_ours(args):
                           "directly: %.1f s; tokens = the %d positions that step committed; compare ms_per_step with ms_per_step"
                           % (t_step, n_tok)}
         print(json.dumps(line))
-    if world > 1:
+    if multi:
         dist.barrier()
         dist.destroy_process_group()
 
