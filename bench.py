@@ -429,6 +429,8 @@ def run_ours(args):
 
     if rank == 0 and not args.no_other_configs:
         line["other_configs"] = other_configs(binding, torch, w, filt, pk, dev, local)
+    if rank == 0 and args.extra_workloads:
+        line["extra_workloads"] = extra_workloads(binding, torch, w, filt, dev, local)
 
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
@@ -511,6 +513,83 @@ def other_configs(binding, torch, w, filt, pk, dev, local):
     return out
 
 
+def extra_workloads(binding, torch, w, filt, dev, local):
+    """Long generation with and without EoTP, the threshold / policy sweep on the C2 decode and filter training at the
+    paper's scale (Sections 4.3-4.4, Algorithm 1): behaviour of the loop on the synthetic model, outside the contract's
+    numbers.  --extra-workloads."""
+    B, P, G, s = DEC.batch, DEC.prompt_len, DEC.gen_len, DEC.block_len
+    d_prompts = torch.from_numpy(wl.make_prompts(B, P, SHAPE, seed=1)).to(dev)
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    extra = {}
+    # long generation (the setting of Section 4.3's EoTP study: generation length 1024, block 32): one sequence, the
+    # EoT logit biased so that the answer ends early; the same decode with and without EoTP
+    Pl, Gl, bias_l = 1024, 1024, 14.0
+    pl_ = torch.from_numpy(wl.make_prompts(1, Pl, SHAPE, seed=7)).to(dev)
+    out_l = torch.empty(1, Gl, dtype=torch.int32, device=dev)
+    rec = {"prompt_len": Pl, "gen_len": Gl, "eot_bias": bias_l}
+    for tag, eotp in (("eotp", True), ("no_eotp", False)):
+        decl = binding.Decoder(SHAPE, w, filt, block_len=s, tau=DEC.tau, max_batch=1, max_seq=Pl + Gl, device=local,
+                               use_eotp=eotp, lm_head_bias=wl.make_eot_bias(SHAPE, bias_l))
+        decl.state_reset_device(pl_, Gl)
+        decl.denoise_step_host()                       # warm-up at this shape
+        ev0.record()
+        ol, st_l, tot_l = decl.decode_device(pl_, Gl, out_l)
+        ev1.record()
+        torch.cuda.synchronize()
+        first_eot = (out_l[0] == SHAPE.eot_id).nonzero()
+        rec[tag] = {"ms": ev0.elapsed_time(ev1), "steps": int(tot_l), "out_len": int(ol[0]),
+                    "first_eot": int(first_eot[0]) if len(first_eot) else -1}
+        decl.close()
+    rec["speedup_from_eotp"] = rec["no_eotp"]["ms"] / rec["eotp"]["ms"]
+    extra["long_generation"] = rec
+
+    # threshold sweep (Section 4.4 studies tau = 0.9 ... 0.99) and the comparison policies on the C2 decode: steps and
+    # generated tokens per second of one sequence with the same synthetic model, filter and EoT bias
+    sweep = {}
+    d_out2 = torch.empty(B, G, dtype=torch.int32, device=dev)
+    for tag, kw, rule in [("tau_0.90", {"tau": 0.90}, None), ("tau_0.96", {"tau": 0.96}, None), ("tau_0.99", {"tau": 0.99}, None),
+                          ("confidence_0.9", {"tau": DEC.tau}, ("confidence", 0.9)),
+                          ("one_token_per_step", {"tau": DEC.tau}, ("confidence", 1.0))]:
+        decs = binding.Decoder(SHAPE, w, filt, block_len=s, max_batch=B, max_seq=P + G, device=local,
+                               lm_head_bias=wl.make_eot_bias(SHAPE, 14.0), **kw)
+        if rule:
+            decs.set_unmask_rule(rule[0], conf_threshold=rule[1])
+        decs.state_reset_device(d_prompts, G)
+        decs.denoise_step_host()
+        ev0.record()
+        ol, st_s, tot_s = decs.decode_device(d_prompts, G, d_out2)
+        ev1.record()
+        torch.cuda.synchronize()
+        ms_s = ev0.elapsed_time(ev1)
+        sweep[tag] = {"steps": int(tot_s), "out_len": int(ol[0]), "ms": ms_s,
+                      "generated_tokens_per_s": float(np.sum(ol)) / (ms_s * 1e-3)}
+        decs.close()
+    base_steps = sweep["one_token_per_step"]["steps"]
+    for v in sweep.values():
+        v["steps_vs_one_token_per_step"] = base_steps / max(v["steps"], 1)
+    extra["policy_sweep_C2"] = sweep
+
+    # filter training at the paper's scale (Section 4.1: 2,640 prompts, 5,000 epochs, lr 0.001): synthetic samples,
+    # one per decoding step of a 32-step-per-prompt EGP run; the whole of stage 2 on the device
+    n_samp = 2640 * 32
+    rng = np.random.default_rng(0)
+    c_s = rng.uniform(0.0, 1.0, size=(n_samp, s)).astype(np.float32)
+    y_s = (c_s + 0.15 * rng.normal(size=(n_samp, s)) > 0.6).astype(np.uint8)
+    tc_s, ty_s = torch.from_numpy(c_s).to(dev), torch.from_numpy(y_s).to(dev)
+    binding.filter_train(filt, tc_s, ty_s, 20)
+    ev0.record()
+    _, tr_losses = binding.filter_train(filt, tc_s, ty_s, 5000)
+    ev1.record()
+    torch.cuda.synchronize()
+    ms_tr = ev0.elapsed_time(ev1)
+    fl_epoch = 10.0 * n_samp * s * s        # two products forward, three backward, 2 flops per multiply-add
+    extra["filter_training"] = {"samples": n_samp, "block_len": s, "epochs": 5000, "batch": "full", "ms": ms_tr,
+                                "us_per_epoch": 1e3 * ms_tr / 5000, "gflops": fl_epoch * 5000 / (ms_tr * 1e-3) / 1e9,
+                                "loss_first": float(tr_losses[0]), "loss_last": float(tr_losses[-1])}
+
+    return extra
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -518,6 +597,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true", help="skip the oracle timing leg")
+    ap.add_argument("--extra-workloads", action="store_true",
+                    help="also run the long-generation pair (with / without EoTP), the threshold and policy sweep on the C2 decode "
+                         "and filter training at the paper's scale; reported under extra_workloads, outside the contract's numbers")
     ap.add_argument("--no-other-configs", action="store_true",
                     help="skip the steps of the batched configurations (C3, C4) and of the dual cache")
     args = ap.parse_args()
