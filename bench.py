@@ -395,8 +395,11 @@ def run_ours(args):
             "step_roofline": {"flops": work["flops"], "weight_bytes": work["weight_bytes"], "act_bytes": work["act_bytes"],
                               "bound": bound, "t_bytes_ms": t_bytes, "t_roof_ms": t_burst, "frac": t_burst / ms_step,
                               "t_roof_sustained_ms": t_sust, "frac_sustained": t_sust / ms_step,
+                              "mcycles_per_step": (ms_step * clocks["sm_mhz"] / 1e3) if clocks and clocks.get("sm_mhz") else None,
                               "note": "frac: against the burst bf16 figure (the target's denominator); frac_sustained: against the "
-                                      "seconds-long figure under the power cap",
+                                      "seconds-long figure under the power cap; mcycles_per_step: ms_per_step x the median SM clock "
+                                      "sampled during the timed region (what the step costs in SM cycles, whatever clock the power "
+                                      "cap allowed)",
                               "peaks": pk, "peak_source": pk_src},
             "decode": {"workload": "C2: full Learn2PD decode, prompt %d + generation %d, block %d, filter + EoTP, EoT logit biased "
                                    "by the constant %.1f; %d sequences (2 per rank, taken from a shared queue)" % (P, G, s, EOT_BIAS, n_dec),

@@ -48,6 +48,8 @@ def main():
     ap.add_argument("--trace", action="store_true", help="step with --chain 1: also print the phases' time stamps of the last step "
                     "(per launch and phase: when the slowest CTA opened it, had its last accumulator ready, finished it)")
     ap.add_argument("--impl", type=int, default=0, help="attn: 0 = tcgen05 kernel, 1 = mma.sync kernel")
+    ap.add_argument("--sustain", type=float, default=0.0, help="also run the launches back to back for this many seconds while the "
+                    "SM clock is sampled (NVML, read-only): time per launch, median MHz and their product in the power-capped state")
     ap.add_argument("--ring", type=int, default=0, help="number of weight buffers to rotate through (0 = enough to exceed L2)")
     a = ap.parse_args()
     dev = "cuda:0"
@@ -159,6 +161,34 @@ def main():
     e1.record()
     torch.cuda.synchronize()
     ms_b2b = e0.elapsed_time(e1) / a.iters
+    sustained = None
+    if a.sustain > 0:
+        import statistics
+        import threading
+        import time
+        import pynvml
+        pynvml.nvmlInit()
+        h = pynvml.nvmlDeviceGetHandleByIndex(torch.cuda.current_device())
+        n = max(a.iters, int(a.sustain * 1e3 / ms_b2b))
+        mhz, stop = [], threading.Event()
+
+        def sample():
+            while not stop.is_set():
+                mhz.append(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+                time.sleep(0.02)
+        th = threading.Thread(target=sample)
+        th.start()
+        e0.record()
+        for i in range(n):
+            run(i)
+        e1.record()
+        torch.cuda.synchronize()
+        stop.set()
+        th.join()
+        us = e0.elapsed_time(e1) / n * 1e3
+        med = statistics.median(mhz[len(mhz) // 3:]) if len(mhz) >= 3 else None   # the clock settles within the first third
+        sustained = {"launches": n, "us": us, "sm_mhz_median": med, "kcycles": us * med / 1e3 if med else None,
+                     "tflops": flops / us / 1e6}
     if a.case == "step" and a.trace and a.chain == 1:
         import numpy as np
         dec.chain_trace_enable(True)
@@ -182,7 +212,7 @@ def main():
                     prev = fin.max()
                 print(json.dumps({"launch": launch, "total_us": round((t[n - 1, 3].max() - t0) / 1e3, 2), "phases": row}))
     print(json.dumps({"case": a.case, "rows": T, "tile_n": a.tile_n, "ms": ms, "ms_back_to_back": ms_b2b, "tflops_b2b": flops / ms_b2b / 1e9, "tflops": flops / ms / 1e9,
-                      "gbs": byts / ms / 1e6, "flops": flops, "bytes": byts}))
+                      "gbs": byts / ms / 1e6, "flops": flops, "bytes": byts, "sustained": sustained}))
 
 
 if __name__ == "__main__":
