@@ -513,6 +513,28 @@ def other_configs(binding, torch, w, filt, pk, dev, local):
         out[name] = dict(rows=rows, first_step_ms=t_first,
                          in_block_step=frac(step_work(SHAPE, rows, Px + Gx, Bx * s, kv), statistics.median(times)))
         decx.close()
+    # the C2 decode of the headline (filter + EoTP, same prompts and EoT bias) with the key/value caches of Section 4.3
+    dsh = wl.DECODES["C2"]
+    prompts = torch.from_numpy(wl.make_prompts(2, dsh.prompt_len, SHAPE, seed=1)).to(dev)
+    d_out = torch.empty(1, dsh.gen_len, dtype=torch.int32, device=dev)
+    bias = wl.make_eot_bias(SHAPE, EOT_BIAS)
+    for mode, key in ((1, "C2_decode_prefix_cache"), (2, "C2_decode_dual_cache")):
+        decx = binding.Decoder(SHAPE, w, filt, block_len=s, tau=dsh.tau, max_batch=1, max_seq=dsh.prompt_len + dsh.gen_len,
+                               device=local, kv_cache=mode, lm_head_bias=bias)
+        decx.decode_device(prompts[0:1], dsh.gen_len, d_out)      # warm-up
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        lens, steps = [], []
+        ev0.record()
+        for i in range(2):
+            ln, st, _ = decx.decode_device(prompts[i:i + 1], dsh.gen_len, d_out)
+            lens.append(int(ln[0])); steps.append(int(st[0]))
+        ev1.record()
+        torch.cuda.synchronize()
+        ms = ev0.elapsed_time(ev1)
+        out[key] = {"sequences": 2, "out_len": lens, "steps": steps, "ms": ms, "generated_tokens_per_s": sum(lens) / (ms * 1e-3),
+                    "note": "the cached steps approximate the keys and values of positions outside the current block, so the "
+                            "trajectory (steps, length) differs from the uncached decode's"}
+        decx.close()
     return out
 
 
